@@ -1,0 +1,190 @@
+/*
+ * ones.h — C ABI of the B200 evolutionary batch-size search (ONES, SC'21).
+ *
+ * One scheduling round of ONES scores a population of candidate schedules and
+ * evolves it (paper, Section 3.2.2: initialisation, uniform crossover, uniform
+ * mutation, selection, update with the best candidate S*).  This library runs
+ * that loop on one GPU.  A candidate S (Eq. 1-2) is one row of int32 exponents,
+ * one per job: job j runs with global batch B_j = b0_j << k_j on
+ * c_j = ceil(B_j / max_per_gpu_j) GPUs; a gene outside [0, kmax_j] means the job
+ * waits (B_j = c_j = 0, text after Eq. 2).
+ *
+ * Conventions
+ *  - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global
+ *    memory of the device that was current at ones_create.  The caller owns every
+ *    buffer it passes, including the device workspace; the handle owns only small
+ *    host-side state.  Nothing here allocates or frees device memory.
+ *  - Genome tables are row-major int32[n][ld], ld >= number of jobs, ld % 4 == 0,
+ *    base address 16-byte aligned.  Columns >= number of jobs are never read as
+ *    genes and never written.
+ *  - All work is enqueued on the CUDA stream given to ones_create.  Calls that
+ *    return data to host memory synchronise that stream; the others do not.
+ *  - Every function returns ONES_OK (0) or a negative ONES_ERR_* code.  Nothing is
+ *    printed, nothing aborts.  An asynchronous CUDA fault surfaces as
+ *    ONES_ERR_CUDA at the next synchronising call.
+ *  - A handle is not thread-safe; different handles may be used from different
+ *    threads.
+ */
+#ifndef ONES_H
+#define ONES_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ones_ctx ones_ctx;
+
+/* One job of the set J (Table 1).  b0 << k, k in [kmin, kmax], is the batch-size
+ * grid and b0 << kmax the batch-size limit R_j (Section 3.2.2, "Evolution");
+ * a, c, d are the coefficients of the job's profiled throughput X_j (Eq. 5):
+ * seconds per iteration t = a + c * (B / g) + d * log2(g) on g GPUs, X = B / t.
+ * weight is the per-job factor Y_processed * (1/rho - 1) of Alg. 1's score; it is
+ * used only with ONES_FLAG_SRUF.  48 bytes. */
+typedef struct {
+    int32_t b0, max_per_gpu, kmin, kmax;
+    double a, c, d, weight;
+} ones_job;
+
+/* Search parameters.  elitism: candidates that survive unchanged per generation;
+ * tournament: draws per parent; p_mut: mutation rate theta per gene ("Uniform
+ * mutation"); penalty: score lost per GPU above the cluster's capacity (Eq. 4 as a
+ * soft constraint).  NULL where a ones_params* is expected means {2, 4, 0.1, 1e3, 0}. */
+typedef struct {
+    int32_t elitism, tournament;
+    double p_mut, penalty;
+    uint32_t flags;
+} ones_params;
+
+/* Score = -(sum_j weight_j * c_j / X_j): Alg. 1 / Eq. 8 (smallest remaining
+ * utilisation first), negated so that higher is better.  Default score:
+ * sum_j X_j (predicted cluster progress in samples per second). */
+#define ONES_FLAG_SRUF 1u
+
+#define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
+#define ONES_MAX_ELITES 256   /* elitism <= 256 */
+
+enum {
+    ONES_OK = 0,
+    ONES_ERR_NULL = -1,       /* a required pointer is NULL */
+    ONES_ERR_BAD_JOB = -2,    /* a job row violates the limits listed at ones_create */
+    ONES_ERR_BAD_PARAM = -3,  /* a scalar argument or ones_params field is out of range */
+    ONES_ERR_ALIGN = -4,      /* pointer not 16-byte aligned or ld % 4 != 0 */
+    ONES_ERR_WORKSPACE = -5,  /* workspace too small for this population / job count */
+    ONES_ERR_CUDA = -6,       /* a CUDA call failed; see ones_last_cuda_error */
+    ONES_ERR_INFEASIBLE = -7, /* repair could not reach the capacity */
+    ONES_ERR_NOMEM = -8       /* host allocation failed */
+};
+
+/* Bytes of device workspace needed for up to n_jobs_max jobs and a population of
+ * pop candidates (two population buffers, fitness, parents, model tables,
+ * scratch).  Returns 0 when an argument is out of range. */
+size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop);
+
+/* Create a search over `n_jobs` jobs on a cluster of `capacity` GPUs with a
+ * population of `pop` candidates (Section 3.2.2 "Initialization": the population
+ * G_0 of simple solutions — every job at its smallest batch, gene kmin_j).
+ *   jobs        host, n_jobs rows.  Required per row: b0 > 0, max_per_gpu > 0,
+ *               0 <= kmin <= kmax <= 15, b0 << kmax < 2^31, a, c, d finite and >= 0,
+ *               t > 0 for every k; else ONES_ERR_BAD_JOB.
+ *   capacity    |C| > 0.   pop >= elitism + 1.   tournament >= 1.   0 <= p_mut <= 1.
+ *   d_workspace device, 256-byte aligned, at least ones_workspace_bytes(n_jobs, pop)
+ *               bytes; a larger workspace lets ones_update_jobs grow the job set up
+ *               to the n_jobs_max it was sized for.
+ *   cuda_stream a cudaStream_t (NULL = the default stream).
+ * Builds the per-(job, exponent) throughput table on the device. */
+int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t capacity, int32_t pop,
+                const ones_params* prm, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Frees the handle's host state.  The workspace stays the caller's. */
+int ones_destroy(ones_ctx* ctx);
+
+/* Replace the population: candidate 0 keeps every job at kmin, every other gene is
+ * drawn uniformly from [kmin_j, kmax_j] (Philox stream keyed by seed, row, job). */
+int ones_randomize(ones_ctx* ctx, uint64_t seed);
+
+/* Copy a population of pop rows in (out of) the handle.  `genomes` is device
+ * memory if on_device != 0, host memory otherwise (then the call synchronises). */
+int ones_set_population(ones_ctx* ctx, const int32_t* genomes, int64_t ld, int on_device);
+int ones_get_population(ones_ctx* ctx, int32_t* genomes, int64_t ld, int on_device);
+
+/* Score candidates (Alg. 1's score step, Eq. 8; capacity constraint Eq. 4):
+ *   gpus[i]    = sum_j c_j                      (int32, wraps modulo 2^32)
+ *   fitness[i] = sum_j term_j - penalty * max(0, gpus[i] - capacity)   (fp64)
+ * with the sum taken in a fixed order: 32 partial sums, job j added to partial
+ * (j / 4) % 32 in increasing j, then a pairwise tree (16, 8, 4, 2, 1) over them.
+ *   d_genomes  device int32[n][ld], or NULL for the handle's current population
+ *              (then ld and n are ignored and n = pop).
+ *   d_fitness  device double[n];  d_gpus device int32[n] or NULL. */
+int ones_evaluate(ones_ctx* ctx, const int32_t* d_genomes, int64_t ld, int32_t n, double* d_fitness,
+                  int32_t* d_gpus);
+
+/* Run `generations` generations (Fig. 4: G_i -> G'_i -> G_{i+1}).  Each one: the
+ * `elitism` best candidates (score descending, index ascending) move unchanged to
+ * rows 0..E-1; for every pair of remaining rows two parents are chosen by
+ * tournament, uniform crossover gives two complementary children ("Uniform
+ * crossover"), each child gene is then redrawn uniformly in [kmin_j, kmax_j] with
+ * probability p_mut ("Uniform mutation"), and the new population is scored.
+ * Random draws come from Philox4x32-10 keyed by (seed; generation, row, job), the
+ * generation counted from ones_create, so evolve(a + b) equals evolve(a) then
+ * evolve(b).  Asynchronous. */
+int ones_evolve(ones_ctx* ctx, int32_t generations, uint64_t seed);
+
+/* The best candidate S* of the current population (Alg. 1, last step), optionally
+ * repaired to fit the cluster: while the GPU demand exceeds the capacity the job
+ * holding the most GPUs (lowest index on ties) that can still shrink goes down one
+ * exponent; when none can, running jobs wait (gene -1) in increasing index.
+ * Host outputs, each nullable: h_genome int32[n_jobs], h_gpus_per_job int32[n_jobs],
+ * h_rate_per_job double[n_jobs] (X_j of the returned genes), fitness, total_gpus,
+ * index (row of the population).  With repair the fitness is that of the repaired
+ * row.  Synchronises. */
+int ones_best(ones_ctx* ctx, int repair, int32_t* h_genome, int32_t* h_gpus_per_job,
+              double* h_rate_per_job, double* fitness, int32_t* total_gpus, int32_t* index);
+
+/* New scheduling round with a changed job set (Section 3.2.2 "Refresh": finished
+ * jobs leave, new jobs arrive, limits R_j move).  Column j of the new population is
+ * column remap[j] of the old one clamped into the new [kmin_j, kmax_j], or kmin_j
+ * when remap[j] == -1; the model tables are rebuilt.  jobs, remap: host, n_jobs
+ * entries; n_jobs must fit the workspace.  Asynchronous apart from argument checks. */
+int ones_update_jobs(ones_ctx* ctx, const ones_job* jobs, int32_t n_jobs, const int32_t* remap,
+                     int32_t capacity);
+
+/* Parents [pairs][2] and elites [elitism] chosen in the last generation (host
+ * outputs, nullable); pairs = (pop - elitism + 1) / 2.  Synchronises. */
+int ones_last_parents(ones_ctx* ctx, int32_t* h_parents, int32_t* h_elites);
+
+/* The device-built model table: X[k][j] and g[k][j] for k = 0..kmax_max (host
+ * outputs, row length n_jobs; entries with k > kmax_j are 0).  *planes receives
+ * kmax_max + 1.  Pass NULL arrays to query *planes only.  Synchronises. */
+int ones_model_table(ones_ctx* ctx, double* h_X, int32_t* h_g, int32_t* planes);
+
+/* Indices of the e best of n scores (descending, ties to the lower index), the
+ * selection step on its own.  d_scratch: device, >= ones_select_top_scratch_bytes(n, e),
+ * 16-byte aligned.  1 <= e <= min(n, ONES_MAX_ELITES).  Asynchronous on `cuda_stream`. */
+size_t ones_select_top_scratch_bytes(int32_t n, int32_t e);
+int ones_select_top(const double* d_fitness, int32_t n, int32_t e, int32_t* d_index,
+                    void* d_scratch, size_t scratch_bytes, void* cuda_stream);
+
+/* Absolute generation counter, jobs and population of the handle. */
+int ones_generation(const ones_ctx* ctx, uint64_t* gen_abs);
+int ones_shape(const ones_ctx* ctx, int32_t* n_jobs, int32_t* pop, int32_t* capacity, int64_t* ld);
+
+/* Kernel launches issued through this handle so far. */
+int ones_kernel_launches(const ones_ctx* ctx, uint64_t* launches);
+
+/* Per-stage device time.  With profiling on, ones_evolve and ones_evaluate bracket
+ * each kernel with CUDA events.  ones_stage_times synchronises and returns, for
+ * stage s in {0 fitness, 1 select+elites, 2 evolve}, the summed milliseconds
+ * ms[s] and launch counts count[s] since the last call, then clears them. */
+int ones_set_profiling(ones_ctx* ctx, int on);
+int ones_stage_times(ones_ctx* ctx, double ms[3], uint64_t count[3]);
+
+/* The cudaError_t of the last failed CUDA call of this handle (0 if none). */
+int ones_last_cuda_error(const ones_ctx* ctx);
+const char* ones_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

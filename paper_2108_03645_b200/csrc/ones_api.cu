@@ -1,0 +1,557 @@
+// C ABI of the evolutionary batch-size search: argument checks, workspace layout, launch order.
+// All arithmetic of the method runs in the kernels of ones_kernels.cu.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "ones.h"
+#include "ones_internal.h"
+
+using namespace ones;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int32_t kPlanesMax = ONES_MAX_EXPONENT + 2;  // exponents 0..15 and the waiting plane
+constexpr int32_t kJobsLimit = 1 << 20;
+constexpr int32_t kPopLimit = 1 << 28;
+
+inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
+inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
+
+struct Layout {
+    size_t pop0, pop1, F, G, parents, elites, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
+        out_gpus, out_rate, out_rec, exp_X, exp_G, status, total;
+};
+
+Layout make_layout(int32_t jmax, int32_t pop) {
+    Layout L;
+    size_t at = 0;
+    auto take = [&](size_t bytes) {
+        size_t here = at;
+        at = up(at + bytes, kAlign);
+        return here;
+    };
+    const size_t ldm = (size_t)ld_of(jmax), jp = (size_t)jpad_of(jmax);
+    const size_t pairs = ((size_t)pop + 1) / 2;
+    L.pop0 = take((size_t)pop * ldm * 4);
+    L.pop1 = take((size_t)pop * ldm * 4);
+    L.F = take((size_t)pop * 8);
+    L.G = take((size_t)pop * 4);
+    L.parents = take(pairs * 2 * 4);
+    L.elites = take((size_t)ONES_MAX_ELITES * 4);
+    L.best_idx = take(16);
+    L.X = take((size_t)kPlanesMax * jp * 8);
+    L.Gt = take((size_t)kPlanesMax * jp * 4);
+    L.kmin = take(jp * 4);
+    L.range = take(jp * 4);
+    L.jobs = take((size_t)jmax * sizeof(ones_job));
+    L.remap = take((size_t)jmax * 4);
+    L.top = take(top_scratch_bytes(pop, ONES_MAX_ELITES));
+    L.work = take(3 * jp * 4);
+    L.out_genome = take((size_t)jmax * 4);
+    L.out_gpus = take((size_t)jmax * 4);
+    L.out_rate = take((size_t)jmax * 8);
+    L.out_rec = take(sizeof(BestOut));
+    L.exp_X = take((size_t)(kPlanesMax - 1) * jmax * 8);
+    L.exp_G = take((size_t)(kPlanesMax - 1) * jmax * 4);
+    L.status = take(16);
+    L.total = at;
+    return L;
+}
+
+struct Prof {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> stage;  // stage of event pair i
+    size_t used = 0;         // events recorded since the last flush
+    double ms[3] = {0, 0, 0};
+    uint64_t count[3] = {0, 0, 0};
+};
+
+}  // namespace
+
+struct ones_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int32_t J = 0, Jmax = 0, N = 0, cap = 0, pairs = 0;
+    int64_t ld = 0;
+    ones_params prm{};
+    uint32_t thr16 = 0;
+    char* ws = nullptr;
+    Layout L{};
+    int cur = 0;
+    bool f_valid = false;
+    uint64_t gen = 0;
+    Tables tab{};
+    std::vector<ones_job> h_jobs;  // the job table the device tables were built from
+    uint64_t launches = 0;
+    int last_cuda = 0;
+    Prof prof;
+
+    int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
+    double* F() { return reinterpret_cast<double*>(ws + L.F); }
+    int32_t* G() { return reinterpret_cast<int32_t*>(ws + L.G); }
+    int32_t* parents() { return reinterpret_cast<int32_t*>(ws + L.parents); }
+    int32_t* elites() { return reinterpret_cast<int32_t*>(ws + L.elites); }
+    int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
+    ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs); }
+    int32_t* remap() { return reinterpret_cast<int32_t*>(ws + L.remap); }
+    int32_t* status() { return reinterpret_cast<int32_t*>(ws + L.status); }
+};
+
+namespace {
+
+int cuda_fail(ones_ctx* c, cudaError_t e) {
+    if (c) c->last_cuda = (int)e;
+    return ONES_ERR_CUDA;
+}
+
+#define CU(c, call)                                     \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess) return cuda_fail(c, e_); \
+    } while (0)
+
+int check_jobs(const ones_job* jobs, int32_t n) {
+    if (!jobs) return ONES_ERR_NULL;
+    if (n <= 0 || n > kJobsLimit) return ONES_ERR_BAD_JOB;
+    for (int32_t j = 0; j < n; ++j) {
+        const ones_job& q = jobs[j];
+        if (q.b0 <= 0 || q.max_per_gpu <= 0) return ONES_ERR_BAD_JOB;
+        if (q.kmin < 0 || q.kmin > q.kmax || q.kmax > ONES_MAX_EXPONENT) return ONES_ERR_BAD_JOB;
+        if (((int64_t)q.b0 << q.kmax) >= ((int64_t)1 << 31)) return ONES_ERR_BAD_JOB;
+        if (!(q.a >= 0.0) || !(q.c >= 0.0) || !(q.d >= 0.0)) return ONES_ERR_BAD_JOB;
+        if (!isfinite(q.a) || !isfinite(q.c) || !isfinite(q.d) || !isfinite(q.weight)) return ONES_ERR_BAD_JOB;
+    }
+    return ONES_OK;
+}
+
+int check_params(const ones_params& p, int32_t pop) {
+    if (p.elitism < 0 || p.elitism > ONES_MAX_ELITES || p.tournament < 1) return ONES_ERR_BAD_PARAM;
+    if (pop < p.elitism + 1) return ONES_ERR_BAD_PARAM;
+    if (!(p.p_mut >= 0.0 && p.p_mut <= 1.0)) return ONES_ERR_BAD_PARAM;
+    if (!isfinite(p.penalty)) return ONES_ERR_BAD_PARAM;
+    return ONES_OK;
+}
+
+uint32_t threshold16(double p) {
+    long t = lround(p * 65536.0);
+    if (t < 0) t = 0;
+    if (t > 65536) t = 65536;
+    return (uint32_t)t;
+}
+
+void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
+    int32_t kmax = 0;
+    for (int32_t j = 0; j < n_jobs; ++j) kmax = jobs[j].kmax > kmax ? jobs[j].kmax : kmax;
+    c->tab.X = reinterpret_cast<double*>(c->ws + c->L.X);
+    c->tab.G = reinterpret_cast<int32_t*>(c->ws + c->L.Gt);
+    c->tab.kmin = reinterpret_cast<int32_t*>(c->ws + c->L.kmin);
+    c->tab.range = reinterpret_cast<int32_t*>(c->ws + c->L.range);
+    c->tab.jpad = jpad_of(n_jobs);
+    c->tab.k1 = kmax + 1;
+}
+
+// ---- per-stage timing with CUDA events on the handle's stream ----
+int prof_flush(ones_ctx* c) {
+    Prof& p = c->prof;
+    if (p.used == 0) return ONES_OK;
+    CU(c, cudaStreamSynchronize(c->stream));
+    for (size_t i = 0; i + 1 < p.used; i += 2) {
+        float ms = 0.f;
+        CU(c, cudaEventElapsedTime(&ms, p.ev[i], p.ev[i + 1]));
+        const int s = p.stage[i / 2];
+        p.ms[s] += (double)ms;
+        p.count[s] += 1;
+    }
+    p.used = 0;
+    return ONES_OK;
+}
+
+int prof_begin(ones_ctx* c, int stage) {
+    Prof& p = c->prof;
+    if (!p.on) return ONES_OK;
+    if (p.used + 2 > p.ev.size()) {
+        int rc = prof_flush(c);
+        if (rc) return rc;
+    }
+    p.stage[p.used / 2] = stage;
+    CU(c, cudaEventRecord(p.ev[p.used], c->stream));
+    return ONES_OK;
+}
+
+int prof_end(ones_ctx* c) {
+    Prof& p = c->prof;
+    if (!p.on) return ONES_OK;
+    CU(c, cudaEventRecord(p.ev[p.used + 1], c->stream));
+    p.used += 2;
+    return ONES_OK;
+}
+
+int run_fitness(ones_ctx* c) {
+    int rc = prof_begin(c, 0);
+    if (rc) return rc;
+    CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
+                         c->stream));
+    c->launches += 1;
+    c->f_valid = true;
+    return prof_end(c);
+}
+
+int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs) {
+    CU(c, cudaMemsetAsync(c->status(), 0, 16, c->stream));
+    CU(c, cudaMemcpyAsync(c->jobs(), h_jobs, sizeof(ones_job) * (size_t)n_jobs, cudaMemcpyHostToDevice, c->stream));
+    set_tables(c, h_jobs, n_jobs);
+    CU(c, launch_build_tables(c->jobs(), n_jobs, c->prm.flags, c->tab, c->status(), c->stream));
+    c->launches += 1;
+    int32_t bad = 0;
+    CU(c, cudaMemcpyAsync(&bad, c->status(), 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    if (bad) return ONES_ERR_BAD_JOB;  // some job has a non-positive or non-finite throughput
+    try {
+        c->h_jobs.assign(h_jobs, h_jobs + n_jobs);
+    } catch (...) {
+        return ONES_ERR_NOMEM;
+    }
+    return ONES_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop) {
+    if (n_jobs_max <= 0 || n_jobs_max > kJobsLimit || pop <= 0 || pop > kPopLimit) return 0;
+    return make_layout(n_jobs_max, pop).total;
+}
+
+int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t capacity, int32_t pop,
+                const ones_params* prm, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!out) return ONES_ERR_NULL;
+    *out = nullptr;
+    if (!jobs || !d_workspace) return ONES_ERR_NULL;
+    int rc = check_jobs(jobs, n_jobs);
+    if (rc) return rc;
+    ones_params p = {2, 4, 0.1, 1e3, 0};
+    if (prm) p = *prm;
+    if (capacity <= 0 || pop <= 0 || pop > kPopLimit) return ONES_ERR_BAD_PARAM;
+    rc = check_params(p, pop);
+    if (rc) return rc;
+    if ((reinterpret_cast<uintptr_t>(d_workspace) & (kAlign - 1)) != 0) return ONES_ERR_ALIGN;
+    if (workspace_bytes < make_layout(n_jobs, pop).total) return ONES_ERR_WORKSPACE;
+    // the largest job count this workspace can hold
+    int32_t lo = n_jobs, hi = kJobsLimit;
+    while (lo < hi) {
+        const int32_t mid = lo + (hi - lo + 1) / 2;
+        if (make_layout(mid, pop).total <= workspace_bytes) lo = mid;
+        else hi = mid - 1;
+    }
+    ones_ctx* c = new (std::nothrow) ones_ctx();
+    if (!c) return ONES_ERR_NOMEM;
+    c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    c->J = n_jobs;
+    c->Jmax = lo;
+    c->N = pop;
+    c->cap = capacity;
+    c->prm = p;
+    c->thr16 = threshold16(p.p_mut);
+    c->pairs = (pop - p.elitism + 1) / 2;
+    c->ld = ld_of(n_jobs);
+    c->ws = reinterpret_cast<char*>(d_workspace);
+    c->L = make_layout(c->Jmax, pop);
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e != cudaSuccess) {
+        delete c;
+        return ONES_ERR_CUDA;
+    }
+    rc = rebuild_tables(c, jobs, n_jobs);
+    if (rc == ONES_OK) {
+        e = launch_fill_min(c->pop(0), c->ld, c->N, c->J, c->tab, c->stream);
+        c->launches += 1;
+        if (e != cudaSuccess) rc = cuda_fail(c, e);
+    }
+    if (rc != ONES_OK) {
+        delete c;
+        return rc;
+    }
+    c->cur = 0;
+    c->f_valid = false;
+    *out = c;
+    return ONES_OK;
+}
+
+int ones_destroy(ones_ctx* c) {
+    if (!c) return ONES_OK;
+    for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
+    delete c;
+    return ONES_OK;
+}
+
+int ones_randomize(ones_ctx* c, uint64_t seed) {
+    if (!c) return ONES_ERR_NULL;
+    CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->J, c->tab, make_round_keys(seed), c->stream));
+    c->launches += 1;
+    c->f_valid = false;
+    return ONES_OK;
+}
+
+int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_device) {
+    if (!c || !genomes) return ONES_ERR_NULL;
+    if (ld < c->J) return ONES_ERR_BAD_PARAM;
+    if (on_device) {
+        CU(c, launch_copy_rows(genomes, ld, c->pop(c->cur), c->ld, c->N, c->J, 1, c->stream));
+        c->launches += 1;
+    } else {
+        if (c->ld != c->J) CU(c, cudaMemsetAsync(c->pop(c->cur), 0, (size_t)c->N * c->ld * 4, c->stream));
+        CU(c, cudaMemcpy2DAsync(c->pop(c->cur), (size_t)c->ld * 4, genomes, (size_t)ld * 4, (size_t)c->J * 4,
+                                (size_t)c->N, cudaMemcpyHostToDevice, c->stream));
+        CU(c, cudaStreamSynchronize(c->stream));
+    }
+    c->f_valid = false;
+    return ONES_OK;
+}
+
+int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device) {
+    if (!c || !genomes) return ONES_ERR_NULL;
+    if (ld < c->J) return ONES_ERR_BAD_PARAM;
+    if (on_device) {
+        CU(c, launch_copy_rows(c->pop(c->cur), c->ld, genomes, ld, c->N, c->J, 0, c->stream));
+        c->launches += 1;
+    } else {
+        CU(c, cudaMemcpy2DAsync(genomes, (size_t)ld * 4, c->pop(c->cur), (size_t)c->ld * 4, (size_t)c->J * 4,
+                                (size_t)c->N, cudaMemcpyDeviceToHost, c->stream));
+        CU(c, cudaStreamSynchronize(c->stream));
+    }
+    return ONES_OK;
+}
+
+int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, double* d_fitness, int32_t* d_gpus) {
+    if (!c || !d_fitness) return ONES_ERR_NULL;
+    if (!d_genomes) {
+        if (!c->f_valid) {
+            int rc = run_fitness(c);
+            if (rc) return rc;
+        }
+        CU(c, cudaMemcpyAsync(d_fitness, c->F(), (size_t)c->N * 8, cudaMemcpyDeviceToDevice, c->stream));
+        if (d_gpus) CU(c, cudaMemcpyAsync(d_gpus, c->G(), (size_t)c->N * 4, cudaMemcpyDeviceToDevice, c->stream));
+        return ONES_OK;
+    }
+    if (n < 0 || ld < c->J) return ONES_ERR_BAD_PARAM;
+    if ((ld & 3) != 0 || !aligned16(d_genomes)) return ONES_ERR_ALIGN;
+    if (n == 0) return ONES_OK;
+    int rc = prof_begin(c, 0);
+    if (rc) return rc;
+    CU(c, launch_fitness(d_genomes, ld, n, c->J, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
+    c->launches += 1;
+    return prof_end(c);
+}
+
+int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
+    if (!c) return ONES_ERR_NULL;
+    if (generations < 0) return ONES_ERR_BAD_PARAM;
+    if (generations == 0) return ONES_OK;
+    int rc;
+    if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
+    const RoundKeys keys = make_round_keys(seed);
+    const int32_t E = c->prm.elitism;
+    for (int32_t it = 0; it < generations; ++it) {
+        if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
+        CU(c, launch_select(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), c->stream));
+        c->launches += c->pairs > 0 ? 1 : 0;
+        int nl = 0;
+        CU(c, launch_top(c->F(), c->N, E, c->elites(), c->ws + c->L.top, c->stream, &nl));
+        c->launches += (uint64_t)nl;
+        if ((rc = prof_end(c)) != ONES_OK) return rc;
+
+        if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
+        CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs, c->parents(),
+                            c->elites(), c->tab, keys, c->gen, c->thr16, c->stream));
+        c->launches += 1;
+        if ((rc = prof_end(c)) != ONES_OK) return rc;
+
+        c->cur ^= 1;
+        c->gen += 1;
+        if ((rc = run_fitness(c)) != ONES_OK) return rc;
+    }
+    return ONES_OK;
+}
+
+int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_job, double* h_rate_per_job,
+              double* fitness, int32_t* total_gpus, int32_t* index) {
+    if (!c) return ONES_ERR_NULL;
+    int rc;
+    if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
+    int nl = 0;
+    CU(c, launch_top(c->F(), c->N, 1, c->best_idx(), c->ws + c->L.top, c->stream, &nl));
+    int32_t* d_genome = reinterpret_cast<int32_t*>(c->ws + c->L.out_genome);
+    int32_t* d_gpus = reinterpret_cast<int32_t*>(c->ws + c->L.out_gpus);
+    double* d_rate = reinterpret_cast<double*>(c->ws + c->L.out_rate);
+    BestOut* d_rec = reinterpret_cast<BestOut*>(c->ws + c->L.out_rec);
+    CU(c, launch_best(c->pop(c->cur), c->ld, c->J, c->best_idx(), c->tab, c->cap, c->prm.penalty, repair,
+                      reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
+    c->launches += (uint64_t)nl + 1;
+    BestOut rec;
+    if (h_genome) CU(c, cudaMemcpyAsync(h_genome, d_genome, (size_t)c->J * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (h_gpus_per_job)
+        CU(c, cudaMemcpyAsync(h_gpus_per_job, d_gpus, (size_t)c->J * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (h_rate_per_job)
+        CU(c, cudaMemcpyAsync(h_rate_per_job, d_rate, (size_t)c->J * 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(&rec, d_rec, sizeof rec, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    if (fitness) *fitness = rec.fitness;
+    if (total_gpus) *total_gpus = rec.total_gpus;
+    if (index) *index = rec.index;
+    return rec.status ? ONES_ERR_INFEASIBLE : ONES_OK;
+}
+
+int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const int32_t* remap, int32_t capacity) {
+    if (!c || !jobs || !remap) return ONES_ERR_NULL;
+    int rc = check_jobs(jobs, n_jobs);
+    if (rc) return rc;
+    if (capacity <= 0) return ONES_ERR_BAD_PARAM;
+    if (n_jobs > c->Jmax) return ONES_ERR_WORKSPACE;
+    for (int32_t j = 0; j < n_jobs; ++j)
+        if (remap[j] < -1 || remap[j] >= c->J) return ONES_ERR_BAD_PARAM;
+    const int64_t old_ld = c->ld;
+    CU(c, cudaMemcpyAsync(c->remap(), remap, (size_t)n_jobs * 4, cudaMemcpyHostToDevice, c->stream));
+    rc = rebuild_tables(c, jobs, n_jobs);
+    if (rc != ONES_OK) {
+        // put the tables of the job set in force back; the population is untouched
+        const std::vector<ones_job> keep = c->h_jobs;
+        int rc2 = rebuild_tables(c, keep.data(), (int32_t)keep.size());
+        return rc2 == ONES_OK ? rc : rc2;
+    }
+    const int64_t new_ld = ld_of(n_jobs);
+    CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(), c->tab.kmin,
+                       c->tab.range, c->stream));
+    c->launches += 1;
+    c->cur ^= 1;
+    c->J = n_jobs;
+    c->ld = new_ld;
+    c->cap = capacity;
+    c->f_valid = false;
+    return ONES_OK;
+}
+
+int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
+    if (!c) return ONES_ERR_NULL;
+    if (h_parents && c->pairs > 0)
+        CU(c, cudaMemcpyAsync(h_parents, c->parents(), (size_t)c->pairs * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (h_elites && c->prm.elitism > 0)
+        CU(c, cudaMemcpyAsync(h_elites, c->elites(), (size_t)c->prm.elitism * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return ONES_OK;
+}
+
+int ones_model_table(ones_ctx* c, double* h_X, int32_t* h_g, int32_t* planes) {
+    if (!c) return ONES_ERR_NULL;
+    if (planes) *planes = c->tab.k1;
+    if (!h_X && !h_g) return ONES_OK;
+    double* dX = reinterpret_cast<double*>(c->ws + c->L.exp_X);
+    int32_t* dG = reinterpret_cast<int32_t*>(c->ws + c->L.exp_G);
+    CU(c, launch_export_tables(c->tab, c->J, dX, dG, c->stream));
+    c->launches += 1;
+    const size_t cells = (size_t)c->tab.k1 * c->J;
+    if (h_X) CU(c, cudaMemcpyAsync(h_X, dX, cells * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (h_g) CU(c, cudaMemcpyAsync(h_g, dG, cells * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return ONES_OK;
+}
+
+size_t ones_select_top_scratch_bytes(int32_t n, int32_t e) {
+    if (n <= 0 || e <= 0 || e > ONES_MAX_ELITES || e > n) return 0;
+    return top_scratch_bytes(n, e);
+}
+
+int ones_select_top(const double* d_fitness, int32_t n, int32_t e, int32_t* d_index, void* d_scratch,
+                    size_t scratch_bytes, void* cuda_stream) {
+    if (!d_fitness || !d_index || !d_scratch) return ONES_ERR_NULL;
+    if (n <= 0 || e <= 0 || e > ONES_MAX_ELITES || e > n) return ONES_ERR_BAD_PARAM;
+    if (!aligned16(d_scratch)) return ONES_ERR_ALIGN;
+    if (scratch_bytes < top_scratch_bytes(n, e)) return ONES_ERR_WORKSPACE;
+    cudaError_t err = launch_top(d_fitness, n, e, d_index, d_scratch, reinterpret_cast<cudaStream_t>(cuda_stream),
+                                 nullptr);
+    return err == cudaSuccess ? ONES_OK : ONES_ERR_CUDA;
+}
+
+int ones_generation(const ones_ctx* c, uint64_t* gen_abs) {
+    if (!c || !gen_abs) return ONES_ERR_NULL;
+    *gen_abs = c->gen;
+    return ONES_OK;
+}
+
+int ones_shape(const ones_ctx* c, int32_t* n_jobs, int32_t* pop, int32_t* capacity, int64_t* ld) {
+    if (!c) return ONES_ERR_NULL;
+    if (n_jobs) *n_jobs = c->J;
+    if (pop) *pop = c->N;
+    if (capacity) *capacity = c->cap;
+    if (ld) *ld = c->ld;
+    return ONES_OK;
+}
+
+int ones_kernel_launches(const ones_ctx* c, uint64_t* launches) {
+    if (!c || !launches) return ONES_ERR_NULL;
+    *launches = c->launches;
+    return ONES_OK;
+}
+
+int ones_set_profiling(ones_ctx* c, int on) {
+    if (!c) return ONES_ERR_NULL;
+    if (on && c->prof.ev.empty()) {
+        const size_t want = 4096;
+        c->prof.ev.reserve(want);
+        for (size_t i = 0; i < want; ++i) {
+            cudaEvent_t ev;
+            CU(c, cudaEventCreate(&ev));
+            c->prof.ev.push_back(ev);
+        }
+        c->prof.stage.assign(want / 2, 0);
+    }
+    if (!on) {
+        int rc = prof_flush(c);
+        if (rc) return rc;
+    }
+    c->prof.on = on != 0;
+    return ONES_OK;
+}
+
+int ones_stage_times(ones_ctx* c, double ms[3], uint64_t count[3]) {
+    if (!c || !ms || !count) return ONES_ERR_NULL;
+    int rc = prof_flush(c);
+    if (rc) return rc;
+    for (int s = 0; s < 3; ++s) {
+        ms[s] = c->prof.ms[s];
+        count[s] = c->prof.count[s];
+        c->prof.ms[s] = 0;
+        c->prof.count[s] = 0;
+    }
+    return ONES_OK;
+}
+
+int ones_last_cuda_error(const ones_ctx* c) { return c ? c->last_cuda : 0; }
+
+const char* ones_strerror(int code) {
+    switch (code) {
+        case ONES_OK: return "ok";
+        case ONES_ERR_NULL: return "a required pointer is NULL";
+        case ONES_ERR_BAD_JOB: return "a job row is out of range";
+        case ONES_ERR_BAD_PARAM: return "an argument or parameter is out of range";
+        case ONES_ERR_ALIGN: return "pointer not 16-byte aligned or ld not a multiple of 4";
+        case ONES_ERR_WORKSPACE: return "workspace too small";
+        case ONES_ERR_CUDA: return "a CUDA call failed";
+        case ONES_ERR_INFEASIBLE: return "repair could not reach the capacity";
+        case ONES_ERR_NOMEM: return "host allocation failed";
+        default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

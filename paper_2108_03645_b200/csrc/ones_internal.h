@@ -1,0 +1,72 @@
+// Internal interface between the C ABI (ones_api.cu) and the kernels (ones_kernels.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ones.h"
+
+namespace ones {
+
+constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
+constexpr int kMaxSmemPerBlock = 232448;  // 227 KiB opt-in dynamic shared memory per CTA
+constexpr int kTopBlocksMax = 128;        // partial top-k blocks
+
+enum Stream : uint32_t { STREAM_INIT = 0, STREAM_SEL_A = 1, STREAM_SEL_B = 2, STREAM_MUT = 3 };
+
+// Philox4x32-10 round keys for one 64-bit seed: key word pair of round r is
+// (k[2r], k[2r+1]).  Passed to kernels by value so they sit in the constant bank.
+struct RoundKeys {
+    uint32_t k[20];
+};
+RoundKeys make_round_keys(uint64_t seed);
+
+// Geometry of the per-(exponent, job) model tables on the device.
+//   X[p * jpad + slot(j)], G[p * jpad + slot(j)], p = min(unsigned(k), k1): plane k1 is the
+//   all-zero "job waits" plane; entries with k > kmax_j or j >= n_jobs are zero too.
+//   slot(j) = (j & ~127) + (j & 3) * 32 + ((j >> 2) & 31): within a block of 128 jobs the
+//   four genes of one int4 load land in four 32-entry runs, one entry per lane.
+struct Tables {
+    double* X;
+    int32_t* G;
+    int32_t* kmin;   // [jpad] lowest exponent of job j (0 for padding columns)
+    int32_t* range;  // [jpad] kmax - kmin + 1 (1 for padding columns)
+    int32_t jpad;    // n_jobs rounded up to a multiple of 128
+    int32_t k1;      // max_j kmax_j + 1
+};
+
+struct BestOut {  // device record written by the best/repair kernel
+    double fitness;
+    int32_t total_gpus;
+    int32_t index;
+    int32_t status;  // 0 ok, 1 could not reach capacity
+    int32_t steps;
+};
+
+cudaError_t launch_build_tables(const ones_job* d_jobs, int32_t n_jobs, uint32_t flags, Tables t,
+                                int32_t* d_bad /*set to 1 when a throughput is not positive and finite*/,
+                                cudaStream_t s);
+cudaError_t launch_fill_min(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t, cudaStream_t s);
+cudaError_t launch_randomize(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+                             RoundKeys keys, cudaStream_t s);
+cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+                           int32_t capacity, double penalty, double* F, int32_t* G, cudaStream_t s);
+cudaError_t launch_select(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
+                          uint64_t gen, int32_t* parents, cudaStream_t s);
+size_t top_scratch_bytes(int32_t n, int32_t e);
+cudaError_t launch_top(const double* F, int32_t n, int32_t e, int32_t* idx_out, void* scratch,
+                       cudaStream_t s, int* launches);
+cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
+                          int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
+                          Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s);
+cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
+                        int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
+                        int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,
+                        cudaStream_t s);
+cudaError_t launch_remap(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                         int32_t n_jobs_new, const int32_t* remap, const int32_t* kmin_new,
+                         const int32_t* range_new, cudaStream_t s);
+cudaError_t launch_copy_rows(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                             int32_t n_jobs, int zero_pad, cudaStream_t s);
+cudaError_t launch_export_tables(Tables t, int32_t n_jobs, double* X_out, int32_t* G_out, cudaStream_t s);
+
+}  // namespace ones

@@ -1,0 +1,757 @@
+// sm_100a kernels of the ONES evolutionary batch-size search.
+//
+// Data layout in HBM
+//   population   int32[N][ld] row-major, one row per candidate schedule, ld = n_jobs rounded up
+//                to 4 so that every row starts on a 16-byte boundary (int4 loads/stores)
+//   F, G         double[N], int32[N]: score and GPU demand per candidate
+//   model tables X (fp64) and G (int32), one plane per exponent, swizzled (see Tables)
+// Nothing here is a dense contraction: the kernels are gathers, adds and a counter-based RNG,
+// bounded by HBM bandwidth (fitness, evolve) or by launch latency (everything else).
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "ones_internal.h"
+
+namespace ones {
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  Round keys are precomputed on the host.
+// ---------------------------------------------------------------------------------------------
+RoundKeys make_round_keys(uint64_t seed) {
+    RoundKeys rk;
+    uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        rk.k[2 * r] = a;
+        rk.k[2 * r + 1] = b;
+        a += 0x9E3779B9u;
+        b += 0xBB67AE85u;
+    }
+    return rk;
+}
+
+__device__ __forceinline__ uint4 philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                        const RoundKeys& rk) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const unsigned long long p0 = (unsigned long long)0xD2511F53u * c0;
+        const unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k[2 * r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k[2 * r + 1];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Fourth counter word: stream id in the low 4 bits, high half of the generation above them.
+__host__ __device__ __forceinline__ uint32_t counter3(uint32_t stream, uint64_t gen) {
+    return stream | ((uint32_t)(gen >> 32) << 4);
+}
+
+// Uniform value in [kmin, kmin + range) from bits 15..1 of a random word.
+__device__ __forceinline__ int32_t draw_gene(uint32_t w, int32_t kmin, int32_t range) {
+    return kmin + (int32_t)__umulhi((w << 16) & 0xFFFE0000u, (uint32_t)range);
+}
+
+__host__ __device__ __forceinline__ int32_t slot_of(int32_t j) {
+    return (j & ~127) + ((j & 3) << 5) + ((j >> 2) & 31);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Model tables: X_j(k), g_j(k) for every job and exponent (throughput model of the job table)
+// ---------------------------------------------------------------------------------------------
+__global__ void k_build_tables(const ones_job* __restrict__ jobs, int32_t n_jobs, uint32_t flags, Tables t,
+                               int32_t* __restrict__ bad) {
+    const int32_t planes = t.k1 + 1;
+    const int64_t total = (int64_t)planes * t.jpad;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t k = (int32_t)(i / t.jpad);
+        const int32_t j = (int32_t)(i % t.jpad);
+        double term = 0.0;
+        int32_t gpus = 0;
+        if (j < n_jobs) {
+            const ones_job job = jobs[j];
+            if (k <= job.kmax && k < t.k1) {
+                const long long b = (long long)job.b0 << k;
+                const long long m = job.max_per_gpu;
+                const long long g = (b + m - 1) / m;
+                const double local = __ddiv_rn((double)b, (double)g);
+                // log2 of a power of two is its exponent, exactly; otherwise the library routine
+                const double lg = ((g & (g - 1)) == 0) ? (double)(63 - __clzll(g)) : log2((double)g);
+                const double sec = __dadd_rn(__dadd_rn(job.a, __dmul_rn(job.c, local)), __dmul_rn(job.d, lg));
+                const double X = __ddiv_rn((double)b, sec);
+                if (!(X > 0.0) || X > 1.7976931348623157e308) atomicOr(bad, 1);  // needs seconds/iteration > 0
+                gpus = (int32_t)g;
+                term = (flags & ONES_FLAG_SRUF) ? -__ddiv_rn(__dmul_rn(job.weight, (double)gpus), X) : X;
+            }
+            if (k == 0) {
+                t.kmin[j] = job.kmin;
+                t.range[j] = job.kmax - job.kmin + 1;
+            }
+        } else if (k == 0) {
+            t.kmin[j] = 0;
+            t.range[j] = 1;
+        }
+        const int64_t at = (int64_t)k * t.jpad + slot_of(j);
+        t.X[at] = term;
+        t.G[at] = gpus;
+    }
+}
+
+cudaError_t launch_build_tables(const ones_job* d_jobs, int32_t n_jobs, uint32_t flags, Tables t,
+                                int32_t* d_bad, cudaStream_t s) {
+    const int64_t total = (int64_t)(t.k1 + 1) * t.jpad;
+    const int grid = (int)((total + 255) / 256);
+    k_build_tables<<<grid < 1024 ? grid : 1024, 256, 0, s>>>(d_jobs, n_jobs, flags, t, d_bad);
+    return cudaGetLastError();
+}
+
+// X[k][j], g[k][j] in plain job order for the host (k < k1)
+__global__ void k_export_tables(Tables t, int32_t n_jobs, double* __restrict__ X_out, int32_t* __restrict__ G_out) {
+    const int64_t total = (int64_t)t.k1 * n_jobs;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t k = (int32_t)(i / n_jobs), j = (int32_t)(i % n_jobs);
+        const int64_t at = (int64_t)k * t.jpad + slot_of(j);
+        X_out[i] = t.X[at];
+        G_out[i] = t.G[at];
+    }
+}
+
+cudaError_t launch_export_tables(Tables t, int32_t n_jobs, double* X_out, int32_t* G_out, cudaStream_t s) {
+    const int64_t total = (int64_t)t.k1 * n_jobs;
+    const int grid = (int)((total + 255) / 256);
+    k_export_tables<<<grid < 1024 ? grid : 1024, 256, 0, s>>>(t, n_jobs, X_out, G_out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Population set-up: all-minimum population, random population, row copies, column remap
+// ---------------------------------------------------------------------------------------------
+__global__ void k_fill_min(int32_t* __restrict__ pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t) {
+    const int64_t total = (int64_t)n * ld;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t j = (int32_t)(i % ld);
+        pop[i] = j < n_jobs ? t.kmin[j] : 0;
+    }
+}
+
+cudaError_t launch_fill_min(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t, cudaStream_t s) {
+    const int64_t total = (int64_t)n * ld;
+    const int64_t grid = (total + 255) / 256;
+    k_fill_min<<<(int)(grid < kSMs * 8 ? grid : kSMs * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t);
+    return cudaGetLastError();
+}
+
+// One thread per int4 of the population: four genes from one Philox call.
+__global__ void k_randomize(int32_t* __restrict__ pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+                            RoundKeys keys) {
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const int64_t total = (int64_t)n * nvec;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t row = (int32_t)(i / nvec), v = (int32_t)(i % nvec);
+        const int4 kmin = *reinterpret_cast<const int4*>(t.kmin + 4 * v);
+        const int4 range = *reinterpret_cast<const int4*>(t.range + 4 * v);
+        int4 out = kmin;  // candidate 0: every job at its smallest batch
+        if (row > 0) {
+            const uint4 w = philox((uint32_t)v, (uint32_t)row, 0u, counter3(STREAM_INIT, 0), keys);
+            out.x = draw_gene(w.x, kmin.x, range.x);
+            out.y = draw_gene(w.y, kmin.y, range.y);
+            out.z = draw_gene(w.z, kmin.z, range.z);
+            out.w = draw_gene(w.w, kmin.w, range.w);
+        }
+        *reinterpret_cast<int4*>(pop + (int64_t)row * ld + 4 * v) = out;
+    }
+}
+
+cudaError_t launch_randomize(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+                             RoundKeys keys, cudaStream_t s) {
+    const int64_t total = (int64_t)n * (ld >> 2);
+    const int64_t grid = (total + 255) / 256;
+    k_randomize<<<(int)(grid < kSMs * 8 ? grid : kSMs * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t, keys);
+    return cudaGetLastError();
+}
+
+__global__ void k_copy_rows(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restrict__ dst,
+                            int64_t ld_dst, int32_t n, int32_t n_jobs, int zero_pad) {
+    const int64_t width = zero_pad ? ld_dst : n_jobs;
+    const int64_t total = (int64_t)n * width;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / width;
+        const int32_t j = (int32_t)(i % width);
+        dst[row * ld_dst + j] = j < n_jobs ? src[row * ld_src + j] : 0;
+    }
+}
+
+cudaError_t launch_copy_rows(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                             int32_t n_jobs, int zero_pad, cudaStream_t s) {
+    const int64_t total = (int64_t)n * (zero_pad ? ld_dst : n_jobs);
+    const int64_t grid = (total + 255) / 256;
+    if (grid == 0) return cudaSuccess;
+    k_copy_rows<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs,
+                                                                          zero_pad);
+    return cudaGetLastError();
+}
+
+__global__ void k_remap(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restrict__ dst,
+                        int64_t ld_dst, int32_t n, int32_t n_jobs_new, const int32_t* __restrict__ remap,
+                        const int32_t* __restrict__ kmin_new, const int32_t* __restrict__ range_new) {
+    const int64_t total = (int64_t)n * ld_dst;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / ld_dst;
+        const int32_t j = (int32_t)(i % ld_dst);
+        int32_t k = 0;
+        if (j < n_jobs_new) {
+            const int32_t lo = kmin_new[j], hi = lo + range_new[j] - 1;
+            const int32_t from = remap[j];
+            k = lo;
+            if (from >= 0) k = min(max(src[row * ld_src + from], lo), hi);
+        }
+        dst[i] = k;
+    }
+}
+
+cudaError_t launch_remap(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                         int32_t n_jobs_new, const int32_t* remap, const int32_t* kmin_new,
+                         const int32_t* range_new, cudaStream_t s) {
+    const int64_t total = (int64_t)n * ld_dst;
+    const int64_t grid = (total + 255) / 256;
+    k_remap<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs_new,
+                                                                      remap, kmin_new, range_new);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fitness: one candidate per warp.  Lane l reads the int4 at genes 4l..4l+3 of every block of 128
+// genes, looks each gene's (X, g) up in the tables and accumulates privately in increasing job
+// order; a five-step butterfly over the 32 lanes finishes the fixed-order sum.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int4 ld_genes(const int4* p) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <bool SMEM, int UNROLL>
+__global__ void __launch_bounds__(1024, 1)
+k_fitness(const int32_t* __restrict__ genomes, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+          int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const double* __restrict__ lutX = t.X;
+    const int32_t* __restrict__ lutG = t.G;
+    if (SMEM) {
+        // stage both tables in shared memory: X planes first, then g planes
+        double* sX = reinterpret_cast<double*>(smem_raw);
+        int32_t* sG = reinterpret_cast<int32_t*>(smem_raw + (size_t)planes * t.jpad * sizeof(double));
+        const int32_t nX = planes * t.jpad / 2;  // int4 = two doubles
+        const int32_t nG = planes * t.jpad / 4;  // int4 = four ints
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) reinterpret_cast<int4*>(sG)[i] = gG[i];
+        __syncthreads();
+        lutX = sX;
+        lutG = sG;
+    }
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (n_jobs + 3) >> 2;
+    const uint32_t kcap = (uint32_t)t.k1;
+    const int32_t jpad = t.jpad;
+
+    for (int64_t cand = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); cand < n; cand += total_warps) {
+        const int4* row = reinterpret_cast<const int4*>(genomes + cand * ld);
+        double sum = 0.0;
+        int32_t gpus = 0;
+        for (int32_t v0 = 0; v0 < nvec; v0 += 32 * UNROLL) {
+            int4 q[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int32_t v = v0 + u * 32 + lane;
+                if (v < nvec) q[u] = ld_genes(row + v);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int32_t v = v0 + u * 32 + lane;
+                if (v < nvec) {
+                    const int32_t base = ((v0 >> 5) + u) * 128 + lane;  // slot of gene 4l of this block
+                    const int32_t i0 = (int32_t)min((uint32_t)q[u].x, kcap) * jpad + base;
+                    const int32_t i1 = (int32_t)min((uint32_t)q[u].y, kcap) * jpad + base + 32;
+                    const int32_t i2 = (int32_t)min((uint32_t)q[u].z, kcap) * jpad + base + 64;
+                    const int32_t i3 = (int32_t)min((uint32_t)q[u].w, kcap) * jpad + base + 96;
+                    sum = __dadd_rn(sum, lutX[i0]); gpus += lutG[i0];
+                    sum = __dadd_rn(sum, lutX[i1]); gpus += lutG[i1];
+                    sum = __dadd_rn(sum, lutX[i2]); gpus += lutG[i2];
+                    sum = __dadd_rn(sum, lutX[i3]); gpus += lutG[i3];
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            gpus += __shfl_xor_sync(0xFFFFFFFFu, gpus, off);
+        }
+        if (lane == 0) {
+            const int32_t over = gpus > capacity ? gpus - capacity : 0;
+            F[cand] = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            if (G) G[cand] = gpus;
+        }
+    }
+}
+
+cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
+                           int32_t capacity, double penalty, double* F, int32_t* G, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const size_t lut_bytes = (size_t)(t.k1 + 1) * t.jpad * 12;
+    const bool big = n >= kSMs * 32;
+    const int threads = big ? 1024 : 256;
+    const int wpb = threads / 32;
+    int64_t blocks = ((int64_t)n + wpb - 1) / wpb;
+    if (lut_bytes <= (size_t)kMaxSmemPerBlock) {
+        int per_sm = (int)(kMaxSmemPerBlock / (lut_bytes + 1024));
+        if (per_sm < 1) per_sm = 1;
+        const int by_threads = 2048 / threads;
+        if (per_sm > by_threads) per_sm = by_threads;
+        if (blocks > (int64_t)kSMs * per_sm) blocks = (int64_t)kSMs * per_sm;
+        cudaError_t e = cudaFuncSetAttribute(k_fitness<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kMaxSmemPerBlock);
+        if (e != cudaSuccess) return e;
+        k_fitness<true, 4><<<(int)blocks, threads, lut_bytes, s>>>(genomes, ld, n, n_jobs, t, capacity, penalty, F, G);
+    } else {
+        // tables too large for shared memory: read them through L1/L2
+        if (blocks > (int64_t)kSMs * (2048 / threads)) blocks = (int64_t)kSMs * (2048 / threads);
+        k_fitness<false, 4><<<(int)blocks, threads, 0, s>>>(genomes, ld, n, n_jobs, t, capacity, penalty, F, G);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tournament selection: one thread per (pair, parent)
+// ---------------------------------------------------------------------------------------------
+__global__ void k_select(const double* __restrict__ F, int32_t n, int32_t tournament, int32_t pairs,
+                         RoundKeys keys, uint32_t gen_lo, uint32_t c3a, uint32_t c3b,
+                         int32_t* __restrict__ parents) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 2 * pairs) return;
+    const uint32_t q = (uint32_t)(i >> 1);
+    const uint32_t c3 = (i & 1) ? c3b : c3a;
+    int32_t win = -1;
+    double fwin = 0.0;
+    for (int32_t t0 = 0; t0 < tournament; t0 += 4) {
+        const uint4 w4 = philox((uint32_t)(t0 >> 2), q, gen_lo, c3, keys);
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (t0 + u < tournament) {
+                const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
+                const double f = F[idx];
+                if (win < 0 || f > fwin || (f == fwin && idx < win)) {
+                    win = idx;
+                    fwin = f;
+                }
+            }
+        }
+    }
+    parents[i] = win;
+}
+
+cudaError_t launch_select(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
+                          uint64_t gen, int32_t* parents, cudaStream_t s) {
+    if (pairs <= 0) return cudaSuccess;
+    const int grid = (2 * pairs + 127) / 128;
+    k_select<<<grid, 128, 0, s>>>(F, n, tournament, pairs, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
+                                  counter3(STREAM_SEL_B, gen), parents);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Top-e selection (score descending, index ascending): per-block partial lists, then one block
+// merges them.  Scores are mapped to order-preserving 64-bit keys; NaN ranks lowest.
+// ---------------------------------------------------------------------------------------------
+struct Rec {
+    unsigned long long key;
+    int32_t idx;
+    int32_t pad;
+};
+
+__device__ __forceinline__ unsigned long long score_key(double f) {
+    if (f != f) return 0ull;
+    const unsigned long long b = (unsigned long long)__double_as_longlong(f + 0.0);  // -0 -> +0
+    return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+
+// true when a ranks before b
+__device__ __forceinline__ bool before(unsigned long long ka, int32_t ia, unsigned long long kb, int32_t ib) {
+    return ka > kb || (ka == kb && ia < ib);
+}
+
+// Block-wide best record that ranks strictly after `prev` (or any record when !have_prev).
+// RAW: items are scores F[i] with index lo + i; else items are Rec.
+template <bool RAW>
+__device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, bool have_prev, Rec prev,
+                               Rec* s_warp) {
+    Rec best;
+    best.key = 0ull;
+    best.idx = -1;
+    best.pad = 0;
+    for (int32_t i = threadIdx.x; i < count; i += blockDim.x) {
+        unsigned long long k;
+        int32_t id;
+        if (RAW) {
+            k = score_key(reinterpret_cast<const double*>(items)[i]);
+            id = lo + i;
+        } else {
+            const Rec r = reinterpret_cast<const Rec*>(items)[i];
+            k = r.key;
+            id = r.idx;
+            if (id < 0) continue;
+        }
+        if (have_prev && !before(prev.key, prev.idx, k, id)) continue;
+        if (best.idx < 0 || before(k, id, best.key, best.idx)) {
+            best.key = k;
+            best.idx = id;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xFFFFFFFFu, best.key, off);
+        const int32_t oi = __shfl_xor_sync(0xFFFFFFFFu, best.idx, off);
+        if (oi >= 0 && (best.idx < 0 || before(ok, oi, best.key, best.idx))) {
+            best.key = ok;
+            best.idx = oi;
+        }
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    __syncthreads();  // s_warp may still be read from the previous round
+    if (lane == 0) s_warp[warp] = best;
+    __syncthreads();
+    Rec r = s_warp[0];
+    for (int w = 1; w < nwarp; ++w) {
+        const Rec o = s_warp[w];
+        if (o.idx >= 0 && (r.idx < 0 || before(o.key, o.idx, r.key, r.idx))) r = o;
+    }
+    return r;
+}
+
+__global__ void __launch_bounds__(256) k_top_partial(const double* __restrict__ F, int32_t n, int32_t e,
+                                                     int32_t per_block, Rec* __restrict__ partial) {
+    __shared__ Rec s_warp[8];
+    const int32_t lo = blockIdx.x * per_block;
+    const int32_t count = min(per_block, n - lo);
+    Rec prev;
+    prev.key = 0;
+    prev.idx = -1;
+    prev.pad = 0;
+    for (int32_t r = 0; r < e; ++r) {
+        Rec best = block_next_best<true>(F + lo, count > 0 ? count : 0, lo, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
+        prev = best;
+        if (best.idx < 0) {  // fewer than e items in this block: mark the rest empty
+            for (int32_t r2 = r + 1 + threadIdx.x; r2 < e; r2 += blockDim.x)
+                partial[(int64_t)blockIdx.x * e + r2] = best;
+            break;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) k_top_final(const Rec* __restrict__ partial, int32_t count, int32_t e,
+                                                   int32_t* __restrict__ idx_out) {
+    __shared__ Rec s_warp[8];
+    Rec prev;
+    prev.key = 0;
+    prev.idx = -1;
+    prev.pad = 0;
+    for (int32_t r = 0; r < e; ++r) {
+        Rec best = block_next_best<false>(partial, count, 0, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) idx_out[r] = best.idx;
+        prev = best;
+    }
+}
+
+static int top_blocks(int32_t n) {
+    int b = (n + 4095) / 4096;
+    if (b < 1) b = 1;
+    if (b > kTopBlocksMax) b = kTopBlocksMax;
+    return b;
+}
+
+size_t top_scratch_bytes(int32_t n, int32_t e) {
+    (void)n;
+    return (size_t)kTopBlocksMax * (size_t)e * sizeof(Rec);
+}
+
+cudaError_t launch_top(const double* F, int32_t n, int32_t e, int32_t* idx_out, void* scratch, cudaStream_t s,
+                       int* launches) {
+    if (e <= 0) return cudaSuccess;
+    const int blocks = top_blocks(n);
+    const int32_t per_block = (n + blocks - 1) / blocks;
+    Rec* partial = reinterpret_cast<Rec*>(scratch);
+    k_top_partial<<<blocks, 256, 0, s>>>(F, n, e, per_block, partial);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    k_top_final<<<1, 256, 0, s>>>(partial, blocks * e, e, idx_out);
+    if (launches) *launches += 2;
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Uniform crossover + uniform mutation, fused: one warp per pair of children.  Lane l handles the
+// int4 at genes 4l..4l+3 of every block of 128 genes: two parent loads, two Philox calls (one per
+// child row; counter = (int4 index, row, generation, stream)), two child stores.  Warps past the
+// last pair copy the elites to rows 0..E-1.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int32_t mutate(uint32_t w, int32_t gene, int32_t kmin, int32_t range, uint32_t thr16) {
+    return ((w >> 16) < thr16) ? draw_gene(w, kmin, range) : gene;
+}
+
+template <int UNROLL>
+__global__ void __launch_bounds__(256)
+k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
+         int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents, const int32_t* __restrict__ elites,
+         Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr16) {
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const int4* __restrict__ kminv = reinterpret_cast<const int4*>(t.kmin);
+    const int4* __restrict__ rangev = reinterpret_cast<const int4*>(t.range);
+
+    for (int64_t w = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); w < (int64_t)pairs + elitism;
+         w += total_warps) {
+        if (w >= pairs) {  // survivor: copy unchanged
+            const int32_t r = (int32_t)(w - pairs);
+            const int4* from = reinterpret_cast<const int4*>(src + (int64_t)elites[r] * ld);
+            int4* to = reinterpret_cast<int4*>(dst + (int64_t)r * ld);
+            for (int32_t v = lane; v < nvec; v += 32) to[v] = from[v];
+            continue;
+        }
+        const int32_t q = (int32_t)w;
+        const int32_t pa = parents[2 * q], pb = parents[2 * q + 1];
+        const int32_t slot0 = elitism + 2 * q, slot1 = slot0 + 1;
+        const bool has1 = slot1 < n;
+        const int4* A = reinterpret_cast<const int4*>(src + (int64_t)pa * ld);
+        const int4* B = reinterpret_cast<const int4*>(src + (int64_t)pb * ld);
+        int4* C0 = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
+        int4* C1 = reinterpret_cast<int4*>(dst + (int64_t)slot1 * ld);
+        for (int32_t v0 = 0; v0 < nvec; v0 += 32 * UNROLL) {
+            int4 a[UNROLL], b[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int32_t v = v0 + u * 32 + lane;
+                if (v < nvec) {
+                    a[u] = A[v];
+                    b[u] = B[v];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int32_t v = v0 + u * 32 + lane;
+                if (v < nvec) {
+                    const int4 kmin = kminv[v];
+                    const int4 range = rangev[v];
+                    const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+                    const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                    int4 c0, c1;
+                    // bit 0 of the even child's word: which child inherits the first parent's gene
+                    c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
+                    c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
+                    c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
+                    c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
+                    c0.x = mutate(w0.x, c0.x, kmin.x, range.x, thr16);
+                    c0.y = mutate(w0.y, c0.y, kmin.y, range.y, thr16);
+                    c0.z = mutate(w0.z, c0.z, kmin.z, range.z, thr16);
+                    c0.w = mutate(w0.w, c0.w, kmin.w, range.w, thr16);
+                    C0[v] = c0;
+                    if (has1) {
+                        c1.x = mutate(w1.x, c1.x, kmin.x, range.x, thr16);
+                        c1.y = mutate(w1.y, c1.y, kmin.y, range.y, thr16);
+                        c1.z = mutate(w1.z, c1.z, kmin.z, range.z, thr16);
+                        c1.w = mutate(w1.w, c1.w, kmin.w, range.w, thr16);
+                        C1[v] = c1;
+                    }
+                }
+            }
+        }
+    }
+}
+
+cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
+                          int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
+                          Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s) {
+    const int64_t warps = (int64_t)pairs + elitism;
+    if (warps <= 0) return cudaSuccess;
+    int64_t blocks = (warps + 7) / 8;
+    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    k_evolve<2><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+                                            (uint32_t)gen, counter3(STREAM_MUT, gen), thr16);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Best candidate and its repair to the cluster's capacity: one block.
+// work[0..jpad) exponent, work[jpad..2jpad) GPUs now, work[2jpad..3jpad) GPUs one exponent lower
+// (-1 when the job cannot shrink).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int2 block_arg_best(int2 mine /*(value, j); value < 0: none*/, int2* s_warp, bool want_max_value) {
+    // max value, ties to the lower j (want_max_value) — or lowest j among value >= 0 otherwise
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        int2 o;
+        o.x = __shfl_xor_sync(0xFFFFFFFFu, mine.x, off);
+        o.y = __shfl_xor_sync(0xFFFFFFFFu, mine.y, off);
+        bool take;
+        if (want_max_value) take = o.x > mine.x || (o.x == mine.x && o.x >= 0 && o.y < mine.y);
+        else take = o.x >= 0 && (mine.x < 0 || o.y < mine.y);
+        if (take) mine = o;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    __syncthreads();
+    if (lane == 0) s_warp[warp] = mine;
+    __syncthreads();
+    int2 r = s_warp[0];
+    for (int w = 1; w < nwarp; ++w) {
+        const int2 o = s_warp[w];
+        bool take;
+        if (want_max_value) take = o.x > r.x || (o.x == r.x && o.x >= 0 && o.y < r.y);
+        else take = o.x >= 0 && (r.x < 0 || o.y < r.y);
+        if (take) r = o;
+    }
+    return r;
+}
+
+__global__ void __launch_bounds__(256)
+k_best(const int32_t* __restrict__ pop, int64_t ld, int32_t n_jobs, const int32_t* __restrict__ best_index, Tables t,
+       int32_t capacity, double penalty, int repair, int32_t* __restrict__ work, int32_t* __restrict__ genome_out,
+       int32_t* __restrict__ gpus_out, double* __restrict__ rate_out, BestOut* __restrict__ out) {
+    __shared__ int2 s_warp[8];
+    __shared__ long long s_total;
+    __shared__ int s_status;
+    const int32_t best = best_index[0];
+    const int32_t* row = pop + (int64_t)best * ld;
+    int32_t* wk = work;
+    int32_t* wg = work + t.jpad;
+    int32_t* wl = work + 2 * t.jpad;
+    const uint32_t kcap = (uint32_t)t.k1;
+
+    if (threadIdx.x == 0) { s_total = 0; s_status = 0; }
+    __syncthreads();
+    long long part = 0;
+    for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) {
+        const int32_t k = row[j];
+        const int32_t p = (int32_t)min((uint32_t)k, kcap);
+        const int32_t g = t.G[(int64_t)p * t.jpad + slot_of(j)];
+        int32_t less = -1;
+        if (g > 0 && k > t.kmin[j]) less = t.G[(int64_t)(p - 1) * t.jpad + slot_of(j)];
+        wk[j] = k;  // genes that already mean "waiting" are returned as stored
+        wg[j] = g;
+        wl[j] = (less >= 0 && less < g) ? less : -1;
+        part += g;
+    }
+    atomicAdd(reinterpret_cast<unsigned long long*>(&s_total), (unsigned long long)part);
+    __syncthreads();
+    long long total = s_total;
+    int32_t steps = 0;
+
+    if (repair) {
+        while (total > capacity) {
+            // the job holding the most GPUs among those that can give some back
+            int2 mine = make_int2(-1, 0x7FFFFFFF);
+            for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x)
+                if (wl[j] >= 0 && wg[j] > mine.x) mine = make_int2(wg[j], j);
+            int2 pick = block_arg_best(mine, s_warp, true);
+            if (pick.x >= 0) {
+                const int32_t j = pick.y;
+                if (threadIdx.x == 0) {
+                    const int32_t k = wk[j] - 1;
+                    const int32_t g = wl[j];
+                    total -= wg[j] - g;
+                    int32_t less = -1;
+                    if (k > t.kmin[j]) less = t.G[(int64_t)(k - 1) * t.jpad + slot_of(j)];
+                    wk[j] = k;
+                    wg[j] = g;
+                    wl[j] = (less >= 0 && less < g) ? less : -1;
+                    s_total = total;
+                }
+            } else {
+                // nothing can shrink: the lowest-indexed running job waits
+                int2 run = make_int2(-1, 0x7FFFFFFF);
+                for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x)
+                    if (wg[j] > 0 && j < run.y) run = make_int2(1, j);
+                int2 park = block_arg_best(run, s_warp, false);
+                if (park.x < 0) {
+                    if (threadIdx.x == 0) s_status = 1;
+                    __syncthreads();
+                    break;
+                }
+                if (threadIdx.x == 0) {
+                    const int32_t j = park.y;
+                    total -= wg[j];
+                    wk[j] = -1;
+                    wg[j] = 0;
+                    wl[j] = -1;
+                    s_total = total;
+                }
+            }
+            __syncthreads();
+            total = s_total;
+            ++steps;
+        }
+    }
+    __syncthreads();
+
+    // outputs and the score of the (repaired) row, summed in the fixed order by warp 0
+    for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) {
+        const int32_t k = wk[j];
+        const int32_t p = (int32_t)min((uint32_t)k, kcap);
+        if (genome_out) genome_out[j] = k;
+        if (gpus_out) gpus_out[j] = wg[j];
+        if (rate_out) rate_out[j] = t.X[(int64_t)p * t.jpad + slot_of(j)];
+    }
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        double sum = 0.0;
+        const int32_t nvec = (n_jobs + 3) >> 2;
+        for (int32_t v = lane; v < nvec; v += 32) {
+            for (int s = 0; s < 4; ++s) {
+                const int32_t j = 4 * v + s;
+                if (j < n_jobs) {
+                    const int32_t p = (int32_t)min((uint32_t)wk[j], kcap);
+                    sum = __dadd_rn(sum, t.X[(int64_t)p * t.jpad + slot_of(j)]);
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+        if (lane == 0) {
+            const int32_t g32 = (int32_t)total;
+            const int32_t over = g32 > capacity ? g32 - capacity : 0;
+            out->fitness = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            out->total_gpus = g32;
+            out->index = best;
+            out->status = s_status;
+            out->steps = steps;
+        }
+    }
+}
+
+cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
+                        int32_t capacity, double penalty, int repair, int32_t* work, int32_t* genome_out,
+                        int32_t* gpus_out, double* rate_out, BestOut* out, cudaStream_t s) {
+    k_best<<<1, 256, 0, s>>>(pop, ld, n_jobs, best_index, t, capacity, penalty, repair, work, genome_out, gpus_out,
+                             rate_out, out);
+    return cudaGetLastError();
+}
+
+}  // namespace ones

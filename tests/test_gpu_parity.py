@@ -1,0 +1,339 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2108_03645_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-12  # fp64 scores, fixed summation order (the build's stated bound; 0 ulp expected)
+
+
+@pytest.fixture(scope="module")
+def ones():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2108_03645_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _pair(ones, w, **kw):
+    p = w.params
+    args = dict(elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut, penalty=p.penalty, flags=p.flags)
+    args.update(kw)
+    sp = inputs.SearchParams(**args)
+    return ones.Search(w.jobs, w.capacity, w.pop, sp), oracle.Search(w.jobs, w.capacity, w.pop, **args)
+
+
+def _rel_err(a, b):
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    scale = np.maximum(np.abs(b), 1e-300)
+    return float(np.max(np.abs(a - b) / scale)) if a.size else 0.0
+
+
+def _same_state(g, o, exact_scores=True):
+    assert (g.get_population() == o.get_population()).all()
+    Fg, Gg = g.evaluate()
+    Fo, Go = o.evaluate()
+    assert (Gg.cpu().numpy() == Go).all()
+    assert _rel_err(Fg.cpu().numpy(), Fo) <= REL_TOL
+    if exact_scores:
+        assert (Fg.cpu().numpy() == Fo).all()
+
+
+# ---- a0: model tables ----------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "paper", "mid", "large"])
+def test_model_table_bit_exact(ones, name):
+    w = inputs.WORKLOADS[name]()
+    s = ones.Search(w.jobs, w.capacity, 8, inputs.SearchParams())
+    X, g = s.model_table()
+    assert X.shape[0] == int(w.jobs["kmax"].max()) + 1
+    for j in range(0, w.n_jobs, max(1, w.n_jobs // 64)):
+        for k in range(X.shape[0]):
+            Xo, go = oracle.model(w.jobs, j, k)
+            assert g[k, j] == go and X[k, j] == Xo, (j, k)
+
+
+def test_model_table_non_power_of_two_and_sruf(ones):
+    w = inputs.custom(50, 64, 8, 1, seed=3, pow2=False)
+    w.jobs["weight"] = np.linspace(1e3, 9e4, 50)
+    for flags in (0, ones.FLAG_SRUF):
+        s = ones.Search(w.jobs, w.capacity, 8, inputs.SearchParams(flags=flags))
+        X, g = s.model_table()
+        want = np.array([[oracle.term(w.jobs, j, k, flags) for j in range(50)] for k in range(X.shape[0])])
+        assert (g == want[:, :, 1]).all()
+        assert _rel_err(X, want[:, :, 0]) <= 1e-15 * 4  # log2 of a non-power of two may differ in the last bit
+
+
+# ---- a1: fitness ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("J,n,ld_extra", [(1, 5, 3), (3, 33, 1), (5, 64, 7), (16, 32, 0), (100, 1000, 4),
+                                          (127, 257, 1), (128, 300, 0), (129, 300, 3), (512, 2051, 0),
+                                          (2048, 5000, 0), (2050, 700, 2)])
+def test_fitness_parity(ones, J, n, ld_extra):
+    w = inputs.custom(J, max(8, 2 * J), 8, 1, seed=J, log_uniform=True)
+    ld = ((J + 3) // 4) * 4 + 4 * ((ld_extra + 3) // 4)
+    genomes = inputs.random_genomes(w.jobs, n, ld=ld, seed=n, waiting_fraction=0.05)
+    genomes[0, :J] = w.jobs["kmax"] + 1  # above every limit: all jobs wait
+    if n > 1:
+        genomes[1, :J] = np.iinfo(np.int32).min
+    g, o = _pair(ones, w)
+    Fg, Gg = g.evaluate(torch.from_numpy(genomes).cuda())
+    Fo, Go = o.evaluate(genomes)
+    assert (Gg.cpu().numpy() == Go).all()
+    assert _rel_err(Fg.cpu().numpy(), Fo) <= REL_TOL
+    assert (Fg.cpu().numpy() == Fo).all()
+    assert Fo[0] == 0.0 and Go[0] == 0
+
+
+def test_fitness_zero_rows_and_sruf(ones):
+    w = inputs.paper_scale(1)
+    w.jobs["weight"] = np.random.default_rng(0).uniform(1e3, 1e6, w.n_jobs)
+    g, o = _pair(ones, w, flags=ones.FLAG_SRUF)
+    genomes = inputs.random_genomes(w.jobs, 77, seed=1)
+    Fg, Gg = g.evaluate(torch.from_numpy(genomes).cuda())
+    Fo, Go = o.evaluate(genomes)
+    assert (Gg.cpu().numpy() == Go).all() and (Fg.cpu().numpy() == Fo).all()
+    empty = torch.zeros((0, 100), dtype=torch.int32, device="cuda")
+    Fe, Ge = g.evaluate(empty)
+    assert Fe.numel() == 0
+
+
+# ---- a2: top-e -----------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,e", [(1, 1), (5, 5), (32, 2), (1000, 7), (4097, 33), (65536, 2), (200000, 256)])
+def test_select_top_parity(ones, n, e):
+    rng = np.random.default_rng(n)
+    F = rng.integers(0, max(2, n // 3), size=n).astype(np.float64) - 5.0  # many ties, both signs
+    F[rng.integers(0, n)] = -0.0
+    got = ones.select_top(torch.from_numpy(F).cuda(), e).cpu().numpy()
+    want = np.array(sorted(range(n), key=lambda i: (-F[i], i))[:e])
+    assert (got == want).all()
+    if n <= 5000:
+        assert (got == oracle.top(F, e)).all()
+
+
+# ---- a3/a4/a5: one generation and many -------------------------------------------------------------
+def test_randomize_parity(ones):
+    for w in (inputs.tiny(), inputs.paper_scale(), inputs.custom(131, 64, 77, 1, seed=2, pinned=9)):
+        g, o = _pair(ones, w)
+        _same_state(g, o)  # all-minimum start
+        g.randomize(12345678901234567)
+        o.randomize(12345678901234567)
+        _same_state(g, o)
+
+
+@pytest.mark.parametrize("name,gens", [("tiny", 10), ("paper", 100)])
+def test_evolve_parity_named_workloads(ones, name, gens):
+    w = inputs.WORKLOADS[name]()
+    g, o = _pair(ones, w)
+    g.randomize(w.seed)
+    o.randomize(w.seed)
+    done = 0
+    for step in (1, 1, 8, gens - 10):
+        g.evolve(step, w.seed)
+        o.evolve(step, w.seed)
+        done += step
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+        assert g.generation == o.generation == done
+    bg, bo = g.best(True), o.best(True)
+    for key in ("genome", "gpus_per_job", "rate_per_job"):
+        assert (bg[key] == bo[key]).all(), key
+    assert bg["fitness"] == bo["fitness"] and bg["total_gpus"] == bo["total_gpus"] and bg["index"] == bo["index"]
+    assert bg["total_gpus"] <= w.capacity
+
+
+def test_evolve_parity_mid_sampled_generations(ones):
+    w = inputs.mid()
+    g, o = _pair(ones, w)
+    g.randomize(3)
+    o.randomize(3)
+    for step in (1, 2):
+        g.evolve(step, 3)
+        o.evolve(step, 3)
+        _same_state(g, o)
+
+
+@pytest.mark.parametrize("kw", [dict(elitism=0), dict(elitism=1), dict(elitism=5, tournament=1),
+                                dict(tournament=9), dict(p_mut=0.0), dict(p_mut=1.0), dict(p_mut=0.02, tournament=8),
+                                dict(penalty=0.0), dict(penalty=37.5)])
+def test_evolve_parity_parameter_corners(ones, kw):
+    w = inputs.custom(37, 48, 101, 6, seed=7, kmax=6, pinned=4)
+    g, o = _pair(ones, w, **kw)
+    g.randomize(5)
+    o.randomize(5)
+    for _ in range(3):
+        g.evolve(2, 99)
+        o.evolve(2, 99)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+
+
+@pytest.mark.parametrize("J,N", [(1, 2), (2, 3), (5, 4), (127, 33), (129, 64), (260, 1025)])
+def test_evolve_parity_ragged_shapes(ones, J, N):
+    w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, params=inputs.SearchParams(1, 3, 0.1, 1e3))
+    g, o = _pair(ones, w)
+    g.randomize(1)
+    o.randomize(1)
+    g.evolve(4, 2 ** 40 + 17)
+    o.evolve(4, 2 ** 40 + 17)
+    _same_state(g, o)
+
+
+def test_evolve_non_power_of_two_gpus_stays_within_tolerance(ones):
+    # log2 of a non-power-of-two GPU count may differ from the oracle's in the last bit, so only the
+    # first generation's scores are comparable gene for gene
+    w = inputs.custom(64, 128, 256, 1, seed=11, pow2=False)
+    g, o = _pair(ones, w)
+    g.randomize(0)
+    o.randomize(0)
+    assert (g.get_population() == o.get_population()).all()
+    Fg, Gg = g.evaluate()
+    Fo, Go = o.evaluate()
+    assert (Gg.cpu().numpy() == Go).all() and _rel_err(Fg.cpu().numpy(), Fo) <= REL_TOL
+
+
+def test_split_runs_and_determinism(ones):
+    w = inputs.paper_scale()
+    a, _ = _pair(ones, w)
+    b, _ = _pair(ones, w)
+    c, _ = _pair(ones, w)
+    for s in (a, b, c):
+        s.randomize(0)
+    a.evolve(10, 0)
+    b.evolve(4, 0)
+    b.evolve(6, 0)
+    c.evolve(10, 1)
+    A, B = a.get_population(), b.get_population()
+    assert (A == B).all() and not (A == c.get_population()).all()
+    assert (a.evaluate()[0] == b.evaluate()[0]).all()
+
+
+def test_set_get_population_roundtrip(ones):
+    w = inputs.custom(30, 64, 50, 1, seed=1)
+    g, o = _pair(ones, w)
+    rows = inputs.random_genomes(w.jobs, 50, ld=36, seed=4)
+    g.set_population(rows)
+    o.set_population(rows)
+    _same_state(g, o)
+    assert (g.get_population(ld=40)[:, :30] == rows[:, :30]).all()
+    dev = torch.from_numpy(rows).cuda()
+    g.set_population(dev)
+    back = g.get_population(on_device=True, ld=32).cpu().numpy()
+    assert (back[:, :30] == rows[:, :30]).all()
+    g.evolve(3, 4)
+    o.evolve(3, 4)
+    _same_state(g, o)
+
+
+# ---- a6: best and repair ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "paper", "mid"])
+def test_best_and_repair_parity(ones, name):
+    w = inputs.WORKLOADS[name]()
+    g, o = _pair(ones, w)
+    g.randomize(7)
+    o.randomize(7)
+    g.evolve(2, 7)
+    o.evolve(2, 7)
+    for repair in (False, True):
+        bg, bo = g.best(repair), o.best(repair)
+        for key in ("genome", "gpus_per_job", "rate_per_job"):
+            assert (bg[key] == bo[key]).all(), (key, repair)
+        assert bg["fitness"] == bo["fitness"] and bg["total_gpus"] == bo["total_gpus"]
+        assert bg["index"] == bo["index"]
+        if repair:
+            assert bg["total_gpus"] <= w.capacity
+
+
+def test_repair_tight_capacity(ones):
+    w = inputs.custom(40, 3, 16, 1, seed=2, kmax=5)  # 40 jobs on 3 GPUs: most must wait
+    g, o = _pair(ones, w)
+    g.randomize(1)
+    o.randomize(1)
+    bg, bo = g.best(True), o.best(True)
+    assert (bg["genome"] == bo["genome"]).all() and bg["total_gpus"] == bo["total_gpus"] <= 3
+    assert (bg["genome"] < 0).sum() >= 37
+
+
+# ---- a7: warm start across a changed job set --------------------------------------------------------
+def test_update_jobs_parity(ones):
+    w = inputs.paper_scale()
+    p = w.params
+    g = ones.Search(w.jobs, w.capacity, w.pop, p, n_jobs_max=160)
+    o = oracle.Search(w.jobs, w.capacity, w.pop, elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut,
+                      penalty=p.penalty)
+    g.randomize(0)
+    o.randomize(0)
+    g.evolve(3, 0)
+    o.evolve(3, 0)
+    rng = np.random.default_rng(0)
+    jobs = w.jobs
+    for rnd in range(3):
+        keep = sorted(rng.choice(jobs.shape[0], size=jobs.shape[0] - 13, replace=False).tolist())
+        fresh = inputs.custom(20 + rnd, 64, 8, 1, seed=100 + rnd, kmax=0).jobs
+        jobs2 = np.concatenate([jobs[keep], fresh])
+        jobs2["kmax"][:len(keep)] = np.minimum(7, jobs2["kmax"][:len(keep)] + rng.integers(-1, 2, len(keep))).clip(0)
+        jobs2["kmin"] = np.minimum(jobs2["kmin"], jobs2["kmax"])
+        remap = np.array(keep + [-1] * fresh.shape[0], dtype=np.int32)
+        g.update_jobs(jobs2, remap, 64 + rnd)
+        o.update_jobs(jobs2, remap, 64 + rnd)
+        _same_state(g, o)
+        g.evolve(3, rnd)
+        o.evolve(3, rnd)
+        _same_state(g, o)
+        jobs = jobs2
+    with pytest.raises(ones.OnesError) as err:
+        g.update_jobs(np.concatenate([jobs] * 3), np.full(3 * jobs.shape[0], -1, dtype=np.int32), 64)
+    assert err.value.code == -5
+
+
+# ---- errors ------------------------------------------------------------------------------------
+def test_errors_are_codes_not_faults(ones):
+    w = inputs.tiny()
+    bad = w.jobs.copy()
+    bad["a"][3] = bad["c"][3] = bad["d"][3] = 0.0
+    with pytest.raises(ones.OnesError) as err:
+        ones.Search(bad, 16, 32)
+    assert err.value.code == -2
+    for kw, code in ((dict(elitism=40), -3), (dict(tournament=0), -3), (dict(p_mut=-0.1), -3)):
+        with pytest.raises(ones.OnesError) as err:
+            ones.Search(w.jobs, 16, 32, inputs.SearchParams(**kw))
+        assert err.value.code == code
+    s = ones.Search(w.jobs, 16, 32)
+    odd = torch.zeros((4, 18), dtype=torch.int32, device="cuda")
+    with pytest.raises(ones.OnesError) as err:
+        s.evaluate(odd)  # ld % 4 != 0
+    assert err.value.code == -4
+    with pytest.raises(ones.OnesError) as err:
+        s.evaluate(torch.zeros((4, 12), dtype=torch.int32, device="cuda"))  # ld < jobs
+    assert err.value.code == -3
+    s.evolve(1, 0)  # the handle still works
+
+
+# ---- full size, in the configuration the benchmark times --------------------------------------------
+def test_large_config_parity_full_population(ones):
+    w = inputs.large()
+    g, o = _pair(ones, w)
+    g.randomize(w.seed)
+    o.randomize(w.seed)
+    assert (g.get_population() == o.get_population()).all()
+    g.evolve(1, w.seed)
+    o.evolve(1, w.seed)
+    pg, eg = g.last_parents()
+    po, eo = o.last_parents()
+    assert (pg == po).all() and (eg == eo).all()
+    _same_state(g, o)
+    # invariants that hold at any size
+    P = g.get_population()
+    assert (P >= w.jobs["kmin"][None, :]).all() and (P <= w.jobs["kmax"][None, :]).all()
+    b0 = g.best()["fitness"]
+    g.evolve(5, w.seed)
+    assert g.best()["fitness"] >= b0
+    rep = g.best(True)
+    assert rep["total_gpus"] <= w.capacity
