@@ -1,0 +1,292 @@
+#!/usr/bin/env python
+"""Benchmark of the evolutionary batch-size search: one step = one generation
+(tournament selection + elites, fused crossover/mutation, scoring of the new
+population) over the "large" workload (2048 jobs, population 65536).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is candidate-schedule evaluations per second over
+all ranks with the population resident in HBM; `e2e` is the same metric when
+every step also uploads the job table from host memory and reads the best
+schedule back; `roofline` is the dominant kernel against the measured HBM copy
+bandwidth; `cpu_baseline` is the single-threaded CPU oracle on a bounded sample.
+With N > 1 every rank runs an independent search (replicas, no data-path
+collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2108_03645_b200 import inputs  # noqa: E402
+
+METRIC = "candidate_evals_per_s"
+UNIT = "candidate-schedule evaluations/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.sm, self.reasons, self.sm_max = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nvml = None
+
+    def _loop(self):
+        nv = self._nvml
+        while not self._stop.is_set():
+            try:
+                self.sm.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self._nvml is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample of the workload
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(w, pop_sample: int, gens: int):
+    """Seconds for `gens` generations of a `pop_sample`-candidate population (single thread)."""
+    import oracle
+    p = w.params
+    s = oracle.Search(w.jobs, w.capacity, pop_sample, elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut,
+                      penalty=p.penalty, flags=p.flags)
+    s.randomize(w.seed)
+    s.evaluate()
+    t0 = time.perf_counter()
+    s.evolve(gens, w.seed)
+    dt = time.perf_counter() - t0
+    s.close()
+    return dt
+
+
+def cpu_baseline(w, pop_sample=8192, gens=8):
+    dt = oracle_sample(w, pop_sample, gens)
+    return {"value": pop_sample * gens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{gens} generations of a {pop_sample}-candidate population (of {w.pop}), "
+                      f"{w.n_jobs} jobs, same job table and parameters; {dt:.1f} s"}
+
+
+def run_reference(args, w):
+    """The reference arm: the CPU oracle as it stands, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    pop_sample = 8192
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, pop_sample, 1)
+    steps = max(1, min(args.steps, 20))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample(w, pop_sample, 1)
+    dt = time.perf_counter() - t0
+    value = pop_sample * steps / dt
+    sample = (f"each step = 1 generation of a {pop_sample}-candidate population (of {w.pop}), {w.n_jobs} jobs, "
+              f"single thread; {steps} steps timed (capped at 20)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "jobs": w.n_jobs, "population": w.pop, "capacity": w.capacity},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-events", action="store_true")
+    args = ap.parse_args()
+    w = inputs.WORKLOADS[args.workload]()
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2108_03645_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    warmup = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+
+    base = cpu_baseline(w) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+
+    seed = w.seed + rank  # replicas: every rank searches on its own random stream
+    s = binding.Search(w.jobs, w.capacity, w.pop, w.params)
+    s.randomize(seed)
+    s.evolve(warmup, seed)
+    torch.cuda.synchronize()
+
+    # ---- device-resident timed region: K generations ----
+    if not args.no_kernel_events:
+        s.set_profiling(True)
+        s.stage_times()
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = s.kernel_launches
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    ev0.record()
+    s.evolve(steps, seed)
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = s.kernel_launches - launches0
+    stage_ms, stage_n = ({}, {})
+    if not args.no_kernel_events:
+        stage_ms, stage_n = s.stage_times()
+        s.set_profiling(False)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end: every step uploads the job table and reads the best schedule back ----
+    J, N, E = w.n_jobs, w.pop, w.params.elitism
+    e2e_steps = min(steps, 100)
+    identity = np.arange(J, dtype=np.int32)
+    jobs_pinned = torch.from_numpy(w.jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
+    jobs_host = jobs_pinned.numpy().view(inputs.JOB_DTYPE)
+    for _ in range(3):
+        s.update_jobs(jobs_host, identity, w.capacity)
+        s.evolve(1, seed)
+        s.best(False)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        s.update_jobs(jobs_host, identity, w.capacity)
+        s.evolve(1, seed)
+        out = s.best(False)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = J * 48 + J * 4
+    d2h = J * (4 + 4 + 8) + 24 + 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    line = {
+        "metric": METRIC, "value": world * N * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "jobs": J, "population": N, "capacity": w.capacity,
+                   "elitism": E, "tournament": w.params.tournament, "p_mut": w.params.p_mut,
+                   "genome_table_bytes": N * J * 4, "l2": "inputs larger than L2 (two 512 MiB population buffers)",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "generations_per_s": world * steps / (ms * 1e-3),
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "e2e": {"value": world * N * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs)",
+                "best_fitness": out["fitness"]},
+    }
+    if stage_n.get("evolve"):
+        ev_ms = stage_ms["evolve"] / stage_n["evolve"]
+        fit_ms = stage_ms["fitness"] / stage_n["fitness"]
+        sel_ms = stage_ms["select"] / stage_n["select"]
+        # algorithmic bytes per launch: evolve reads one parent row and writes one child row per child
+        # (8 B per child gene) and copies the elites; fitness reads every gene once and writes F and G
+        evolve_bytes = 8 * J * (N - E) + 8 * J * E + 8 * ((N - E + 1) // 2) + 4 * E
+        fitness_bytes = 4 * J * N + 12 * N
+        ach = evolve_bytes / (ev_ms * 1e-3) / 1e9
+        line["roofline"] = {"kernel": "k_evolve", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                            "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                            "bytes_per_launch": evolve_bytes, "ms_per_launch": ev_ms,
+                            "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS}
+        fach = fitness_bytes / (fit_ms * 1e-3) / 1e9
+        line["kernels"] = {
+            "k_fitness": {"bound": "hbm", "achieved": fach, "peak": peak, "unit": "GB/s", "frac": fach / peak,
+                          "bytes_per_launch": fitness_bytes, "ms_per_launch": fit_ms,
+                          "frac_of_nominal_8TBs": fach / NOMINAL_HBM_GBS},
+            "select_and_elites": {"ms_per_generation": sel_ms},
+        }
+    if base is not None:
+        line["cpu_baseline"] = base
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

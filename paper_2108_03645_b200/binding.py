@@ -198,6 +198,8 @@ class Search:
             G = torch.empty(n, dtype=torch.int32, device=self.device)
         else:
             F, G = out
+        if genomes is not None and n == 0:
+            return F, G  # an empty tensor has no address to pass
         self._check(lib().ones_evaluate(self._h, ptr, ld, n, _t_ptr(F), _t_ptr(G)), "ones_evaluate")
         return F, G
 
