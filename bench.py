@@ -156,8 +156,13 @@ def main():
     ap.add_argument("--workload", default="large", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-events", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling a smaller case)")
     args = ap.parse_args()
     w = inputs.WORKLOADS[args.workload]()
+    if args.pop:
+        import dataclasses
+        w = dataclasses.replace(w, pop=args.pop)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -214,28 +219,31 @@ def main():
 
     # ---- end to end: every step uploads the job table and reads the best schedule back ----
     J, N, E = w.n_jobs, w.pop, w.params.elitism
-    e2e_steps = min(steps, 100)
+    e2e_steps = 0 if args.no_e2e else min(steps, 100)
     identity = np.arange(J, dtype=np.int32)
     jobs_pinned = torch.from_numpy(w.jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
     jobs_host = jobs_pinned.numpy().view(inputs.JOB_DTYPE)
-    for _ in range(3):
-        s.update_jobs(jobs_host, identity, w.capacity)
-        s.evolve(1, seed)
-        s.best(False)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        s.update_jobs(jobs_host, identity, w.capacity)
-        s.evolve(1, seed)
-        out = s.best(False)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    out = {"fitness": None}
+    e2e_s = float("nan")
+    if e2e_steps:
+        for _ in range(3):
+            s.update_jobs(jobs_host, identity, w.capacity)
+            s.evolve(1, seed)
+            s.best(False)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            s.update_jobs(jobs_host, identity, w.capacity)
+            s.evolve(1, seed)
+            out = s.best(False)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
     h2d = J * 48 + J * 4
     d2h = J * (4 + 4 + 8) + 24 + 4
 
@@ -256,7 +264,7 @@ def main():
         "generations_per_s": world * steps / (ms * 1e-3),
         "gpu_launches": launches,
         "clocks": clocks,
-        "e2e": {"value": world * N * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": None if not e2e_steps else {"value": world * N * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs)",
                 "best_fitness": out["fitness"]},
