@@ -166,6 +166,26 @@ size_t ones_select_top_scratch_bytes(int32_t n, int32_t e);
 int ones_select_top(const double* d_fitness, int32_t n, int32_t e, int32_t* d_index,
                     void* d_scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* The same selection for callers that cannot pass scratch memory.  (The paper has no counterpart:
+ * this is a deployment variant of ones_select_top, not a step of the method.)  It is meant for
+ * code that cannot obtain device memory when it runs — e.g. a scheduler plug-in inside a process
+ * whose framework already owns the whole device, where cudaMalloc fails and the framework's
+ * allocator is out of reach, or a round loop that cannot afford the device-wide synchronisation
+ * an allocation implies.  The scratch is a fixed 128 KiB array inside the library's device image
+ * (held by every GPU that loads the library until the process exits); the call allocates and
+ * frees nothing.
+ *   d_fitness, d_index  device, as for ones_select_top.   1 <= e <= min(n, ONES_NOALLOC_MAX_TOP);
+ *   a larger e returns ONES_ERR_WORKSPACE (use ones_select_top with your own scratch).
+ * The first call on each device looks up the array's device address (that device must be
+ * current); make that first call before any stream capture begins.  All calls on a device share
+ * the one array, which keeps whatever the last call left in it: no part of it needs clearing
+ * (each call overwrites every record it later reads), but two calls whose kernels may overlap on
+ * the GPU — different streams, or different threads — race on it; serialise them.
+ * Asynchronous on `cuda_stream`; results equal those of ones_select_top. */
+#define ONES_NOALLOC_MAX_TOP 64
+int ones_select_top_noalloc(const double* d_fitness, int32_t n, int32_t e, int32_t* d_index,
+                            void* cuda_stream);
+
 /* Absolute generation counter, jobs and population of the handle. */
 int ones_generation(const ones_ctx* ctx, uint64_t* gen_abs);
 int ones_shape(const ones_ctx* ctx, int32_t* n_jobs, int32_t* pop, int32_t* capacity, int64_t* ld);

@@ -56,6 +56,7 @@ _SIGNATURES = {
     "ones_select_top_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
     "ones_select_top": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t,
                                   C.c_void_p]),
+    "ones_select_top_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "ones_generation": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ones_shape": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ones_kernel_launches": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -110,6 +111,21 @@ def select_top(fitness: torch.Tensor, e: int) -> torch.Tensor:
     rc = lib().ones_select_top(_t_ptr(fitness), n, e, _t_ptr(out), _t_ptr(scratch), nbytes, _stream_ptr())
     if rc:
         raise OnesError(rc, "ones_select_top")
+    return out
+
+
+NOALLOC_MAX_TOP = 64
+
+
+def select_top_noalloc(fitness: torch.Tensor, e: int, out: torch.Tensor) -> torch.Tensor:
+    """``ones_select_top_noalloc``: as `select_top`, but the library's built-in scratch is used and
+    the caller supplies the output tensor, so nothing is allocated on the way (for callers that
+    cannot get device memory at call time).  Calls that may overlap on the GPU must be serialised."""
+    assert fitness.is_cuda and fitness.dtype == torch.float64 and fitness.is_contiguous()
+    assert out.is_cuda and out.dtype == torch.int32 and out.is_contiguous() and out.numel() >= e
+    rc = lib().ones_select_top_noalloc(_t_ptr(fitness), fitness.numel(), e, _t_ptr(out), _stream_ptr())
+    if rc:
+        raise OnesError(rc, "ones_select_top_noalloc")
     return out
 
 
