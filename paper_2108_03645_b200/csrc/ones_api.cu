@@ -365,11 +365,10 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     const int32_t E = c->prm.elitism;
     for (int32_t it = 0; it < generations; ++it) {
         if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
-        CU(c, launch_select(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), c->stream));
-        c->launches += c->pairs > 0 ? 1 : 0;
-        int nl = 0;
-        CU(c, launch_top(c->F(), c->N, E, c->elites(), c->ws + c->L.top, c->stream, &nl));
-        c->launches += (uint64_t)nl;
+        CU(c, launch_select_stage(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), E,
+                                  c->elites(), c->ws + c->L.top, reinterpret_cast<unsigned int*>(c->status() + 1),
+                                  c->stream));
+        c->launches += 1;
         if ((rc = prof_end(c)) != ONES_OK) return rc;
 
         if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;

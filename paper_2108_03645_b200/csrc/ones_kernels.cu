@@ -413,9 +413,10 @@ __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, boo
             k = score_key(reinterpret_cast<const double*>(items)[i]);
             id = lo + i;
         } else {
-            const Rec r = reinterpret_cast<const Rec*>(items)[i];
-            k = r.key;
-            id = r.idx;
+            // records may have been written by other CTAs of the same launch: read them through L2
+            const int4 raw = __ldcg(reinterpret_cast<const int4*>(items) + i);
+            k = ((unsigned long long)(uint32_t)raw.y << 32) | (uint32_t)raw.x;
+            id = raw.z;
             if (id < 0) continue;
         }
         if (have_prev && !before(prev.key, prev.idx, k, id)) continue;
@@ -481,7 +482,7 @@ __global__ void __launch_bounds__(256) k_top_final(const Rec* __restrict__ parti
 }
 
 static int top_blocks(int32_t n) {
-    int b = (n + 4095) / 4096;
+    int b = (n + 1023) / 1024;
     if (b < 1) b = 1;
     if (b > kTopBlocksMax) b = kTopBlocksMax;
     return b;
@@ -506,6 +507,93 @@ cudaError_t launch_top(const double* F, int32_t n, int32_t e, int32_t* idx_out, 
     return cudaGetLastError();
 }
 
+static int top_blocks(int32_t n);
+
+// Selection stage of one generation in a single launch: CTAs [0, top_blocks) build the partial
+// top-e lists and the last of them to finish merges the lists into `elites`; the remaining CTAs run
+// the tournaments.  `done` counts finished top CTAs; it must be zero at launch and is zero again
+// at exit.  Nothing waits: the merging CTA is simply the one whose increment completes the count.
+__device__ __forceinline__ void tournament_thread(const double* __restrict__ F, int32_t n, int32_t tournament,
+                                                  int32_t i, const RoundKeys& keys, uint32_t gen_lo, uint32_t c3,
+                                                  int32_t* __restrict__ parents) {
+    const uint32_t q = (uint32_t)(i >> 1);
+    int32_t win = -1;
+    double fwin = 0.0;
+    for (int32_t t0 = 0; t0 < tournament; t0 += 4) {
+        const uint4 w4 = philox((uint32_t)(t0 >> 2), q, gen_lo, c3, keys);
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (t0 + u < tournament) {
+                const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
+                const double f = F[idx];
+                if (win < 0 || f > fwin || (f == fwin && idx < win)) {
+                    win = idx;
+                    fwin = f;
+                }
+            }
+        }
+    }
+    parents[i] = win;
+}
+
+__global__ void __launch_bounds__(256)
+k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
+               uint32_t gen_lo, uint32_t c3a, uint32_t c3b, int32_t* __restrict__ parents, int32_t e,
+               int32_t top_blocks, int32_t per_block, Rec* __restrict__ partial, int32_t* __restrict__ elites,
+               unsigned int* __restrict__ done) {
+    if ((int32_t)blockIdx.x >= top_blocks) {
+        const int32_t i = ((int32_t)blockIdx.x - top_blocks) * blockDim.x + threadIdx.x;
+        if (i < 2 * pairs) tournament_thread(F, n, tournament, i, keys, gen_lo, (i & 1) ? c3b : c3a, parents);
+        return;
+    }
+    __shared__ Rec s_warp[8];
+    __shared__ bool s_last;
+    const int32_t lo = blockIdx.x * per_block;
+    const int32_t count = max(0, min(per_block, n - lo));
+    Rec prev;
+    prev.key = 0;
+    prev.idx = -1;
+    prev.pad = 0;
+    for (int32_t r = 0; r < e; ++r) {
+        Rec best = block_next_best<true>(F + lo, count, lo, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
+        prev = best;
+        if (best.idx < 0) {  // fewer than e items in this slice: mark the rest empty
+            for (int32_t r2 = r + 1 + threadIdx.x; r2 < e; r2 += blockDim.x)
+                partial[(int64_t)blockIdx.x * e + r2] = best;
+            break;
+        }
+    }
+    __threadfence();  // every thread's records before the CTA is counted as finished
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(done, 1u) == (unsigned int)(top_blocks - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    prev.key = 0;
+    prev.idx = -1;
+    for (int32_t r = 0; r < e; ++r) {
+        Rec best = block_next_best<false>(partial, top_blocks * e, 0, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) elites[r] = best.idx;
+        prev = best;
+    }
+    if (threadIdx.x == 0) *done = 0u;
+}
+
+cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
+                                uint64_t gen, int32_t* parents, int32_t e, int32_t* elites, void* scratch,
+                                unsigned int* done, cudaStream_t s) {
+    const int top_b = e > 0 ? top_blocks(n) : 0;
+    const int sel_b = (2 * pairs + 255) / 256;
+    if (top_b + sel_b == 0) return cudaSuccess;
+    const int32_t per_block = top_b ? (n + top_b - 1) / top_b : 0;
+    k_select_stage<<<top_b + sel_b, 256, 0, s>>>(F, n, tournament, pairs, keys, (uint32_t)gen,
+                                                 counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), parents, e,
+                                                 top_b, per_block, reinterpret_cast<Rec*>(scratch), elites, done);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 // Uniform crossover + uniform mutation, fused: one warp per pair of children.  Lane l handles the
 // int4 at genes 4l..4l+3 of every block of 128 genes: two parent loads, two Philox calls (one per
@@ -517,7 +605,7 @@ __device__ __forceinline__ int32_t mutate(uint32_t w, int32_t gene, int32_t kmin
 }
 
 template <int UNROLL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
          int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents, const int32_t* __restrict__ elites,
          Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr16) {
@@ -592,8 +680,9 @@ cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t 
                           Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s) {
     const int64_t warps = (int64_t)pairs + elitism;
     if (warps <= 0) return cudaSuccess;
+    // one warp per pair, no grid-stride: measured faster than a persistent grid at population 65536
     int64_t blocks = (warps + 7) / 8;
-    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    if (blocks > 0x7FFFFFFF) blocks = 0x7FFFFFFF;
     k_evolve<2><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
                                             (uint32_t)gen, counter3(STREAM_MUT, gen), thr16);
     return cudaGetLastError();
