@@ -62,6 +62,11 @@ typedef struct {
  * sum_j X_j (predicted cluster progress in samples per second). */
 #define ONES_FLAG_SRUF 1u
 
+/* Score each new population with a separate pass over it instead of inside the kernel that
+ * writes it.  Results are identical; this only selects the launch sequence (used to time the
+ * crossover/mutation and the fitness kernels on their own). */
+#define ONES_FLAG_UNFUSED 2u
+
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
 #define ONES_MAX_ELITES 256   /* elitism <= 256 */
 
@@ -195,7 +200,8 @@ int ones_kernel_launches(const ones_ctx* ctx, uint64_t* launches);
 
 /* Per-stage device time.  With profiling on, ones_evolve and ones_evaluate bracket
  * each kernel with CUDA events.  ones_stage_times synchronises and returns, for
- * stage s in {0 fitness, 1 select+elites, 2 evolve}, the summed milliseconds
+ * stage s in {0 fitness (separate scoring passes), 1 select+elites, 2 evolve (crossover, mutation
+ * and, unless ONES_FLAG_UNFUSED, the scoring of the children)}, the summed milliseconds
  * ms[s] and launch counts count[s] since the last call, then clears them. */
 int ones_set_profiling(ones_ctx* ctx, int on);
 int ones_stage_times(ones_ctx* ctx, double ms[3], uint64_t count[3]);

@@ -17,6 +17,7 @@ from . import build as _build
 from .inputs import JOB_DTYPE, SearchParams
 
 FLAG_SRUF = 1
+FLAG_UNFUSED = 2
 MAX_ELITES = 256
 
 ERRORS = {0: "ONES_OK", -1: "ONES_ERR_NULL", -2: "ONES_ERR_BAD_JOB", -3: "ONES_ERR_BAD_PARAM",

@@ -90,6 +90,7 @@ struct ones_ctx {
     bool f_valid = false;
     uint64_t gen = 0;
     Tables tab{};
+    bool fused = false;  // children are scored inside the evolve kernel
     std::vector<ones_job> h_jobs;  // the job table the device tables were built from
     uint64_t launches = 0;
     int last_cuda = 0;
@@ -157,6 +158,13 @@ void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
     c->tab.range = reinterpret_cast<int32_t*>(c->ws + c->L.range);
     c->tab.jpad = jpad_of(n_jobs);
     c->tab.k1 = kmax + 1;
+    // the fused evolve+score kernel keeps GPU counts as 16-bit values in shared memory
+    bool narrow = true;
+    for (int32_t j = 0; j < n_jobs; ++j) {
+        const int64_t b = (int64_t)jobs[j].b0 << jobs[j].kmax, m = jobs[j].max_per_gpu;
+        if ((b + m - 1) / m > 65535) narrow = false;
+    }
+    c->fused = narrow && !(c->prm.flags & ONES_FLAG_UNFUSED) && evolve_score_smem(c->tab) <= (size_t)kMaxSmemPerBlock;
 }
 
 // ---- per-stage timing with CUDA events on the handle's stream ----
@@ -372,14 +380,20 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         if ((rc = prof_end(c)) != ONES_OK) return rc;
 
         if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
-        CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs, c->parents(),
-                            c->elites(), c->tab, keys, c->gen, c->thr16, c->stream));
+        if (c->fused) {
+            CU(c, launch_evolve_score(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs,
+                                      c->parents(), c->elites(), c->tab, keys, c->gen, c->thr16, c->cap,
+                                      c->prm.penalty, c->F(), c->G(), c->stream));
+        } else {
+            CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs, c->parents(),
+                                c->elites(), c->tab, keys, c->gen, c->thr16, c->stream));
+        }
         c->launches += 1;
         if ((rc = prof_end(c)) != ONES_OK) return rc;
 
         c->cur ^= 1;
         c->gen += 1;
-        if ((rc = run_fitness(c)) != ONES_OK) return rc;
+        if (!c->fused && (rc = run_fitness(c)) != ONES_OK) return rc;
     }
     return ONES_OK;
 }

@@ -62,6 +62,12 @@ cudaError_t launch_top(const double* F, int32_t n, int32_t e, int32_t* idx_out, 
 cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                           int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                           Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s);
+// crossover + mutation + scoring of the children in one pass; needs evolve_score_smem(t) <= kMaxSmemPerBlock
+size_t evolve_score_smem(Tables t);
+cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
+                                int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
+                                Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
+                                double penalty, double* F, int32_t* G, cudaStream_t s);
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,

@@ -600,15 +600,18 @@ cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, 
 // child row; counter = (int4 index, row, generation, stream)), two child stores.  Warps past the
 // last pair copy the elites to rows 0..E-1.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ int32_t mutate(uint32_t w, int32_t gene, int32_t kmin, int32_t range, uint32_t thr16) {
-    return ((w >> 16) < thr16) ? draw_gene(w, kmin, range) : gene;
+// The mutation decision compares the word's high half with thr16; as (w >> 16) < thr16 is
+// w < (thr16 << 16) for thr16 < 65536, kernels take thr32 = thr16 << 16 and ALWAYS for thr16 = 65536.
+template <bool ALWAYS>
+__device__ __forceinline__ int32_t mutate(uint32_t w, int32_t gene, int32_t kmin, int32_t range, uint32_t thr32) {
+    return (ALWAYS || w < thr32) ? draw_gene(w, kmin, range) : gene;
 }
 
-template <int UNROLL>
+template <int UNROLL, bool ALWAYS>
 __global__ void __launch_bounds__(256, 4)
 k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
          int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents, const int32_t* __restrict__ elites,
-         Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr16) {
+         Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr32) {
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
@@ -657,16 +660,16 @@ k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld,
                     c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
                     c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
                     c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
-                    c0.x = mutate(w0.x, c0.x, kmin.x, range.x, thr16);
-                    c0.y = mutate(w0.y, c0.y, kmin.y, range.y, thr16);
-                    c0.z = mutate(w0.z, c0.z, kmin.z, range.z, thr16);
-                    c0.w = mutate(w0.w, c0.w, kmin.w, range.w, thr16);
+                    c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
+                    c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
+                    c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
+                    c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
                     C0[v] = c0;
                     if (has1) {
-                        c1.x = mutate(w1.x, c1.x, kmin.x, range.x, thr16);
-                        c1.y = mutate(w1.y, c1.y, kmin.y, range.y, thr16);
-                        c1.z = mutate(w1.z, c1.z, kmin.z, range.z, thr16);
-                        c1.w = mutate(w1.w, c1.w, kmin.w, range.w, thr16);
+                        c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
+                        c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
+                        c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
+                        c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
                         C1[v] = c1;
                     }
                 }
@@ -683,8 +686,182 @@ cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t 
     // one warp per pair, no grid-stride: measured faster than a persistent grid at population 65536
     int64_t blocks = (warps + 7) / 8;
     if (blocks > 0x7FFFFFFF) blocks = 0x7FFFFFFF;
-    k_evolve<2><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
-                                            (uint32_t)gen, counter3(STREAM_MUT, gen), thr16);
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    if (thr16 >= 65536u)
+        k_evolve<2, true><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+                                                      (uint32_t)gen, counter3(STREAM_MUT, gen), thr32);
+    else
+        k_evolve<2, false><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+                                                       (uint32_t)gen, counter3(STREAM_MUT, gen), thr32);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Crossover + mutation + scoring in one pass: as k_evolve, and each child is scored from registers
+// while it is written, so the new population is not read back for its fitness.  One persistent CTA
+// per SM holds the model tables (and the per-job ranges, packed to bytes) in shared memory; a warp
+// takes one pair of children at a time.  Scores are summed in the same fixed order as k_fitness
+// (lane l accumulates the genes it owns in increasing job order, then the butterfly), so F and G
+// are bit-identical to scoring the written rows afterwards.  Elite rows are copied and re-scored.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void score4(const int4 g, int32_t base, uint32_t kcap, int32_t jpad,
+                                       const double* __restrict__ sX, const uint16_t* __restrict__ sG,
+                                       double& sum, int32_t& gpus) {
+    const int32_t i0 = (int32_t)min((uint32_t)g.x, kcap) * jpad + base;
+    const int32_t i1 = (int32_t)min((uint32_t)g.y, kcap) * jpad + base + 32;
+    const int32_t i2 = (int32_t)min((uint32_t)g.z, kcap) * jpad + base + 64;
+    const int32_t i3 = (int32_t)min((uint32_t)g.w, kcap) * jpad + base + 96;
+    sum = __dadd_rn(sum, sX[i0]); gpus += sG[i0];
+    sum = __dadd_rn(sum, sX[i1]); gpus += sG[i1];
+    sum = __dadd_rn(sum, sX[i2]); gpus += sG[i2];
+    sum = __dadd_rn(sum, sX[i3]); gpus += sG[i3];
+}
+
+// Shared memory: X planes (fp64), g planes narrowed to 16 bits (the host checks that every GPU count
+// fits), kmin and range per job (int32).
+template <int THREADS, int UNROLL, bool ALWAYS>
+__global__ void __launch_bounds__(THREADS, 1)
+k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
+               int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents,
+               const int32_t* __restrict__ elites, Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3,
+               uint32_t thr32, int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const int32_t jpad = t.jpad;
+    double* sX = reinterpret_cast<double*>(smem_raw);
+    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
+    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
+    int4* sRange = sKmin + jpad / 4;
+    {
+        const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
+            const int4 g = gG[i];
+            reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
+                                                         (uint32_t)g.z | ((uint32_t)g.w << 16));
+        }
+        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
+            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
+            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const uint32_t kcap = (uint32_t)t.k1;
+
+    for (int64_t w = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); w < (int64_t)pairs + elitism;
+         w += total_warps) {
+        double sum0 = 0.0, sum1 = 0.0;
+        int32_t gp0 = 0, gp1 = 0;
+        int32_t slot0, slot1;
+        bool has1;
+        if (w >= pairs) {  // survivor: copy unchanged and score again
+            slot0 = (int32_t)(w - pairs);
+            slot1 = slot0;
+            has1 = false;
+            const int4* from = reinterpret_cast<const int4*>(src + (int64_t)elites[slot0] * ld);
+            int4* to = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
+            for (int32_t v = lane; v < nvec; v += 32) {
+                const int4 g = from[v];
+                to[v] = g;
+                score4(g, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
+            }
+        } else {
+            const int32_t q = (int32_t)w;
+            const int32_t pa = parents[2 * q], pb = parents[2 * q + 1];
+            slot0 = elitism + 2 * q;
+            slot1 = slot0 + 1;
+            has1 = slot1 < n;
+            const int4* A = reinterpret_cast<const int4*>(src + (int64_t)pa * ld);
+            const int4* B = reinterpret_cast<const int4*>(src + (int64_t)pb * ld);
+            int4* C0 = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
+            int4* C1 = reinterpret_cast<int4*>(dst + (int64_t)slot1 * ld);
+            for (int32_t v0 = 0; v0 < nvec; v0 += 32 * UNROLL) {
+                int4 a[UNROLL], b[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int32_t v = v0 + u * 32 + lane;
+                    if (v < nvec) {
+                        a[u] = A[v];
+                        b[u] = B[v];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int32_t v = v0 + u * 32 + lane;
+                    if (v < nvec) {
+                        const int4 kmin = sKmin[v];
+                        const int4 range = sRange[v];
+                        const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+                        const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                        int4 c0, c1;
+                        c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
+                        c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
+                        c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
+                        c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
+                        c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
+                        c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
+                        c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
+                        c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
+                        C0[v] = c0;
+                        const int32_t base = (v >> 5) * 128 + lane;
+                        score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
+                        if (has1) {
+                            c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
+                            c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
+                            c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
+                            c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
+                            C1[v] = c1;
+                            score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
+            gp0 += __shfl_xor_sync(0xFFFFFFFFu, gp0, off);
+            sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
+            gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
+        }
+        if (lane == 0) {
+            const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
+            F[slot0] = __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+            G[slot0] = gp0;
+            if (has1) {
+                const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                F[slot1] = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                G[slot1] = gp1;
+            }
+        }
+    }
+}
+
+size_t evolve_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (size_t)t.jpad * 8; }
+
+cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
+                                int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
+                                Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
+                                double penalty, double* F, int32_t* G, cudaStream_t s) {
+    const int64_t warps = (int64_t)pairs + elitism;
+    if (warps <= 0) return cudaSuccess;
+    const size_t smem = evolve_score_smem(t);
+    if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
+    constexpr int kThreads = 1024;  // one CTA per SM; measured best with one int4 per parent in flight per lane
+    int64_t blocks = (warps + kThreads / 32 - 1) / (kThreads / 32);
+    if (blocks > kSMs) blocks = kSMs;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    auto kern = thr16 >= 65536u ? k_evolve_score<kThreads, 1, true> : k_evolve_score<kThreads, 1, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
+    if (e != cudaSuccess) return e;
+    kern<<<(int)blocks, kThreads, smem, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+                                             (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G);
     return cudaGetLastError();
 }
 

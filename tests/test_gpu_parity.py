@@ -124,10 +124,10 @@ def test_randomize_parity(ones):
         _same_state(g, o)
 
 
-@pytest.mark.parametrize("name,gens", [("tiny", 10), ("paper", 100)])
-def test_evolve_parity_named_workloads(ones, name, gens):
+@pytest.mark.parametrize("name,gens,flags", [("tiny", 10, 0), ("paper", 100, 0), ("paper", 100, 2)])
+def test_evolve_parity_named_workloads(ones, name, gens, flags):
     w = inputs.WORKLOADS[name]()
-    g, o = _pair(ones, w)
+    g, o = _pair(ones, w, flags=flags)
     g.randomize(w.seed)
     o.randomize(w.seed)
     done = 0
@@ -160,7 +160,8 @@ def test_evolve_parity_mid_sampled_generations(ones):
 
 @pytest.mark.parametrize("kw", [dict(elitism=0), dict(elitism=1), dict(elitism=5, tournament=1),
                                 dict(tournament=9), dict(p_mut=0.0), dict(p_mut=1.0), dict(p_mut=0.02, tournament=8),
-                                dict(penalty=0.0), dict(penalty=37.5)])
+                                dict(penalty=0.0), dict(penalty=37.5), dict(flags=2), dict(flags=2, p_mut=1.0),
+                                dict(flags=3)])
 def test_evolve_parity_parameter_corners(ones, kw):
     w = inputs.custom(37, 48, 101, 6, seed=7, kmax=6, pinned=4)
     g, o = _pair(ones, w, **kw)
@@ -317,9 +318,10 @@ def test_errors_are_codes_not_faults(ones):
 
 
 # ---- full size, in the configuration the benchmark times --------------------------------------------
-def test_large_config_parity_full_population(ones):
+@pytest.mark.parametrize("flags", [0, 2])  # children scored inside the evolve kernel / by a separate pass
+def test_large_config_parity_full_population(ones, flags):
     w = inputs.large()
-    g, o = _pair(ones, w)
+    g, o = _pair(ones, w, flags=flags)
     g.randomize(w.seed)
     o.randomize(w.seed)
     assert (g.get_population() == o.get_population()).all()
