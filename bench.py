@@ -147,18 +147,66 @@ def run_reference(args, w):
 
 
 # ----------------------------------------------------------------------------------------------
+# online loop: per-round search latency and simulated job completion time
+# ----------------------------------------------------------------------------------------------
+def run_online(args):
+    import torch
+    from paper_2108_03645_b200 import binding, online
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    trace = inputs.online_trace()
+
+    def gpu_engine(jobs, capacity, pop, params, n_jobs_max):
+        return binding.Search(jobs, capacity, pop, params, n_jobs_max=n_jobs_max)
+
+    def cpu_engine(jobs, capacity, pop, params, n_jobs_max):
+        import oracle
+        return oracle.Search(jobs, capacity, pop, elitism=params.elitism, tournament=params.tournament,
+                             p_mut=params.p_mut, penalty=params.penalty, flags=params.flags)
+
+    online.simulate(trace, gpu_engine, max_rounds=20, sync=torch.cuda.synchronize)  # warm-up
+    res = online.simulate(trace, gpu_engine, keep_schedules=True, sync=torch.cuda.synchronize)
+    lat = np.array(res.latency_s) * 1e3
+    line = {"metric": "online_round_latency_ms", "value": float(lat.mean()), "unit": "ms per scheduling round "
+            "(ones_update_jobs + 50 generations of a 4096-candidate population + ones_best with repair)",
+            "n_gpus": 1, "higher_is_better": False, "data": "synthetic", "dtype": "f64",
+            "config": {"workload": "online", "trace_jobs": int(trace.jobs.shape[0]), "capacity": trace.capacity,
+                       "population": trace.pop, "generations_per_round": trace.generations,
+                       "period_s": trace.period_s},
+            "rounds": res.rounds, "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
+            "max_ms": float(lat.max()), "mean_active_jobs": float(np.mean(res.active)),
+            "max_active_jobs": int(max(res.active)), "mean_jct_s": res.mean_jct,
+            "jobs_finished": int(np.isfinite(res.jct).sum())}
+    if not args.no_cpu_baseline:
+        k = 12
+        t0 = time.perf_counter()
+        ref = online.simulate(trace, cpu_engine, max_rounds=k, keep_schedules=True)
+        dt = time.perf_counter() - t0
+        same = all(ia == ib and (ga == gb).all() for (_, ia, ga), (_, ib, gb) in zip(res.deployed, ref.deployed))
+        line["cpu_baseline"] = {"value": 1e3 * float(np.mean(ref.latency_s)), "unit": "ms per scheduling round",
+                                "cores": 1, "kind": "oracle",
+                                "sample": f"first {k} rounds of the same trace; {dt:.1f} s",
+                                "schedules_identical_to_gpu": bool(same)}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--workload", default="large", choices=sorted(inputs.WORKLOADS) + ["online"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-events", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling a smaller case)")
     args = ap.parse_args()
+    if args.workload == "online":
+        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
+            run_online(args)
+        return
     w = inputs.WORKLOADS[args.workload]()
     if args.pop:
         import dataclasses

@@ -1,0 +1,81 @@
+"""The online scheduling loop (host simulation) driven by the CPU oracle, and by the CUDA library."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2108_03645_b200 import inputs, online
+
+
+def oracle_engine(jobs, capacity, pop, params, n_jobs_max):
+    return oracle.Search(jobs, capacity, pop, elitism=params.elitism, tournament=params.tournament,
+                         p_mut=params.p_mut, penalty=params.penalty, flags=params.flags)
+
+
+def small_trace(seed=0, n=40, capacity=16, pop=64, gens=6):
+    return inputs.online_trace(n, seed, mean_interarrival_s=20.0, median_length=2e5, sigma=1.0,
+                               capacity=capacity, pop=pop, generations=gens)
+
+
+def test_online_loop_invariants_with_oracle():
+    tr = small_trace()
+    res = online.simulate(tr, oracle_engine, keep_schedules=True)
+    assert np.isfinite(res.jct).all() and (res.jct > 0).all()          # every job finishes
+    assert max(res.gpus_used) <= tr.capacity                           # repair holds the capacity
+    assert len(res.latency_s) == res.rounds == len(res.deployed)
+    # limits: a job is at its smallest batch in its first round and may double each round after
+    first = {}
+    for rnd, ids, genome in res.deployed:
+        for c, j in enumerate(ids):
+            first.setdefault(j, rnd)
+            assert genome[c] <= min(7, rnd - first[j])
+    # no job can finish faster than at its best throughput over all exponents
+    for j in range(tr.jobs.shape[0]):
+        best_rate = max(oracle.model(tr.jobs, j, k)[0] for k in range(8))
+        assert res.jct[j] >= tr.length[j] / best_rate * (1 - 1e-12)
+    # deterministic
+    again = online.simulate(tr, oracle_engine)
+    assert (again.jct == res.jct).all() and again.best_fitness == res.best_fitness
+
+
+def test_online_loop_skips_idle_time_and_respects_max_rounds():
+    tr = inputs.online_trace(6, 3, mean_interarrival_s=2000.0, median_length=1e4, sigma=0.5, capacity=8, pop=32,
+                             generations=3)
+    res = online.simulate(tr, oracle_engine)
+    assert np.isfinite(res.jct).all()
+    assert res.rounds < 40  # idle stretches between far-apart arrivals are jumped over
+    cut = online.simulate(tr, oracle_engine, max_rounds=2)
+    assert cut.rounds == 2 and np.isnan(cut.jct).any()
+
+
+def test_online_loop_regrows_engine_when_job_set_outgrows_it():
+    tr = inputs.online_trace(30, 1, mean_interarrival_s=25.0, median_length=5e6, sigma=0.3, capacity=8, pop=32,
+                             generations=2)
+    made = []
+
+    def eng(jobs, capacity, pop, params, n_jobs_max):
+        made.append((jobs.shape[0], n_jobs_max))
+        return oracle_engine(jobs, capacity, pop, params, n_jobs_max)
+
+    res = online.simulate(tr, eng, n_jobs_max=2, max_rounds=8)
+    assert len(made) >= 2 and all(n <= m for n, m in made)
+    assert max(res.gpus_used) <= 8
+
+
+@pytest.mark.gpu
+def test_online_loop_gpu_matches_oracle():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2108_03645_b200 import binding
+
+    def gpu_engine(jobs, capacity, pop, params, n_jobs_max):
+        return binding.Search(jobs, capacity, pop, params, n_jobs_max=n_jobs_max)
+
+    tr = small_trace(seed=2, n=60, capacity=24, pop=256, gens=8)
+    a = online.simulate(tr, gpu_engine, keep_schedules=True, n_jobs_max=16, sync=torch.cuda.synchronize)
+    b = online.simulate(tr, oracle_engine, keep_schedules=True, n_jobs_max=16)
+    assert a.rounds == b.rounds and a.gpus_used == b.gpus_used and a.active == b.active
+    assert a.best_fitness == b.best_fitness
+    for (ra, ia, ga), (rb, ib, gb) in zip(a.deployed, b.deployed):
+        assert ra == rb and ia == ib and (ga == gb).all()
+    assert (a.jct == b.jct).all()
