@@ -26,7 +26,7 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, G, parents, elites, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
+    size_t pop0, pop1, F, F1, G, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
         out_gpus, out_rate, out_rec, exp_X, exp_G, status, total;
 };
 
@@ -43,9 +43,11 @@ Layout make_layout(int32_t jmax, int32_t pop) {
     L.pop0 = take((size_t)pop * ldm * 4);
     L.pop1 = take((size_t)pop * ldm * 4);
     L.F = take((size_t)pop * 8);
+    L.F1 = take((size_t)pop * 8);
     L.G = take((size_t)pop * 4);
     L.parents = take(pairs * 2 * 4);
     L.elites = take((size_t)ONES_MAX_ELITES * 4);
+    L.elites1 = take((size_t)ONES_MAX_ELITES * 4);
     L.best_idx = take(16);
     L.X = take((size_t)kPlanesMax * jp * 8);
     L.Gt = take((size_t)kPlanesMax * jp * 4);
@@ -53,7 +55,10 @@ Layout make_layout(int32_t jmax, int32_t pop) {
     L.range = take(jp * 4);
     L.jobs = take((size_t)jmax * sizeof(ones_job));
     L.remap = take((size_t)jmax * 4);
-    L.top = take(top_scratch_bytes(pop, ONES_MAX_ELITES));
+    {
+        const size_t a = top_scratch_bytes(pop, ONES_MAX_ELITES), b = generation_scratch_bytes(ONES_MAX_ELITES);
+        L.top = take(a > b ? a : b);
+    }
     L.work = take(3 * jp * 4);
     L.out_genome = take((size_t)jmax * 4);
     L.out_gpus = take((size_t)jmax * 4);
@@ -86,7 +91,11 @@ struct ones_ctx {
     uint32_t thr16 = 0;
     char* ws = nullptr;
     Layout L{};
-    int cur = 0;
+    int cur = 0;            // population buffer in force
+    int fcur = 0;           // score buffer in force
+    int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
+    int elast = 0;          // elites buffer used by the last generation
+    bool elites_valid = false;
     bool f_valid = false;
     uint64_t gen = 0;
     Tables tab{};
@@ -97,10 +106,11 @@ struct ones_ctx {
     Prof prof;
 
     int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
-    double* F() { return reinterpret_cast<double*>(ws + L.F); }
+    double* Fbuf(int which) { return reinterpret_cast<double*>(ws + (which ? L.F1 : L.F)); }
+    double* F() { return Fbuf(fcur); }
     int32_t* G() { return reinterpret_cast<int32_t*>(ws + L.G); }
     int32_t* parents() { return reinterpret_cast<int32_t*>(ws + L.parents); }
-    int32_t* elites() { return reinterpret_cast<int32_t*>(ws + L.elites); }
+    int32_t* elites(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.elites1 : L.elites)); }
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
     ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs); }
     int32_t* remap() { return reinterpret_cast<int32_t*>(ws + L.remap); }
@@ -210,6 +220,7 @@ int run_fitness(ones_ctx* c) {
                          c->stream));
     c->launches += 1;
     c->f_valid = true;
+    c->elites_valid = false;
     return prof_end(c);
 }
 
@@ -293,6 +304,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     }
     c->cur = 0;
     c->f_valid = false;
+    c->elites_valid = false;
     *out = c;
     return ONES_OK;
 }
@@ -309,6 +321,7 @@ int ones_randomize(ones_ctx* c, uint64_t seed) {
     CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->J, c->tab, make_round_keys(seed), c->stream));
     c->launches += 1;
     c->f_valid = false;
+    c->elites_valid = false;
     return ONES_OK;
 }
 
@@ -325,6 +338,7 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
         CU(c, cudaStreamSynchronize(c->stream));
     }
     c->f_valid = false;
+    c->elites_valid = false;
     return ONES_OK;
 }
 
@@ -371,22 +385,51 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
     const RoundKeys keys = make_round_keys(seed);
     const int32_t E = c->prm.elitism;
+    unsigned int* done = reinterpret_cast<unsigned int*>(c->status() + 1);
+    const GenerationShape shape = c->fused ? generation_shape(c->tab, c->pairs, E) : GenerationShape{0, 0, 0, 0};
+    if (shape.blocks > 0) {
+        // one launch per generation; each launch also leaves the elites of the population it wrote
+        if (E > 0 && !c->elites_valid) {
+            if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
+            int nl = 0;
+            CU(c, launch_top(c->F(), c->N, E, c->elites(c->ecur), c->ws + c->L.top, c->stream, &nl));
+            c->launches += (uint64_t)nl;
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+        }
+        for (int32_t it = 0; it < generations; ++it) {
+            if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
+            CU(c, launch_generation(shape, c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs,
+                                    c->prm.tournament, c->Fbuf(c->fcur), c->Fbuf(c->fcur ^ 1), c->G(), c->parents(),
+                                    c->elites(c->ecur), c->elites(c->ecur ^ 1), c->tab, keys, c->gen, c->thr16, c->cap,
+                                    c->prm.penalty, c->ws + c->L.top, done, c->stream));
+            c->launches += 1;
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+            c->elast = c->ecur;
+            c->cur ^= 1;
+            c->fcur ^= 1;
+            c->ecur ^= 1;
+            c->elites_valid = true;
+            c->gen += 1;
+        }
+        return ONES_OK;
+    }
     for (int32_t it = 0; it < generations; ++it) {
         if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
         CU(c, launch_select_stage(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), E,
-                                  c->elites(), c->ws + c->L.top, reinterpret_cast<unsigned int*>(c->status() + 1),
-                                  c->stream));
+                                  c->elites(0), c->ws + c->L.top, done, c->stream));
         c->launches += 1;
+        c->elast = 0;
+        c->elites_valid = false;
         if ((rc = prof_end(c)) != ONES_OK) return rc;
 
         if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
         if (c->fused) {
             CU(c, launch_evolve_score(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs,
-                                      c->parents(), c->elites(), c->tab, keys, c->gen, c->thr16, c->cap,
+                                      c->parents(), c->elites(0), c->tab, keys, c->gen, c->thr16, c->cap,
                                       c->prm.penalty, c->F(), c->G(), c->stream));
         } else {
             CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs, c->parents(),
-                                c->elites(), c->tab, keys, c->gen, c->thr16, c->stream));
+                                c->elites(0), c->tab, keys, c->gen, c->thr16, c->stream));
         }
         c->launches += 1;
         if ((rc = prof_end(c)) != ONES_OK) return rc;
@@ -452,6 +495,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
     c->ld = new_ld;
     c->cap = capacity;
     c->f_valid = false;
+    c->elites_valid = false;
     return ONES_OK;
 }
 
@@ -460,7 +504,7 @@ int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
     if (h_parents && c->pairs > 0)
         CU(c, cudaMemcpyAsync(h_parents, c->parents(), (size_t)c->pairs * 8, cudaMemcpyDeviceToHost, c->stream));
     if (h_elites && c->prm.elitism > 0)
-        CU(c, cudaMemcpyAsync(h_elites, c->elites(), (size_t)c->prm.elitism * 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(c, cudaMemcpyAsync(h_elites, c->elites(c->elast), (size_t)c->prm.elitism * 4, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
     return ONES_OK;
 }

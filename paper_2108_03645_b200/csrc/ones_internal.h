@@ -68,6 +68,19 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
                                 int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                                 Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
                                 double penalty, double* F, int32_t* G, cudaStream_t s);
+// One launch per generation (tournaments + crossover + mutation + scoring + the next generation's elites).
+struct GenerationShape {
+    int blocks, threads;  // blocks == 0: not applicable, use the multi-launch sequence
+    int32_t queue_cap;
+    size_t smem;
+};
+size_t generation_scratch_bytes(int32_t e);
+GenerationShape generation_shape(Tables t, int32_t pairs, int32_t elitism);
+cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t* dst, int64_t ld, int32_t n,
+                              int32_t n_jobs, int32_t elitism, int32_t pairs, int32_t tournament, const double* F_old,
+                              double* F_new, int32_t* G, int32_t* parents, const int32_t* elites,
+                              int32_t* elites_next, Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16,
+                              int32_t capacity, double penalty, void* scratch, unsigned int* done, cudaStream_t s);
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,

@@ -398,8 +398,9 @@ __device__ __forceinline__ bool before(unsigned long long ka, int32_t ia, unsign
 }
 
 // Block-wide best record that ranks strictly after `prev` (or any record when !have_prev).
-// RAW: items are scores F[i] with index lo + i; else items are Rec.
-template <bool RAW>
+// SRC 0: items are scores F[i] with index lo + i; 1: Rec in global memory, possibly written by other
+// CTAs of the same launch (read through L2); 2: Rec in shared memory.  s_warp holds one Rec per warp.
+template <int SRC>
 __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, bool have_prev, Rec prev,
                                Rec* s_warp) {
     Rec best;
@@ -409,12 +410,13 @@ __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, boo
     for (int32_t i = threadIdx.x; i < count; i += blockDim.x) {
         unsigned long long k;
         int32_t id;
-        if (RAW) {
+        if (SRC == 0) {
             k = score_key(reinterpret_cast<const double*>(items)[i]);
             id = lo + i;
         } else {
-            // records may have been written by other CTAs of the same launch: read them through L2
-            const int4 raw = __ldcg(reinterpret_cast<const int4*>(items) + i);
+            int4 raw;
+            if (SRC == 1) raw = __ldcg(reinterpret_cast<const int4*>(items) + i);
+            else raw = reinterpret_cast<const int4*>(items)[i];
             k = ((unsigned long long)(uint32_t)raw.y << 32) | (uint32_t)raw.x;
             id = raw.z;
             if (id < 0) continue;
@@ -448,7 +450,7 @@ __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, boo
 
 __global__ void __launch_bounds__(256) k_top_partial(const double* __restrict__ F, int32_t n, int32_t e,
                                                      int32_t per_block, Rec* __restrict__ partial) {
-    __shared__ Rec s_warp[8];
+    __shared__ Rec s_warp[32];
     const int32_t lo = blockIdx.x * per_block;
     const int32_t count = min(per_block, n - lo);
     Rec prev;
@@ -456,7 +458,7 @@ __global__ void __launch_bounds__(256) k_top_partial(const double* __restrict__ 
     prev.idx = -1;
     prev.pad = 0;
     for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<true>(F + lo, count > 0 ? count : 0, lo, r > 0, prev, s_warp);
+        Rec best = block_next_best<0>(F + lo, count > 0 ? count : 0, lo, r > 0, prev, s_warp);
         if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
         prev = best;
         if (best.idx < 0) {  // fewer than e items in this block: mark the rest empty
@@ -469,13 +471,13 @@ __global__ void __launch_bounds__(256) k_top_partial(const double* __restrict__ 
 
 __global__ void __launch_bounds__(256) k_top_final(const Rec* __restrict__ partial, int32_t count, int32_t e,
                                                    int32_t* __restrict__ idx_out) {
-    __shared__ Rec s_warp[8];
+    __shared__ Rec s_warp[32];
     Rec prev;
     prev.key = 0;
     prev.idx = -1;
     prev.pad = 0;
     for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<false>(partial, count, 0, r > 0, prev, s_warp);
+        Rec best = block_next_best<1>(partial, count, 0, r > 0, prev, s_warp);
         if (threadIdx.x == 0) idx_out[r] = best.idx;
         prev = best;
     }
@@ -547,7 +549,7 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
         if (i < 2 * pairs) tournament_thread(F, n, tournament, i, keys, gen_lo, (i & 1) ? c3b : c3a, parents);
         return;
     }
-    __shared__ Rec s_warp[8];
+    __shared__ Rec s_warp[32];
     __shared__ bool s_last;
     const int32_t lo = blockIdx.x * per_block;
     const int32_t count = max(0, min(per_block, n - lo));
@@ -556,7 +558,7 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
     prev.idx = -1;
     prev.pad = 0;
     for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<true>(F + lo, count, lo, r > 0, prev, s_warp);
+        Rec best = block_next_best<0>(F + lo, count, lo, r > 0, prev, s_warp);
         if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
         prev = best;
         if (best.idx < 0) {  // fewer than e items in this slice: mark the rest empty
@@ -574,7 +576,7 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
     prev.key = 0;
     prev.idx = -1;
     for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<false>(partial, top_blocks * e, 0, r > 0, prev, s_warp);
+        Rec best = block_next_best<1>(partial, top_blocks * e, 0, r > 0, prev, s_warp);
         if (threadIdx.x == 0) elites[r] = best.idx;
         prev = best;
     }
@@ -841,6 +843,296 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             }
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// A whole generation in one launch: each warp runs the two tournaments of its pair (one draw per
+// lane, butterfly for the winner), then crossover, mutation and scoring as k_evolve_score, and
+// queues the scores it produced in shared memory; at the end every CTA reduces its queue to its e
+// best and the last CTA to finish merges those lists into the elites of the NEXT generation.
+// F_old is read (tournaments), F_new written: two score buffers.  `done` as in k_select_stage.
+// ---------------------------------------------------------------------------------------------
+// A tournament in two halves so that the score gathers of the NEXT pair are in flight while the
+// current pair's rows are processed: draw (one draw per lane, private best) and reduce (butterfly).
+struct Draw {
+    int32_t idx;
+    double f;
+};
+
+__device__ __forceinline__ Draw tournament_draw(const double* __restrict__ F, int32_t n, int32_t tournament, uint32_t q,
+                                                uint32_t gen_lo, uint32_t c3, const RoundKeys& keys, int lane) {
+    Draw d;
+    d.idx = -1;
+    d.f = 0.0;
+    for (int32_t t0 = 0; t0 < tournament; t0 += 32) {
+        const int32_t t = t0 + lane;
+        if (t < tournament) {
+            const uint4 w4 = philox((uint32_t)(t >> 2), q, gen_lo, c3, keys);
+            const uint32_t w = (t & 2) ? ((t & 1) ? w4.w : w4.z) : ((t & 1) ? w4.y : w4.x);
+            const int32_t idx = (int32_t)__umulhi(w, (uint32_t)n);
+            const double f = F[idx];
+            if (d.idx < 0 || f > d.f || (f == d.f && idx < d.idx)) {
+                d.idx = idx;
+                d.f = f;
+            }
+        }
+    }
+    return d;
+}
+
+__device__ __forceinline__ int32_t tournament_reduce(Draw d) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const int32_t oi = __shfl_xor_sync(0xFFFFFFFFu, d.idx, off);
+        const double of = __shfl_xor_sync(0xFFFFFFFFu, d.f, off);
+        if (oi >= 0 && (d.idx < 0 || of > d.f || (of == d.f && oi < d.idx))) {
+            d.idx = oi;
+            d.f = of;
+        }
+    }
+    return d.idx;
+}
+
+template <int THREADS, int UNROLL, bool ALWAYS>
+__global__ void __launch_bounds__(THREADS, 1)
+k_generation(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
+             int32_t elitism, int32_t pairs, int32_t tournament, const double* __restrict__ F_old,
+             double* __restrict__ F_new, int32_t* __restrict__ G, int32_t* __restrict__ parents,
+             const int32_t* __restrict__ elites, int32_t* __restrict__ elites_next, Tables t, RoundKeys keys,
+             uint32_t gen_lo, uint32_t c3, uint32_t c3a, uint32_t c3b, uint32_t thr32, int32_t capacity,
+             double penalty, Rec* __restrict__ partial, unsigned int* __restrict__ done, int32_t queue_cap) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ Rec s_warp[32];
+    __shared__ int s_queued;
+    __shared__ bool s_last;
+    const int32_t planes = t.k1 + 1;
+    const int32_t jpad = t.jpad;
+    double* sX = reinterpret_cast<double*>(smem_raw);
+    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
+    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
+    int4* sRange = sKmin + jpad / 4;
+    Rec* queue = reinterpret_cast<Rec*>(smem_raw + (size_t)planes * jpad * 10 + (size_t)jpad * 8);
+    {
+        if (threadIdx.x == 0) s_queued = 0;
+        const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
+            const int4 g = gG[i];
+            reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
+                                                         (uint32_t)g.z | ((uint32_t)g.w << 16));
+        }
+        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
+            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
+            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const uint32_t kcap = (uint32_t)t.k1;
+
+    const int64_t w_first = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    Draw da, db;
+    da.idx = db.idx = -1;
+    da.f = db.f = 0.0;
+    if (w_first < pairs) {
+        da = tournament_draw(F_old, n, tournament, (uint32_t)w_first, gen_lo, c3a, keys, lane);
+        db = tournament_draw(F_old, n, tournament, (uint32_t)w_first, gen_lo, c3b, keys, lane);
+    }
+    for (int64_t w = w_first; w < (int64_t)pairs + elitism; w += total_warps) {
+        double sum0 = 0.0, sum1 = 0.0;
+        int32_t gp0 = 0, gp1 = 0;
+        int32_t slot0, slot1;
+        bool has1;
+        if (w >= pairs) {  // survivor: copy unchanged and score again
+            slot0 = (int32_t)(w - pairs);
+            slot1 = slot0;
+            has1 = false;
+            const int4* from = reinterpret_cast<const int4*>(src + (int64_t)elites[slot0] * ld);
+            int4* to = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
+            for (int32_t v = lane; v < nvec; v += 32) {
+                const int4 g = from[v];
+                to[v] = g;
+                score4(g, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
+            }
+        } else {
+            const int32_t q = (int32_t)w;
+            const int32_t pa = tournament_reduce(da);
+            const int32_t pb = tournament_reduce(db);
+            if (w + total_warps < pairs) {  // next pair's draws: their score gathers overlap this pair's rows
+                da = tournament_draw(F_old, n, tournament, (uint32_t)(w + total_warps), gen_lo, c3a, keys, lane);
+                db = tournament_draw(F_old, n, tournament, (uint32_t)(w + total_warps), gen_lo, c3b, keys, lane);
+            }
+            if (lane == 0) {
+                parents[2 * q] = pa;
+                parents[2 * q + 1] = pb;
+            }
+            slot0 = elitism + 2 * q;
+            slot1 = slot0 + 1;
+            has1 = slot1 < n;
+            const int4* A = reinterpret_cast<const int4*>(src + (int64_t)pa * ld);
+            const int4* B = reinterpret_cast<const int4*>(src + (int64_t)pb * ld);
+            int4* C0 = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
+            int4* C1 = reinterpret_cast<int4*>(dst + (int64_t)slot1 * ld);
+            for (int32_t v0 = 0; v0 < nvec; v0 += 32 * UNROLL) {
+                int4 a[UNROLL], b[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int32_t v = v0 + u * 32 + lane;
+                    if (v < nvec) {
+                        a[u] = A[v];
+                        b[u] = B[v];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int32_t v = v0 + u * 32 + lane;
+                    if (v < nvec) {
+                        const int4 kmin = sKmin[v];
+                        const int4 range = sRange[v];
+                        const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+                        const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                        int4 c0, c1;
+                        c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
+                        c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
+                        c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
+                        c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
+                        c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
+                        c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
+                        c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
+                        c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
+                        C0[v] = c0;
+                        const int32_t base = (v >> 5) * 128 + lane;
+                        score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
+                        if (has1) {
+                            c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
+                            c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
+                            c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
+                            c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
+                            C1[v] = c1;
+                            score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
+            gp0 += __shfl_xor_sync(0xFFFFFFFFu, gp0, off);
+            sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
+            gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
+        }
+        if (lane == 0) {
+            const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
+            const double f0 = __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+            F_new[slot0] = f0;
+            G[slot0] = gp0;
+            int32_t at = elitism > 0 ? atomicAdd(&s_queued, has1 ? 2 : 1) : queue_cap;
+            if (at < queue_cap) {
+                Rec r;
+                r.key = score_key(f0);
+                r.idx = slot0;
+                r.pad = 0;
+                queue[at] = r;
+            }
+            if (has1) {
+                const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                const double f1 = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                F_new[slot1] = f1;
+                G[slot1] = gp1;
+                if (at + 1 < queue_cap) {
+                    Rec r;
+                    r.key = score_key(f1);
+                    r.idx = slot1;
+                    r.pad = 0;
+                    queue[at + 1] = r;
+                }
+            }
+        }
+    }
+    if (elitism <= 0) return;
+    // this CTA's e best of what it produced, then the last CTA merges all lists
+    __syncthreads();
+    const int32_t queued = min(s_queued, queue_cap);
+    Rec prev;
+    prev.key = 0;
+    prev.idx = -1;
+    prev.pad = 0;
+    for (int32_t r = 0; r < elitism; ++r) {
+        Rec best = block_next_best<2>(queue, queued, 0, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * elitism + r] = best;
+        prev = best;
+        if (best.idx < 0) {
+            for (int32_t r2 = r + 1 + threadIdx.x; r2 < elitism; r2 += blockDim.x)
+                partial[(int64_t)blockIdx.x * elitism + r2] = best;
+            break;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(done, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    prev.key = 0;
+    prev.idx = -1;
+    for (int32_t r = 0; r < elitism; ++r) {
+        Rec best = block_next_best<1>(partial, (int32_t)gridDim.x * elitism, 0, r > 0, prev, s_warp);
+        if (threadIdx.x == 0) elites_next[r] = best.idx;
+        prev = best;
+    }
+    if (threadIdx.x == 0) *done = 0u;
+}
+
+size_t generation_scratch_bytes(int32_t e) { return (size_t)kSMs * (size_t)e * sizeof(Rec); }
+
+// Launch shape of k_generation for this problem, or blocks = 0 when it does not apply (tables or the
+// score queue do not fit shared memory, or the merge scratch would overflow).
+GenerationShape generation_shape(Tables t, int32_t pairs, int32_t elitism) {
+    GenerationShape g{0, 0, 0, 0};
+    const int64_t warps = (int64_t)pairs + elitism;
+    if (warps <= 0) return g;
+    // Large populations are HBM-bound and measured faster as two launches (k_select_stage, then
+    // k_evolve_score with the parents known up front); the single launch pays off when the generation is
+    // launch-latency-bound.
+    if (warps >= (int64_t)kSMs * 16) return g;
+    g.threads = 256;
+    const int wpb = g.threads / 32;
+    int64_t blocks = (warps + wpb - 1) / wpb;
+    if (blocks > kSMs) blocks = kSMs;  // the merge scratch holds kSMs lists (generation_scratch_bytes)
+    const int64_t total_warps = blocks * wpb;
+    const int64_t per_warp = (warps + total_warps - 1) / total_warps;
+    g.queue_cap = (int32_t)(2 * per_warp * wpb);
+    g.smem = evolve_score_smem(t) + (size_t)g.queue_cap * sizeof(Rec);
+    if (g.smem + 1024 > (size_t)kMaxSmemPerBlock) return g;  // 1 KiB for the kernel's static shared memory
+    g.blocks = (int)blocks;
+    return g;
+}
+
+cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t* dst, int64_t ld, int32_t n,
+                              int32_t n_jobs, int32_t elitism, int32_t pairs, int32_t tournament, const double* F_old,
+                              double* F_new, int32_t* G, int32_t* parents, const int32_t* elites,
+                              int32_t* elites_next, Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16,
+                              int32_t capacity, double penalty, void* scratch, unsigned int* done, cudaStream_t s) {
+    if (shape.blocks <= 0) return cudaErrorInvalidConfiguration;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    const bool always = thr16 >= 65536u;
+    void (*kern)(const int32_t*, int32_t*, int64_t, int32_t, int32_t, int32_t, int32_t, int32_t, const double*,
+                 double*, int32_t*, int32_t*, const int32_t*, int32_t*, Tables, RoundKeys, uint32_t, uint32_t,
+                 uint32_t, uint32_t, uint32_t, int32_t, double, Rec*, unsigned int*, int32_t);
+    kern = always ? k_generation<256, 1, true> : k_generation<256, 1, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
+    if (e != cudaSuccess) return e;
+    kern<<<shape.blocks, shape.threads, shape.smem, s>>>(
+        src, dst, ld, n, n_jobs, elitism, pairs, tournament, F_old, F_new, G, parents, elites, elites_next, t, keys,
+        (uint32_t)gen, counter3(STREAM_MUT, gen), counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), thr32,
+        capacity, penalty, reinterpret_cast<Rec*>(scratch), done, shape.queue_cap);
+    return cudaGetLastError();
 }
 
 size_t evolve_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (size_t)t.jpad * 8; }
