@@ -19,7 +19,8 @@
  *    constraint (Eq. 4) enters as a penalty on sum_j c_j - |C|.
  *  - Uniform crossover gives two complementary children (Section 3.2.2, "Uniform
  *    crossover"); uniform mutation touches each job independently with rate
- *    theta ("Uniform mutation"), never leaving [kmin_j, kmax_j] (limit R_j).
+ *    theta ("Uniform mutation"), never leaving [kmin_j, kmax_j] (limit R_j).  One random word
+ *    per job and pair of siblings carries the crossover bit and both children's mutation draws.
  *  - Selection: tournament for parents, the E best survive unchanged, S* is the
  *    best-scored candidate (Alg. 1, last step).
  */
@@ -189,12 +190,19 @@ uint32_t oracle_thr16(double p_mut) {
     return (uint32_t)t;
 }
 
-/* uniform value in [kmin, kmax] from the 15-bit field of a random word */
-static int32_t draw_gene(uint32_t word, int32_t kmin, int32_t kmax) {
-    uint32_t frac = (word >> 1) & 0x7FFFu;
-    uint32_t range = (uint32_t)(kmax - kmin + 1);
-    return kmin + (int32_t)((frac * range) >> 15);
+/* uniform value in [kmin, kmax] from a 32-bit fraction: kmin + floor(frac * range / 2^32) */
+static int32_t draw_gene(uint32_t frac, int32_t kmin, int32_t kmax) {
+    uint64_t range = (uint64_t)(kmax - kmin + 1);
+    return kmin + (int32_t)(((uint64_t)frac * range) >> 32);
 }
+
+/* One random word W serves one job of a pair of sibling children.  Its low half e is the
+ * even child's 16-bit mutation field, its high half o the odd child's; bit 0 decides which
+ * child inherits the first parent's gene.  A child mutates when its field is below the
+ * threshold; its new value is drawn with the fraction (other field + own field * M) mod 2^16
+ * in the top half of a 32-bit word, which is uniform because the other child's field is. */
+static uint32_t even_fraction(uint32_t W) { return W * 0x9E360001u; }            /* top half: o + e*0x9E36 */
+static uint32_t odd_fraction(uint32_t W) { return ((W << 16) | (W >> 16)) * 0x85EB0001u; } /* e + o*0x85EB */
 
 /* ------------------------------------------------------------------------- */
 /* Repair                                                                      */
@@ -382,15 +390,14 @@ int oracle_evolve(oracle_ctx* c, int32_t generations, uint64_t seed) {
             const int32_t* B = &c->pop[(size_t)pb * J];
             for (int32_t j = 0; j < J; ++j) {
                 const oracle_job* jb = &c->jobs[j];
-                uint32_t w0 = oracle_word(seed, gen, (uint32_t)slot0, (uint32_t)j, ORACLE_STREAM_MUT);
-                int flip = (int)(w0 & 1u); /* which child inherits the first parent's gene */
+                uint32_t W = oracle_word(seed, gen, (uint32_t)slot0, (uint32_t)j, ORACLE_STREAM_MUT);
+                int flip = (int)(W & 1u); /* which child inherits the first parent's gene */
                 int32_t child0 = flip ? B[j] : A[j];
                 int32_t child1 = flip ? A[j] : B[j];
-                if ((w0 >> 16) < thr) child0 = draw_gene(w0, jb->kmin, jb->kmax);
+                if ((W & 0xFFFFu) < thr) child0 = draw_gene(even_fraction(W), jb->kmin, jb->kmax);
                 c->next[(size_t)slot0 * J + j] = child0;
                 if (slot1 < N) {
-                    uint32_t w1 = oracle_word(seed, gen, (uint32_t)slot1, (uint32_t)j, ORACLE_STREAM_MUT);
-                    if ((w1 >> 16) < thr) child1 = draw_gene(w1, jb->kmin, jb->kmax);
+                    if ((W >> 16) < thr) child1 = draw_gene(odd_fraction(W), jb->kmin, jb->kmax);
                     c->next[(size_t)slot1 * J + j] = child1;
                 }
             }

@@ -51,9 +51,9 @@ __host__ __device__ __forceinline__ uint32_t counter3(uint32_t stream, uint64_t 
     return stream | ((uint32_t)(gen >> 32) << 4);
 }
 
-// Uniform value in [kmin, kmin + range) from bits 15..1 of a random word.
-__device__ __forceinline__ int32_t draw_gene(uint32_t w, int32_t kmin, int32_t range) {
-    return kmin + (int32_t)__umulhi((w << 16) & 0xFFFE0000u, (uint32_t)range);
+// Uniform value in [kmin, kmin + range): kmin + floor(frac * range / 2^32).
+__device__ __forceinline__ int32_t draw_gene(uint32_t frac, int32_t kmin, int32_t range) {
+    return kmin + (int32_t)__umulhi(frac, (uint32_t)range);
 }
 
 __host__ __device__ __forceinline__ int32_t slot_of(int32_t j) {
@@ -602,15 +602,34 @@ cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, 
 // child row; counter = (int4 index, row, generation, stream)), two child stores.  Warps past the
 // last pair copy the elites to rows 0..E-1.
 // ---------------------------------------------------------------------------------------------
-// The mutation decision compares the word's high half with thr16; as (w >> 16) < thr16 is
-// w < (thr16 << 16) for thr16 < 65536, kernels take thr32 = thr16 << 16 and ALWAYS for thr16 = 65536.
+// One random word W per job and pair of sibling children: low half = the even child's mutation
+// field, high half = the odd child's, bit 0 = which child inherits the first parent's gene.  A child
+// mutates when its field is below thr16, i.e. when the word with that field in its top half is below
+// thr32 = thr16 << 16 (ALWAYS stands for thr16 = 65536).  Its new value uses the fraction
+// (other field + own field * M) mod 2^16, placed in the top half by one multiply; the other child's
+// field is uniform and independent of this child's decision, so the fraction is uniform.
 template <bool ALWAYS>
-__device__ __forceinline__ int32_t mutate(uint32_t w, int32_t gene, int32_t kmin, int32_t range, uint32_t thr32) {
-    return (ALWAYS || w < thr32) ? draw_gene(w, kmin, range) : gene;
+__device__ __forceinline__ void sibling_gene(uint32_t W, int32_t a, int32_t b, int32_t kmin, int32_t range,
+                                             uint32_t thr32, bool has1, int32_t& c0, int32_t& c1) {
+    const bool flip = (W & 1u) != 0u;
+    const uint32_t R = __funnelshift_l(W, W, 16);  // halves swapped: even child's field on top
+    c0 = flip ? b : a;
+    c1 = flip ? a : b;
+    if (ALWAYS || R < thr32) c0 = draw_gene(W * 0x9E360001u, kmin, range);
+    if (has1 && (ALWAYS || W < thr32)) c1 = draw_gene(R * 0x85EB0001u, kmin, range);
 }
 
-template <int UNROLL, bool ALWAYS>
-__global__ void __launch_bounds__(256, 4)
+template <bool ALWAYS>
+__device__ __forceinline__ void sibling_int4(const uint4 W, const int4 a, const int4 b, const int4 kmin,
+                                             const int4 range, uint32_t thr32, bool has1, int4& c0, int4& c1) {
+    sibling_gene<ALWAYS>(W.x, a.x, b.x, kmin.x, range.x, thr32, has1, c0.x, c1.x);
+    sibling_gene<ALWAYS>(W.y, a.y, b.y, kmin.y, range.y, thr32, has1, c0.y, c1.y);
+    sibling_gene<ALWAYS>(W.z, a.z, b.z, kmin.z, range.z, thr32, has1, c0.z, c1.z);
+    sibling_gene<ALWAYS>(W.w, a.w, b.w, kmin.w, range.w, thr32, has1, c0.w, c1.w);
+}
+
+template <int UNROLL, bool ALWAYS, int MINB = 4>
+__global__ void __launch_bounds__(256, MINB)
 k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
          int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents, const int32_t* __restrict__ elites,
          Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr32) {
@@ -654,26 +673,11 @@ k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld,
                 if (v < nvec) {
                     const int4 kmin = kminv[v];
                     const int4 range = rangev[v];
-                    const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
-                    const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                    const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
                     int4 c0, c1;
-                    // bit 0 of the even child's word: which child inherits the first parent's gene
-                    c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
-                    c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
-                    c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
-                    c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
-                    c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
-                    c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
-                    c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
-                    c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
+                    sibling_int4<ALWAYS>(W, a[u], b[u], kmin, range, thr32, has1, c0, c1);
                     C0[v] = c0;
-                    if (has1) {
-                        c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
-                        c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
-                        c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
-                        c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
-                        C1[v] = c1;
-                    }
+                    if (has1) C1[v] = c1;
                 }
             }
         }
@@ -799,25 +803,13 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
                     if (v < nvec) {
                         const int4 kmin = sKmin[v];
                         const int4 range = sRange[v];
-                        const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
-                        const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                        const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
                         int4 c0, c1;
-                        c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
-                        c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
-                        c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
-                        c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
-                        c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
-                        c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
-                        c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
-                        c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
+                        sibling_int4<ALWAYS>(W, a[u], b[u], kmin, range, thr32, has1, c0, c1);
                         C0[v] = c0;
                         const int32_t base = (v >> 5) * 128 + lane;
                         score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
                         if (has1) {
-                            c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
-                            c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
-                            c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
-                            c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
                             C1[v] = c1;
                             score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
                         }
@@ -994,25 +986,13 @@ k_generation(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t
                     if (v < nvec) {
                         const int4 kmin = sKmin[v];
                         const int4 range = sRange[v];
-                        const uint4 w0 = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
-                        const uint4 w1 = philox((uint32_t)v, (uint32_t)slot1, gen_lo, c3, keys);
+                        const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
                         int4 c0, c1;
-                        c0.x = (w0.x & 1u) ? b[u].x : a[u].x;  c1.x = (w0.x & 1u) ? a[u].x : b[u].x;
-                        c0.y = (w0.y & 1u) ? b[u].y : a[u].y;  c1.y = (w0.y & 1u) ? a[u].y : b[u].y;
-                        c0.z = (w0.z & 1u) ? b[u].z : a[u].z;  c1.z = (w0.z & 1u) ? a[u].z : b[u].z;
-                        c0.w = (w0.w & 1u) ? b[u].w : a[u].w;  c1.w = (w0.w & 1u) ? a[u].w : b[u].w;
-                        c0.x = mutate<ALWAYS>(w0.x, c0.x, kmin.x, range.x, thr32);
-                        c0.y = mutate<ALWAYS>(w0.y, c0.y, kmin.y, range.y, thr32);
-                        c0.z = mutate<ALWAYS>(w0.z, c0.z, kmin.z, range.z, thr32);
-                        c0.w = mutate<ALWAYS>(w0.w, c0.w, kmin.w, range.w, thr32);
+                        sibling_int4<ALWAYS>(W, a[u], b[u], kmin, range, thr32, has1, c0, c1);
                         C0[v] = c0;
                         const int32_t base = (v >> 5) * 128 + lane;
                         score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
                         if (has1) {
-                            c1.x = mutate<ALWAYS>(w1.x, c1.x, kmin.x, range.x, thr32);
-                            c1.y = mutate<ALWAYS>(w1.y, c1.y, kmin.y, range.y, thr32);
-                            c1.z = mutate<ALWAYS>(w1.z, c1.z, kmin.z, range.z, thr32);
-                            c1.w = mutate<ALWAYS>(w1.w, c1.w, kmin.w, range.w, thr32);
                             C1[v] = c1;
                             score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
                         }

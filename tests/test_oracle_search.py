@@ -317,3 +317,31 @@ def test_bad_arguments_are_reported():
         oracle.Search(w.jobs, 16, 32, p_mut=1.5)
     with pytest.raises(oracle.OracleError):
         oracle.Search(w.jobs, 16, 32, tournament=0)
+
+
+def test_sibling_children_mutate_independently():
+    # p = 1: both children of a pair redraw every gene from one shared random word; the two new values
+    # must still be jointly uniform over all pairs of values, and rates per child must agree
+    w = inputs.custom(48, 10 ** 6, 1025, 1, seed=8, kmax=5)
+    row = np.zeros(48, dtype=np.int32)
+    s = _search(w, p_mut=1.0, elitism=1)
+    s.set_population(np.tile(row, (w.pop, 1)))
+    s.evolve(1, 21)
+    kids = s.get_population()[1:]
+    even, odd = kids[0::2].ravel(), kids[1::2].ravel()
+    joint = np.bincount(even * 6 + odd, minlength=36)
+    exp = even.size / 36
+    assert ((joint - exp) ** 2 / exp).sum() < 80  # 35 dof, p ~ 2e-5
+    for p in (0.1, 0.02):
+        s = _search(w, p_mut=p, elitism=1)
+        s.set_population(np.tile(row, (w.pop, 1)))
+        s.evolve(1, 22)
+        kids = s.get_population()[1:]
+        rate = oracle.thr16(p) / 65536 * (5 / 6)
+        for part in (kids[0::2], kids[1::2]):
+            n = part.size
+            assert abs(int((part != 0).sum()) - n * rate) < 5 * (n * rate * (1 - rate)) ** 0.5
+        # a hit on one child says nothing about its sibling at the same gene
+        both = int(((kids[0::2] != 0) & (kids[1::2] != 0)).sum())
+        n = kids[0::2].size
+        assert abs(both - n * rate * rate) < 6 * (n * rate * rate) ** 0.5 + 3
