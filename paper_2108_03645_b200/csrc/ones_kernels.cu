@@ -598,9 +598,9 @@ cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, 
 
 // ---------------------------------------------------------------------------------------------
 // Uniform crossover + uniform mutation, fused: one warp per pair of children.  Lane l handles the
-// int4 at genes 4l..4l+3 of every block of 128 genes: two parent loads, two Philox calls (one per
-// child row; counter = (int4 index, row, generation, stream)), two child stores.  Warps past the
-// last pair copy the elites to rows 0..E-1.
+// int4 at genes 4l..4l+3 of every block of 128 genes: two parent loads, one Philox call (counter =
+// (int4 index, even child's row, generation, stream); each of its four words serves one job of both
+// children), two child stores.  Warps past the last pair copy the elites to rows 0..E-1.
 // ---------------------------------------------------------------------------------------------
 // One random word W per job and pair of sibling children: low half = the even child's mutation
 // field, high half = the odd child's, bit 0 = which child inherits the first parent's gene.  A child
