@@ -47,6 +47,30 @@ def measured_peak():
 
 
 # ----------------------------------------------------------------------------------------------
+# multi-rank plumbing (replicas: no data-path collective, only the barrier and the timing reduction)
+# ----------------------------------------------------------------------------------------------
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank searches on its own random stream."""
+    return base_seed + rank
+
+
+def max_over_ranks(x: float, device="cpu") -> float:
+    """The slowest rank's figure (all-reduce MAX); identity when not distributed."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, units_per_rank_step: int, steps: int, ms: float) -> float:
+    """Units all ranks processed per second, over the slowest rank's time."""
+    return world * units_per_rank_step * steps / (ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------------------------
 # clocks during the timed region (read-only NVML queries)
 # ----------------------------------------------------------------------------------------------
 class ClockSampler:
@@ -230,7 +254,7 @@ def main():
 
     base = cpu_baseline(w) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
 
-    seed = w.seed + rank  # replicas: every rank searches on its own random stream
+    seed = rank_seed(w.seed, rank)
     s = binding.Search(w.jobs, w.capacity, w.pop, w.params)
     s.randomize(seed)
     s.evolve(warmup, seed)
@@ -260,10 +284,7 @@ def main():
     if not args.no_kernel_events:
         stage_ms, stage_n = s.stage_times()
         s.set_profiling(False)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, "cuda")
 
     # ---- end to end: every step uploads the job table and reads the best schedule back ----
     J, N, E = w.n_jobs, w.pop, w.params.elitism
@@ -288,10 +309,7 @@ def main():
             out = s.best(False)
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, "cuda")
     h2d = J * 48 + J * 4
     d2h = J * (4 + 4 + 8) + 24 + 4
 
@@ -320,7 +338,7 @@ def main():
 
     peak, peak_kind = measured_peak()
     line = {
-        "metric": METRIC, "value": world * N * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_rate(world, N, steps, ms), "unit": UNIT, "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "jobs": J, "population": N, "capacity": w.capacity,
