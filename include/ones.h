@@ -141,7 +141,8 @@ int ones_evolve(ones_ctx* ctx, int32_t generations, uint64_t seed);
  * holding the most GPUs (lowest index on ties) that can still shrink goes down one
  * exponent; when none can, running jobs wait (gene -1) in increasing index.
  * Host outputs, each nullable: h_genome int32[n_jobs], h_gpus_per_job int32[n_jobs],
- * h_rate_per_job double[n_jobs] (X_j of the returned genes), fitness, total_gpus,
+ * h_rate_per_job double[n_jobs] (X_j of the returned genes; with ONES_FLAG_SRUF the per-job score
+ * terms -weight_j * c_j / X_j instead), fitness, total_gpus,
  * index (row of the population).  With repair the fitness is that of the repaired
  * row.  Synchronises. */
 int ones_best(ones_ctx* ctx, int repair, int32_t* h_genome, int32_t* h_gpus_per_job,
@@ -193,6 +194,10 @@ int ones_select_top_noalloc(const double* d_fitness, int32_t n, int32_t e, int32
 
 /* Absolute generation counter, jobs and population of the handle. */
 int ones_generation(const ones_ctx* ctx, uint64_t* gen_abs);
+/* Resume a saved search: a handle created with the same jobs and parameters, given the saved
+ * population (ones_set_population) and the saved generation counter, continues exactly as the
+ * original would have (the random draws are keyed by the absolute generation). */
+int ones_set_generation(ones_ctx* ctx, uint64_t gen_abs);
 int ones_shape(const ones_ctx* ctx, int32_t* n_jobs, int32_t* pop, int32_t* capacity, int64_t* ld);
 
 /* Kernel launches issued through this handle so far. */

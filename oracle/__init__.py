@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.oracle_update_jobs.argtypes = [vp, vp, i32, vp, i32]
         L.oracle_last_parents.argtypes = [vp, vp, vp]
         L.oracle_generation.argtypes = [vp, vp]
+        L.oracle_set_generation.argtypes = [vp, u64]
         L.oracle_pairs.argtypes = [vp]
         L.oracle_pairs.restype = i32
         _lib = L
@@ -260,6 +261,9 @@ class Search:
         e = np.zeros(max(self.E, 1), dtype=np.int32)
         _check(lib().oracle_last_parents(self._h, _ptr(p), _ptr(e)), "last_parents")
         return p[:pairs], e[:self.E]
+
+    def set_generation(self, gen: int):
+        _check(lib().oracle_set_generation(self._h, gen), "set_generation")
 
     @property
     def generation(self) -> int:

@@ -486,4 +486,10 @@ int oracle_generation(const oracle_ctx* c, uint64_t* gen_abs) {
     return ORACLE_OK;
 }
 
+int oracle_set_generation(oracle_ctx* c, uint64_t gen_abs) {
+    if (!c) return ORACLE_ERR_NULL;
+    c->gen_abs = gen_abs;
+    return ORACLE_OK;
+}
+
 int32_t oracle_pairs(const oracle_ctx* c) { return c ? c->pairs : 0; }

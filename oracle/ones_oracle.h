@@ -93,6 +93,7 @@ int oracle_update_jobs(oracle_ctx*, const oracle_job* jobs, int32_t n_jobs, cons
                        int32_t capacity);
 int oracle_last_parents(oracle_ctx*, int32_t* parents /*[pairs][2]*/, int32_t* elites /*[E]*/);
 int oracle_generation(const oracle_ctx*, uint64_t* gen_abs);
+int oracle_set_generation(oracle_ctx*, uint64_t gen_abs); /* resume a saved search */
 int32_t oracle_pairs(const oracle_ctx*);
 
 #ifdef __cplusplus

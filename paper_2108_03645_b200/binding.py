@@ -59,6 +59,7 @@ _SIGNATURES = {
                                   C.c_void_p]),
     "ones_select_top_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "ones_generation": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ones_set_generation": (C.c_int, [C.c_void_p, C.c_uint64]),
     "ones_shape": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ones_kernel_launches": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ones_set_profiling": (C.c_int, [C.c_void_p, C.c_int]),
@@ -258,6 +259,9 @@ class Search:
         g = np.zeros((planes.value, self.J), dtype=np.int32)
         self._check(lib().ones_model_table(self._h, _np_ptr(X), _np_ptr(g), C.byref(planes)), "ones_model_table")
         return X, g
+
+    def set_generation(self, gen: int):
+        self._check(lib().ones_set_generation(self._h, gen), "ones_set_generation")
 
     @property
     def generation(self) -> int:

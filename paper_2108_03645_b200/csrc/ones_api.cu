@@ -546,6 +546,12 @@ int ones_generation(const ones_ctx* c, uint64_t* gen_abs) {
     return ONES_OK;
 }
 
+int ones_set_generation(ones_ctx* c, uint64_t gen_abs) {
+    if (!c) return ONES_ERR_NULL;
+    c->gen = gen_abs;
+    return ONES_OK;
+}
+
 int ones_shape(const ones_ctx* c, int32_t* n_jobs, int32_t* pop, int32_t* capacity, int64_t* ld) {
     if (!c) return ONES_ERR_NULL;
     if (n_jobs) *n_jobs = c->J;

@@ -24,6 +24,21 @@ import numpy as np
 from .inputs import JOB_DTYPE, Trace
 
 
+def sruf_weights(y_processed, alpha, beta, rng: np.random.Generator) -> np.ndarray:
+    """Per-job weights for the ONES_FLAG_SRUF score of one scheduling round.
+
+    Alg. 1 draws one progress sample rho_j ~ Be(alpha_j, beta_j) per job, shared by every
+    candidate of the round; Eq. 7 turns it into the remaining workload
+    Y_j = Y_processed,j * (1/rho_j - 1), which is the job's weight in the score
+    sum_j Y_j * c_j / X_j (Eq. 8).  alpha, beta >= 1 come from the caller's progress predictor.
+    """
+    y = np.asarray(y_processed, dtype=np.float64)
+    a = np.maximum(np.asarray(alpha, dtype=np.float64), 1.0)
+    b = np.maximum(np.asarray(beta, dtype=np.float64), 1.0)
+    rho = np.clip(rng.beta(a, b), 1e-12, 1.0)
+    return y * (1.0 / rho - 1.0)
+
+
 @dataclass
 class OnlineResult:
     jct: np.ndarray                 # seconds from arrival to completion, per job (nan if unfinished)

@@ -216,6 +216,22 @@ def test_split_runs_and_determinism(ones):
     assert (a.evaluate()[0] == b.evaluate()[0]).all()
 
 
+def test_checkpoint_and_resume(ones):
+    w = inputs.paper_scale()
+    a, o = _pair(ones, w)
+    a.randomize(3)
+    o.randomize(3)
+    a.evolve(4, 3)
+    o.evolve(9, 3)
+    saved, gen = a.get_population(), a.generation
+    b, _ = _pair(ones, w)  # a fresh handle picks the search up from the saved state
+    b.set_population(saved)
+    b.set_generation(gen)
+    b.evolve(5, 3)
+    assert b.generation == 9
+    _same_state(b, o)
+
+
 def test_set_get_population_roundtrip(ones):
     w = inputs.custom(30, 64, 50, 1, seed=1)
     g, o = _pair(ones, w)

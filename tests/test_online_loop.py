@@ -61,6 +61,64 @@ def test_online_loop_regrows_engine_when_job_set_outgrows_it():
     assert max(res.gpus_used) <= 8
 
 
+def test_sruf_weights_follow_eq7():
+    class Fixed:
+        def __init__(self, rho):
+            self.rho = np.asarray(rho, dtype=np.float64)
+
+        def beta(self, a, b):
+            return self.rho
+
+    y = np.array([1000.0, 4000.0, 50.0])
+    w = online.sruf_weights(y, [2, 3, 1], [2, 1, 5], Fixed([0.5, 0.25, 1.0]))
+    assert (w == np.array([1000.0, 12000.0, 0.0])).all()  # Y * (1/rho - 1)
+    rng = np.random.default_rng(0)
+    many = np.array([online.sruf_weights([1.0], [4.0], [2.0], rng)[0] for _ in range(4000)])
+    # E[1/rho - 1] for Be(4, 2) is (a + b - 1)/(a - 1) - 1 = 2/3
+    assert abs(many.mean() - 2 / 3) < 0.05
+
+
+def test_sruf_search_prefers_fewer_gpus_for_poorly_scaling_jobs():
+    # the paper's objective (Eq. 3): with a large per-doubling cost d, holding many GPUs is wasteful
+    w = inputs.custom(12, 10 ** 6, 128, 40, seed=3, kmax=5)
+    jobs = w.jobs.copy()
+    jobs["d"] = 0.5
+    jobs["weight"] = online.sruf_weights(np.full(12, 1e5), np.full(12, 3.0), np.full(12, 3.0),
+                                         np.random.default_rng(1))
+    s = oracle.Search(jobs, w.capacity, w.pop, flags=oracle.FLAG_SRUF)
+    s.randomize(0)
+    s.evolve(40, 0)
+    best = s.best()
+    # exhaustive per-job optimum of weight * g / X (the score separates over jobs without a capacity limit)
+    want = [min(range(6), key=lambda k: oracle.model(jobs, j, k)[1] / oracle.model(jobs, j, k)[0]) for j in range(12)]
+    assert list(best["genome"]) == want
+
+
+@pytest.mark.gpu
+def test_sruf_evolve_gpu_matches_oracle():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2108_03645_b200 import binding
+    w = inputs.paper_scale(4)
+    jobs = w.jobs.copy()
+    jobs["weight"] = online.sruf_weights(np.random.default_rng(2).uniform(1e3, 1e6, 100), np.full(100, 2.0),
+                                         np.full(100, 4.0), np.random.default_rng(3))
+    p = inputs.SearchParams(2, 4, 0.1, 1e3, binding.FLAG_SRUF)
+    g = binding.Search(jobs, w.capacity, w.pop, p)
+    o = oracle.Search(jobs, w.capacity, w.pop, flags=oracle.FLAG_SRUF)
+    g.randomize(1)
+    o.randomize(1)
+    g.evolve(20, 1)
+    o.evolve(20, 1)
+    assert (g.get_population() == o.get_population()).all()
+    Fg, Gg = g.evaluate()
+    Fo, Go = o.evaluate()
+    assert (Fg.cpu().numpy() == Fo).all() and (Gg.cpu().numpy() == Go).all()
+    bg, bo = g.best(True), o.best(True)
+    assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
+
+
 @pytest.mark.gpu
 def test_online_loop_gpu_matches_oracle():
     torch = pytest.importorskip("torch")

@@ -345,3 +345,15 @@ def test_sibling_children_mutate_independently():
         both = int(((kids[0::2] != 0) & (kids[1::2] != 0)).sum())
         n = kids[0::2].size
         assert abs(both - n * rate * rate) < 6 * (n * rate * rate) ** 0.5 + 3
+
+
+def test_checkpoint_and_resume():
+    w = inputs.paper_scale(0)
+    a = _search(w); a.randomize(3); a.evolve(9, 3)
+    b = _search(w); b.randomize(3); b.evolve(4, 3)
+    saved, gen = b.get_population(), b.generation
+    c = _search(w)  # a fresh handle picks the search up from the saved state
+    c.set_population(saved)
+    c.set_generation(gen)
+    c.evolve(5, 3)
+    assert (c.get_population() == a.get_population()).all() and c.generation == 9
