@@ -262,7 +262,7 @@ def main():
 
     # ---- device-resident timed region: K generations ----
     if not args.no_kernel_events:
-        s.set_profiling(True)
+        s.set_profiling(8 if steps >= 64 else 1)  # event pairs around every 8th generation's kernels
         s.stage_times()
     sampler = ClockSampler(local)
     if world > 1:

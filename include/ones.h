@@ -203,7 +203,8 @@ int ones_shape(const ones_ctx* ctx, int32_t* n_jobs, int32_t* pop, int32_t* capa
 /* Kernel launches issued through this handle so far. */
 int ones_kernel_launches(const ones_ctx* ctx, uint64_t* launches);
 
-/* Per-stage device time.  With profiling on, ones_evolve and ones_evaluate bracket
+/* Per-stage device time.  With profiling on (on = 1: every generation, on = n > 1: every n-th
+ * generation of a ones_evolve call), ones_evolve and ones_evaluate bracket
  * each kernel with CUDA events.  ones_stage_times synchronises and returns, for
  * stage s in {0 fitness (separate scoring passes), 1 select+elites, 2 evolve (crossover, mutation
  * and, unless ONES_FLAG_UNFUSED, the scoring of the children)}, the summed milliseconds

@@ -275,7 +275,8 @@ class Search:
         self._check(lib().ones_kernel_launches(self._h, C.byref(n)), "ones_kernel_launches")
         return int(n.value)
 
-    def set_profiling(self, on: bool):
+    def set_profiling(self, on):
+        """False/0 off, True/1 every generation, n > 1 every n-th generation."""
         self._check(lib().ones_set_profiling(self._h, int(on)), "ones_set_profiling")
 
     def stage_times(self):

@@ -73,6 +73,8 @@ Layout make_layout(int32_t jmax, int32_t pop) {
 
 struct Prof {
     bool on = false;
+    int every = 1;        // bracket every n-th generation
+    bool sample = true;   // this generation is bracketed
     std::vector<cudaEvent_t> ev;
     std::vector<int> stage;  // stage of event pair i
     size_t used = 0;         // events recorded since the last flush
@@ -195,7 +197,7 @@ int prof_flush(ones_ctx* c) {
 
 int prof_begin(ones_ctx* c, int stage) {
     Prof& p = c->prof;
-    if (!p.on) return ONES_OK;
+    if (!p.on || !p.sample) return ONES_OK;
     if (p.used + 2 > p.ev.size()) {
         int rc = prof_flush(c);
         if (rc) return rc;
@@ -207,7 +209,7 @@ int prof_begin(ones_ctx* c, int stage) {
 
 int prof_end(ones_ctx* c) {
     Prof& p = c->prof;
-    if (!p.on) return ONES_OK;
+    if (!p.on || !p.sample) return ONES_OK;
     CU(c, cudaEventRecord(p.ev[p.used + 1], c->stream));
     p.used += 2;
     return ONES_OK;
@@ -382,6 +384,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     if (generations < 0) return ONES_ERR_BAD_PARAM;
     if (generations == 0) return ONES_OK;
     int rc;
+    c->prof.sample = true;
     if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
     const RoundKeys keys = make_round_keys(seed);
     const int32_t E = c->prm.elitism;
@@ -397,6 +400,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
             if ((rc = prof_end(c)) != ONES_OK) return rc;
         }
         for (int32_t it = 0; it < generations; ++it) {
+            c->prof.sample = it % c->prof.every == 0;
             if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
             CU(c, launch_generation(shape, c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs,
                                     c->prm.tournament, c->Fbuf(c->fcur), c->Fbuf(c->fcur ^ 1), c->G(), c->parents(),
@@ -411,9 +415,11 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
             c->elites_valid = true;
             c->gen += 1;
         }
+        c->prof.sample = true;
         return ONES_OK;
     }
     for (int32_t it = 0; it < generations; ++it) {
+        c->prof.sample = it % c->prof.every == 0;
         if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
         CU(c, launch_select_stage(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), E,
                                   c->elites(0), c->ws + c->L.top, done, c->stream));
@@ -438,6 +444,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         c->gen += 1;
         if (!c->fused && (rc = run_fitness(c)) != ONES_OK) return rc;
     }
+    c->prof.sample = true;
     return ONES_OK;
 }
 
@@ -584,6 +591,8 @@ int ones_set_profiling(ones_ctx* c, int on) {
         if (rc) return rc;
     }
     c->prof.on = on != 0;
+    c->prof.every = on > 1 ? on : 1;
+    c->prof.sample = true;
     return ONES_OK;
 }
 
