@@ -17,6 +17,7 @@ _SRC = os.path.join(_HERE, "ones_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 FLAG_SRUF = 1
+FLAG_TRUNCATION = 4
 STREAM_INIT, STREAM_SEL_A, STREAM_SEL_B, STREAM_MUT = 0, 1, 2, 3
 
 JOB_DTYPE = np.dtype(
@@ -69,6 +70,7 @@ def lib() -> C.CDLL:
         L.oracle_tournament.argtypes = [vp, i32, i32, u64, u64, u32, u32]
         L.oracle_tournament.restype = i32
         L.oracle_top.argtypes = [vp, i32, i32, vp]
+        L.oracle_keep_best.argtypes = [vp, i32, i32, vp]
         L.oracle_thr16.argtypes = [dbl]
         L.oracle_thr16.restype = u32
         L.oracle_create.argtypes = [vp, vp, i32, i32, i32, vp]
@@ -170,6 +172,13 @@ def top(F, e: int) -> np.ndarray:
     idx = np.zeros(max(e, 1), dtype=np.int32)
     _check(lib().oracle_top(_ptr(f), f.shape[0], e, _ptr(idx)), "top")
     return idx[:e]
+
+
+def keep_best(F, k: int) -> np.ndarray:
+    f = np.ascontiguousarray(F, dtype=np.float64)
+    idx = np.zeros(max(k, 1), dtype=np.int32)
+    _check(lib().oracle_keep_best(_ptr(f), f.shape[0], k, _ptr(idx)), "keep_best")
+    return idx[:k]
 
 
 def thr16(p: float) -> int:

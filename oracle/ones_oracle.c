@@ -285,7 +285,7 @@ int oracle_create(oracle_ctx** out, const oracle_job* jobs, int32_t n_jobs, int3
     oracle_ctx* c = (oracle_ctx*)calloc(1, sizeof *c);
     if (!c) return ORACLE_ERR_NOMEM;
     c->J = n_jobs; c->cap = capacity; c->N = pop; c->prm = p;
-    c->pairs = (pop - p.elitism + 1) / 2;
+    c->pairs = (p.flags & ORACLE_FLAG_TRUNCATION) ? pop : (pop - p.elitism + 1) / 2;
     size_t cells = (size_t)pop * (size_t)n_jobs;
     c->jobs = (oracle_job*)malloc(sizeof(oracle_job) * (size_t)n_jobs);
     c->pop = (int32_t*)malloc(sizeof(int32_t) * cells);
@@ -367,9 +367,114 @@ int oracle_evaluate(oracle_ctx* c, const int32_t* genomes, int64_t ld, int32_t n
     return ORACLE_OK;
 }
 
+/* Indices of the k best of n scores (score descending, index ascending), returned in ascending index
+ * order: truncation selection that keeps the survivors in the order they had. */
+int oracle_keep_best(const double* F, int32_t n, int32_t k, int32_t* kept) {
+    if (!F || !kept) return ORACLE_ERR_NULL;
+    if (k < 0 || k > n) return ORACLE_ERR_BAD_PARAM;
+    int32_t* order = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    char* keep = (char*)calloc((size_t)(n > 0 ? n : 1), 1);
+    if (!order || !keep) { free(order); free(keep); return ORACLE_ERR_NOMEM; }
+    for (int32_t i = 0; i < n; ++i) order[i] = i;
+    /* heap sort under better(): the heap's root is the candidate that ranks last */
+    for (int32_t i = 1; i < n; ++i) {
+        int32_t c = i;
+        while (c > 0) {
+            int32_t p = (c - 1) / 2;
+            if (!better(F, order[p], order[c])) break;
+            int32_t t = order[p]; order[p] = order[c]; order[c] = t;
+            c = p;
+        }
+    }
+    for (int32_t end = n; end > 1; --end) {
+        int32_t t = order[0]; order[0] = order[end - 1]; order[end - 1] = t;
+        int32_t c = 0;
+        for (;;) {
+            int32_t l = 2 * c + 1, r = l + 1, w = c;
+            if (l < end - 1 && better(F, order[w], order[l])) w = l;
+            if (r < end - 1 && better(F, order[w], order[r])) w = r;
+            if (w == c) break;
+            t = order[c]; order[c] = order[w]; order[w] = t;
+            c = w;
+        }
+    }
+    for (int32_t r = 0; r < k; ++r) keep[order[r]] = 1; /* order[] is best first */
+    int32_t at = 0;
+    for (int32_t i = 0; i < n; ++i)
+        if (keep[i]) kept[at++] = i;
+    free(order);
+    free(keep);
+    return ORACLE_OK;
+}
+
+/* One generation of the paper's own scheme (Section 3.2.2 "Evolution" and "Selection"): from the K
+ * candidates of G_i derive G'_i = the K candidates themselves, 2K children of K uniformly drawn
+ * parent pairs (uniform crossover, no mutation) and K mutants of K uniformly drawn candidates
+ * (each job redrawn with rate theta); score all 4K and keep the best K (score descending, position
+ * in G'_i ascending), in the order they had in G'_i. */
+static int truncation_generation(oracle_ctx* c, uint64_t seed) {
+    const int32_t K = c->N, J = c->J;
+    const uint64_t gen = c->gen_abs;
+    const uint32_t thr = oracle_thr16(c->prm.p_mut);
+    const size_t rows = (size_t)4 * K;
+    int32_t* pool = (int32_t*)malloc(sizeof(int32_t) * rows * (size_t)J);
+    double* F = (double*)malloc(sizeof(double) * rows);
+    int32_t* G = (int32_t*)malloc(sizeof(int32_t) * rows);
+    char* keep = NULL;
+    if (!pool || !F || !G) { free(pool); free(F); free(G); return ORACLE_ERR_NOMEM; }
+    memcpy(pool, c->pop, sizeof(int32_t) * (size_t)K * J);
+    for (int32_t q = 0; q < K; ++q) { /* crossover children at rows K + 2q, K + 2q + 1 */
+        int32_t pa = oracle_tournament(c->F, K, 1, seed, gen, (uint32_t)q, ORACLE_STREAM_SEL_A);
+        int32_t pb = oracle_tournament(c->F, K, 1, seed, gen, (uint32_t)q, ORACLE_STREAM_SEL_B);
+        c->parents[2 * q] = pa;
+        c->parents[2 * q + 1] = pb;
+        for (int32_t j = 0; j < J; ++j) {
+            uint32_t W = oracle_word(seed, gen, (uint32_t)(2 * q), (uint32_t)j, ORACLE_STREAM_MUT);
+            int flip = (int)(W & 1u);
+            int32_t ga = c->pop[(size_t)pa * J + j], gb = c->pop[(size_t)pb * J + j];
+            pool[((size_t)K + 2 * q) * J + j] = flip ? gb : ga;
+            pool[((size_t)K + 2 * q + 1) * J + j] = flip ? ga : gb;
+        }
+    }
+    for (int32_t m = 0; m < K; ++m) { /* mutants at rows 3K + m */
+        int32_t from = oracle_tournament(c->F, K, 1, seed, gen, (uint32_t)m, ORACLE_STREAM_PICK);
+        for (int32_t j = 0; j < J; ++j) {
+            uint32_t W = oracle_word(seed, gen, (uint32_t)m, (uint32_t)j, ORACLE_STREAM_MUTANT);
+            int32_t g = c->pop[(size_t)from * J + j];
+            if ((W & 0xFFFFu) < thr) g = draw_gene(even_fraction(W), c->jobs[j].kmin, c->jobs[j].kmax);
+            pool[((size_t)3 * K + m) * J + j] = g;
+        }
+    }
+    for (size_t i = 0; i < rows; ++i)
+        oracle_fitness(c->jobs, J, c->cap, c->prm.penalty, c->prm.flags, &pool[i * J], &F[i], &G[i]);
+    int32_t* order = (int32_t*)malloc(sizeof(int32_t) * (size_t)K);
+    if (!order) { free(pool); free(F); free(G); free(keep); return ORACLE_ERR_NOMEM; }
+    int rc = oracle_keep_best(F, (int32_t)rows, K, order);
+    if (rc) { free(order); free(pool); free(F); free(G); free(keep); return rc; }
+    for (int32_t at = 0; at < K; ++at) {
+        const size_t i = (size_t)order[at];
+        memcpy(&c->next[(size_t)at * J], &pool[i * J], sizeof(int32_t) * (size_t)J);
+        c->F[at] = F[i];
+        c->G[at] = G[i];
+    }
+    int32_t* tmp = c->pop; c->pop = c->next; c->next = tmp;
+    c->gen_abs = gen + 1;
+    c->f_valid = 1;
+    free(order); free(pool); free(F); free(G); free(keep);
+    return ORACLE_OK;
+}
+
 int oracle_evolve(oracle_ctx* c, int32_t generations, uint64_t seed) {
     if (!c) return ORACLE_ERR_NULL;
     if (generations < 0) return ORACLE_ERR_BAD_PARAM;
+    if (c->prm.flags & ORACLE_FLAG_TRUNCATION) {
+        if (!c->f_valid) score_population(c);
+        for (int32_t it = 0; it < generations; ++it) {
+            int rc = truncation_generation(c, seed);
+            if (rc) return rc;
+        }
+        return ORACLE_OK;
+    }
     const int32_t N = c->N, J = c->J, E = c->prm.elitism, T = c->prm.tournament;
     const uint32_t thr = oracle_thr16(c->prm.p_mut);
     if (!c->f_valid) score_population(c);

@@ -39,6 +39,8 @@ typedef struct {
 } oracle_params;
 
 #define ORACLE_FLAG_SRUF 1u /* score = -(sum_j weight_j * c_j / X_j): Alg. 1 score, negated */
+/* bit 2 (value 2) only selects a launch sequence in the CUDA library; it means nothing here */
+#define ORACLE_FLAG_TRUNCATION 4u /* the paper's selection: best K of K originals + 2K crossover children + K mutants */
 
 enum {
     ORACLE_OK = 0,
@@ -49,7 +51,8 @@ enum {
     ORACLE_ERR_INFEASIBLE = -5
 };
 
-enum { ORACLE_STREAM_INIT = 0, ORACLE_STREAM_SEL_A = 1, ORACLE_STREAM_SEL_B = 2, ORACLE_STREAM_MUT = 3 };
+enum { ORACLE_STREAM_INIT = 0, ORACLE_STREAM_SEL_A = 1, ORACLE_STREAM_SEL_B = 2, ORACLE_STREAM_MUT = 3,
+       ORACLE_STREAM_PICK = 4, ORACLE_STREAM_MUTANT = 5 };
 
 typedef struct oracle_ctx oracle_ctx;
 
@@ -73,6 +76,8 @@ int32_t oracle_tournament(const double* F, int32_t n, int32_t tournament, uint64
                           uint64_t gen_abs, uint32_t q, uint32_t stream);
 /* indices of the e best candidates (F descending, index ascending) */
 int oracle_top(const double* F, int32_t n, int32_t e, int32_t* idx);
+/* the k best of n scores, as ascending indices (truncation selection, order preserved) */
+int oracle_keep_best(const double* F, int32_t n, int32_t k, int32_t* kept);
 /* mutation threshold on the 16-bit decision field for probability p */
 uint32_t oracle_thr16(double p_mut);
 
