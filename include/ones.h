@@ -67,6 +67,16 @@ typedef struct {
  * crossover/mutation and the fitness kernels on their own). */
 #define ONES_FLAG_UNFUSED 2u
 
+/* ones_evolve runs the paper's own scheme (Section 3.2.2 "Evolution", "Selection") instead of
+ * tournament + elitism: per generation the pool G' = the pop current candidates (rows 0..pop-1),
+ * 2*pop children of pop uniformly drawn parent pairs (uniform crossover, no mutation; rows
+ * pop..3*pop-1) and pop mutants of pop uniformly drawn candidates (each job redrawn with rate p_mut;
+ * rows 3*pop..4*pop-1) is scored and the best pop of the 4*pop (score descending, row ascending)
+ * survive, in the order of their rows.  elitism and tournament are ignored.  The workspace must be
+ * sized with ones_workspace_bytes_flags (the pool takes 4x the rows).  ones_last_parents then
+ * returns [pop][2] parent rows. */
+#define ONES_FLAG_TRUNCATION 4u
+
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
 #define ONES_MAX_ELITES 256   /* elitism <= 256 */
 
@@ -86,6 +96,8 @@ enum {
  * pop candidates (two population buffers, fitness, parents, model tables,
  * scratch).  Returns 0 when an argument is out of range. */
 size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop);
+/* The same for a handle created with `flags` (ONES_FLAG_TRUNCATION needs room for its candidate pool). */
+size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flags);
 
 /* Create a search over `n_jobs` jobs on a cluster of `capacity` GPUs with a
  * population of `pop` candidates (Section 3.2.2 "Initialization": the population

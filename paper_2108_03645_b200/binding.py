@@ -18,6 +18,7 @@ from .inputs import JOB_DTYPE, SearchParams
 
 FLAG_SRUF = 1
 FLAG_UNFUSED = 2
+FLAG_TRUNCATION = 4
 MAX_ELITES = 256
 
 ERRORS = {0: "ONES_OK", -1: "ONES_ERR_NULL", -2: "ONES_ERR_BAD_JOB", -3: "ONES_ERR_BAD_PARAM",
@@ -41,6 +42,7 @@ _lib = None
 
 _SIGNATURES = {
     "ones_workspace_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
+    "ones_workspace_bytes_flags": (C.c_size_t, [C.c_int32, C.c_int32, C.c_uint32]),
     "ones_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                               C.c_size_t, C.c_void_p]),
     "ones_destroy": (C.c_int, [C.c_void_p]),
@@ -97,8 +99,8 @@ def _stream_ptr():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def workspace_bytes(n_jobs_max: int, pop: int) -> int:
-    return int(lib().ones_workspace_bytes(n_jobs_max, pop))
+def workspace_bytes(n_jobs_max: int, pop: int, flags: int = 0) -> int:
+    return int(lib().ones_workspace_bytes_flags(n_jobs_max, pop, flags))
 
 
 def select_top(fitness: torch.Tensor, e: int) -> torch.Tensor:
@@ -146,7 +148,7 @@ class Search:
         self.J = int(jobs.shape[0])
         self.capacity = int(capacity)
         nmax = max(self.J, int(n_jobs_max or 0))
-        nbytes = workspace_bytes(nmax, pop)
+        nbytes = workspace_bytes(nmax, pop, p.flags)
         if nbytes == 0:
             raise OnesError(-3, "ones_workspace_bytes")
         self.device = torch.device("cuda", torch.cuda.current_device())
@@ -246,7 +248,7 @@ class Search:
 
     # -- inspection ---------------------------------------------------------------
     def last_parents(self):
-        pairs = (self.N - self.params.elitism + 1) // 2
+        pairs = self.N if self.params.flags & FLAG_TRUNCATION else (self.N - self.params.elitism + 1) // 2
         p = np.zeros((max(pairs, 1), 2), dtype=np.int32)
         e = np.zeros(max(self.params.elitism, 1), dtype=np.int32)
         self._check(lib().ones_last_parents(self._h, _np_ptr(p), _np_ptr(e)), "ones_last_parents")

@@ -26,11 +26,11 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
+    size_t pop0, pop1, F, F1, G, G1, trunc, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
         out_gpus, out_rate, out_rec, exp_X, exp_G, status, total;
 };
 
-Layout make_layout(int32_t jmax, int32_t pop) {
+Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
     Layout L;
     size_t at = 0;
     auto take = [&](size_t bytes) {
@@ -39,12 +39,16 @@ Layout make_layout(int32_t jmax, int32_t pop) {
         return here;
     };
     const size_t ldm = (size_t)ld_of(jmax), jp = (size_t)jpad_of(jmax);
-    const size_t pairs = ((size_t)pop + 1) / 2;
-    L.pop0 = take((size_t)pop * ldm * 4);
-    L.pop1 = take((size_t)pop * ldm * 4);
-    L.F = take((size_t)pop * 8);
-    L.F1 = take((size_t)pop * 8);
-    L.G = take((size_t)pop * 4);
+    // the truncation scheme keeps a pool of 4 * pop rows (originals, crossover children, mutants)
+    const size_t rows = trunc ? 4 * (size_t)pop : (size_t)pop;
+    const size_t pairs = trunc ? 3 * (size_t)pop : ((size_t)pop + 1) / 2;  // 2K parents + K mutant sources
+    L.pop0 = take(rows * ldm * 4);
+    L.pop1 = take(rows * ldm * 4);
+    L.F = take(rows * 8);
+    L.F1 = take(rows * 8);
+    L.G = take(rows * 4);
+    L.G1 = take(rows * 4);
+    L.trunc = take(trunc ? trunc_scratch_bytes(pop) : 16);
     L.parents = take(pairs * 2 * 4);
     L.elites = take((size_t)ONES_MAX_ELITES * 4);
     L.elites1 = take((size_t)ONES_MAX_ELITES * 4);
@@ -95,6 +99,8 @@ struct ones_ctx {
     Layout L{};
     int cur = 0;            // population buffer in force
     int fcur = 0;           // score buffer in force
+    int gcur = 0;           // GPU-count buffer in force (only the truncation scheme alternates it)
+    bool trunc = false;     // ONES_FLAG_TRUNCATION
     int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
     int elast = 0;          // elites buffer used by the last generation
     bool elites_valid = false;
@@ -110,7 +116,8 @@ struct ones_ctx {
     int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
     double* Fbuf(int which) { return reinterpret_cast<double*>(ws + (which ? L.F1 : L.F)); }
     double* F() { return Fbuf(fcur); }
-    int32_t* G() { return reinterpret_cast<int32_t*>(ws + L.G); }
+    int32_t* Gbuf(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.G1 : L.G)); }
+    int32_t* G() { return Gbuf(gcur); }
     int32_t* parents() { return reinterpret_cast<int32_t*>(ws + L.parents); }
     int32_t* elites(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.elites1 : L.elites)); }
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
@@ -250,9 +257,13 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 extern "C" {
 
-size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop) {
+size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop) { return ones_workspace_bytes_flags(n_jobs_max, pop, 0u); }
+
+size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flags) {
     if (n_jobs_max <= 0 || n_jobs_max > kJobsLimit || pop <= 0 || pop > kPopLimit) return 0;
-    return make_layout(n_jobs_max, pop).total;
+    const bool trunc = (flags & ONES_FLAG_TRUNCATION) != 0;
+    if (trunc && pop > kPopLimit / 4) return 0;
+    return make_layout(n_jobs_max, pop, trunc).total;
 }
 
 int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t capacity, int32_t pop,
@@ -268,12 +279,14 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     rc = check_params(p, pop);
     if (rc) return rc;
     if ((reinterpret_cast<uintptr_t>(d_workspace) & (kAlign - 1)) != 0) return ONES_ERR_ALIGN;
-    if (workspace_bytes < make_layout(n_jobs, pop).total) return ONES_ERR_WORKSPACE;
+    const bool trunc = (p.flags & ONES_FLAG_TRUNCATION) != 0;
+    if (trunc && pop > kPopLimit / 4) return ONES_ERR_BAD_PARAM;
+    if (workspace_bytes < make_layout(n_jobs, pop, trunc).total) return ONES_ERR_WORKSPACE;
     // the largest job count this workspace can hold
     int32_t lo = n_jobs, hi = kJobsLimit;
     while (lo < hi) {
         const int32_t mid = lo + (hi - lo + 1) / 2;
-        if (make_layout(mid, pop).total <= workspace_bytes) lo = mid;
+        if (make_layout(mid, pop, trunc).total <= workspace_bytes) lo = mid;
         else hi = mid - 1;
     }
     ones_ctx* c = new (std::nothrow) ones_ctx();
@@ -285,10 +298,11 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     c->cap = capacity;
     c->prm = p;
     c->thr16 = threshold16(p.p_mut);
-    c->pairs = (pop - p.elitism + 1) / 2;
+    c->trunc = trunc;
+    c->pairs = trunc ? pop : (pop - p.elitism + 1) / 2;
     c->ld = ld_of(n_jobs);
     c->ws = reinterpret_cast<char*>(d_workspace);
-    c->L = make_layout(c->Jmax, pop);
+    c->L = make_layout(c->Jmax, pop, trunc);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) {
         delete c;
@@ -387,6 +401,27 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     c->prof.sample = true;
     if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
     const RoundKeys keys = make_round_keys(seed);
+    if (c->trunc) {
+        // the paper's scheme: pool of 4K rows, best K survive (elitism and tournament size do not apply)
+        for (int32_t it = 0; it < generations; ++it) {
+            c->prof.sample = it % c->prof.every == 0;
+            if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
+            int nl = 0;
+            CU(c, launch_truncation_generation(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, c->Fbuf(c->fcur),
+                                               c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1), c->Gbuf(c->gcur ^ 1),
+                                               c->parents(), c->tab, keys, c->gen, c->thr16, c->cap, c->prm.penalty,
+                                               c->ws + c->L.trunc, c->stream, &nl));
+            c->launches += (uint64_t)nl;
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+            c->cur ^= 1;
+            c->fcur ^= 1;
+            c->gcur ^= 1;
+            c->gen += 1;
+        }
+        c->prof.sample = true;
+        c->elites_valid = false;
+        return ONES_OK;
+    }
     const int32_t E = c->prm.elitism;
     unsigned int* done = reinterpret_cast<unsigned int*>(c->status() + 1);
     const GenerationShape shape = c->fused ? generation_shape(c->tab, c->pairs, E) : GenerationShape{0, 0, 0, 0};
@@ -510,7 +545,7 @@ int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
     if (!c) return ONES_ERR_NULL;
     if (h_parents && c->pairs > 0)
         CU(c, cudaMemcpyAsync(h_parents, c->parents(), (size_t)c->pairs * 8, cudaMemcpyDeviceToHost, c->stream));
-    if (h_elites && c->prm.elitism > 0)
+    if (h_elites && c->prm.elitism > 0 && !c->trunc)
         CU(c, cudaMemcpyAsync(h_elites, c->elites(c->elast), (size_t)c->prm.elitism * 4, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
     return ONES_OK;

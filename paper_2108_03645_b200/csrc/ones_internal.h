@@ -11,7 +11,9 @@ constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
 constexpr int kMaxSmemPerBlock = 232448;  // 227 KiB opt-in dynamic shared memory per CTA
 constexpr int kTopBlocksMax = 128;        // partial top-k blocks
 
-enum Stream : uint32_t { STREAM_INIT = 0, STREAM_SEL_A = 1, STREAM_SEL_B = 2, STREAM_MUT = 3 };
+enum Stream : uint32_t {
+    STREAM_INIT = 0, STREAM_SEL_A = 1, STREAM_SEL_B = 2, STREAM_MUT = 3, STREAM_PICK = 4, STREAM_MUTANT = 5
+};
 
 // Philox4x32-10 round keys for one 64-bit seed: key word pair of round r is
 // (k[2r], k[2r+1]).  Passed to kernels by value so they sit in the constant bank.
@@ -81,6 +83,12 @@ cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t
                               double* F_new, int32_t* G, int32_t* parents, const int32_t* elites,
                               int32_t* elites_next, Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16,
                               int32_t capacity, double penalty, void* scratch, unsigned int* done, cudaStream_t s);
+// The paper's truncation selection over a pool of 4K rows (ONES_FLAG_TRUNCATION)
+size_t trunc_scratch_bytes(int32_t k);
+cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, int32_t n_jobs,
+                                         double* F, int32_t* G, double* F_next, int32_t* G_next, int32_t* draws,
+                                         Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
+                                         double penalty, void* scratch, cudaStream_t s, int* launches);
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,

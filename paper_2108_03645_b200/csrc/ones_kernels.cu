@@ -1138,6 +1138,258 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
 }
 
 // ---------------------------------------------------------------------------------------------
+// The paper's own selection (Section 3.2.2 "Evolution" / "Selection"): the candidate pool G'_i holds
+// the K current candidates (rows 0..K-1), 2K crossover children of K uniformly drawn parent pairs
+// (rows K..3K-1, no mutation) and K mutants of K uniformly drawn candidates (rows 3K..4K-1); the best K
+// of the 4K (score descending, row ascending) survive in the order of their rows.
+// ---------------------------------------------------------------------------------------------
+// draws[0..2K): parents of pair q at 2q, 2q+1; draws[2K..3K): source row of mutant m
+__global__ void k_trunc_draws(int32_t k, RoundKeys keys, uint32_t gen_lo, uint32_t c3a, uint32_t c3b, uint32_t c3pick,
+                              int32_t* __restrict__ draws) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 3 * k) return;
+    uint32_t row, c3;
+    if (i < 2 * k) {
+        row = (uint32_t)(i >> 1);
+        c3 = (i & 1) ? c3b : c3a;
+    } else {
+        row = (uint32_t)(i - 2 * k);
+        c3 = c3pick;
+    }
+    const uint4 w = philox(0u, row, gen_lo, c3, keys);
+    draws[i] = (int32_t)__umulhi(w.x, (uint32_t)k);
+}
+
+// one warp per work item: items 0..K-1 are crossover pairs, K..2K-1 mutants
+template <bool ALWAYS>
+__global__ void __launch_bounds__(256, 4)
+k_trunc_children(int32_t* __restrict__ pool, int64_t ld, int32_t k, const int32_t* __restrict__ draws, Tables t,
+                 RoundKeys keys, uint32_t gen_lo, uint32_t c3cross, uint32_t c3mutant, uint32_t thr32) {
+    const int lane = threadIdx.x & 31;
+    const int64_t item = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (item >= 2 * (int64_t)k) return;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const int4* __restrict__ kminv = reinterpret_cast<const int4*>(t.kmin);
+    const int4* __restrict__ rangev = reinterpret_cast<const int4*>(t.range);
+    if (item < k) {
+        const int32_t q = (int32_t)item;
+        const int4* A = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q] * ld);
+        const int4* B = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q + 1] * ld);
+        int4* C0 = reinterpret_cast<int4*>(pool + ((int64_t)k + 2 * q) * ld);
+        int4* C1 = reinterpret_cast<int4*>(pool + ((int64_t)k + 2 * q + 1) * ld);
+        for (int32_t v = lane; v < nvec; v += 32) {
+            const uint4 W = philox((uint32_t)v, (uint32_t)(2 * q), gen_lo, c3cross, keys);
+            int4 c0, c1;
+            sibling_int4<false>(W, A[v], B[v], kminv[v], rangev[v], 0u, true, c0, c1);  // threshold 0: no mutation
+            C0[v] = c0;
+            C1[v] = c1;
+        }
+    } else {
+        const int32_t m = (int32_t)(item - k);
+        const int4* S = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * k + m] * ld);
+        int4* C = reinterpret_cast<int4*>(pool + ((int64_t)3 * k + m) * ld);
+        for (int32_t v = lane; v < nvec; v += 32) {
+            const uint4 W = philox((uint32_t)v, (uint32_t)m, gen_lo, c3mutant, keys);
+            const int4 g = S[v];
+            int4 c0, c1;
+            sibling_int4<ALWAYS>(W, g, g, kminv[v], rangev[v], thr32, false, c0, c1);  // the even child's draws
+            C[v] = c0;
+        }
+    }
+}
+
+struct TruncPick {  // result of the selection threshold search
+    unsigned long long key;  // key of the K-th best candidate
+    int32_t quota;           // how many candidates with exactly that key survive (lowest rows first)
+    int32_t pad;
+};
+
+// K-th largest of n score keys by an 8-pass radix search (one CTA)
+__global__ void __launch_bounds__(1024) k_trunc_threshold(const double* __restrict__ F, int32_t n, int32_t k,
+                                                          TruncPick* __restrict__ out) {
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ int32_t s_remaining;
+    if (threadIdx.x == 0) {
+        s_prefix = 0ull;
+        s_remaining = k;
+    }
+    unsigned long long mask = 0ull;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int shift = 56 - 8 * pass;
+        for (int d = threadIdx.x; d < 256; d += blockDim.x) hist[d] = 0u;
+        __syncthreads();
+        const unsigned long long prefix = s_prefix;
+        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
+            const unsigned long long key = score_key(F[i]);
+            if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int32_t above = 0, d = 255;
+            for (; d > 0; --d) {
+                if (above + (int32_t)hist[d] >= s_remaining) break;
+                above += (int32_t)hist[d];
+            }
+            s_remaining -= above;
+            s_prefix = prefix | ((unsigned long long)d << shift);
+        }
+        mask |= 0xFFull << shift;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        out->key = s_prefix;
+        out->quota = s_remaining;
+        out->pad = 0;
+    }
+}
+
+// per block of `per_block` consecutive rows: how many rank above the threshold, how many tie with it
+__global__ void __launch_bounds__(256) k_trunc_count(const double* __restrict__ F, int32_t n, int32_t per_block,
+                                                     const TruncPick* __restrict__ pick, int32_t* __restrict__ bsum) {
+    __shared__ int32_t s_gt, s_eq;
+    if (threadIdx.x == 0) s_gt = s_eq = 0;
+    __syncthreads();
+    const unsigned long long T = pick->key;
+    const int32_t lo = blockIdx.x * per_block, hi = min(n, lo + per_block);
+    int32_t gt = 0, eq = 0;
+    for (int32_t i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+        const unsigned long long key = score_key(F[i]);
+        gt += key > T;
+        eq += key == T;
+    }
+    atomicAdd(&s_gt, gt);
+    atomicAdd(&s_eq, eq);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bsum[2 * blockIdx.x] = s_gt;
+        bsum[2 * blockIdx.x + 1] = s_eq;
+    }
+}
+
+// exclusive scan of the per-block counts (one CTA, blocks <= 1024)
+__global__ void __launch_bounds__(1024) k_trunc_scan(int32_t* __restrict__ bsum, int32_t blocks) {
+    __shared__ int32_t sg[1024], se[1024];
+    const int t = threadIdx.x;
+    sg[t] = t < blocks ? bsum[2 * t] : 0;
+    se[t] = t < blocks ? bsum[2 * t + 1] : 0;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        const int32_t a = t >= off ? sg[t - off] : 0, b = t >= off ? se[t - off] : 0;
+        __syncthreads();
+        sg[t] += a;
+        se[t] += b;
+        __syncthreads();
+    }
+    if (t < blocks) {
+        bsum[2 * t] = sg[t] - (t < blocks ? bsum[2 * t] : 0);      // exclusive
+        bsum[2 * t + 1] = se[t] - (t < blocks ? bsum[2 * t + 1] : 0);
+    }
+}
+
+// kept[p] = row of the p-th survivor (rows ascending): p = (#above before row) + min(#ties before row, quota)
+__global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ F, int32_t n, int32_t per_block,
+                                                     const TruncPick* __restrict__ pick,
+                                                     const int32_t* __restrict__ bsum, int32_t* __restrict__ kept) {
+    __shared__ int32_t tg[256], te[256];
+    const unsigned long long T = pick->key;
+    const int32_t quota = pick->quota;
+    const int32_t lo = blockIdx.x * per_block, hi = min(n, lo + per_block);
+    const int32_t per_thread = per_block / 256;  // per_block is a multiple of 256
+    const int32_t mylo = lo + threadIdx.x * per_thread, myhi = min(hi, mylo + per_thread);
+    int32_t gt = 0, eq = 0;
+    for (int32_t i = mylo; i < myhi; ++i) {
+        const unsigned long long key = score_key(F[i]);
+        gt += key > T;
+        eq += key == T;
+    }
+    tg[threadIdx.x] = gt;
+    te[threadIdx.x] = eq;
+    __syncthreads();
+    for (int off = 1; off < 256; off <<= 1) {
+        const int32_t a = (int)threadIdx.x >= off ? tg[threadIdx.x - off] : 0;
+        const int32_t b = (int)threadIdx.x >= off ? te[threadIdx.x - off] : 0;
+        __syncthreads();
+        tg[threadIdx.x] += a;
+        te[threadIdx.x] += b;
+        __syncthreads();
+    }
+    int32_t g_before = bsum[2 * blockIdx.x] + tg[threadIdx.x] - gt;
+    int32_t e_before = bsum[2 * blockIdx.x + 1] + te[threadIdx.x] - eq;
+    for (int32_t i = mylo; i < myhi; ++i) {
+        const unsigned long long key = score_key(F[i]);
+        if (key > T) {
+            kept[g_before + min(e_before, quota)] = i;
+            ++g_before;
+        } else if (key == T) {
+            if (e_before < quota) kept[g_before + e_before] = i;
+            ++e_before;
+        }
+    }
+}
+
+// survivors move to rows 0..K-1 of the other pool, with their scores and GPU counts
+__global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict__ src, int32_t* __restrict__ dst,
+                                                      int64_t ld, int32_t k, const int32_t* __restrict__ kept,
+                                                      const double* __restrict__ F, const int32_t* __restrict__ G,
+                                                      double* __restrict__ F_new, int32_t* __restrict__ G_new) {
+    const int lane = threadIdx.x & 31;
+    const int64_t p = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (p >= k) return;
+    const int32_t from = kept[p];
+    const int4* S = reinterpret_cast<const int4*>(src + (int64_t)from * ld);
+    int4* D = reinterpret_cast<int4*>(dst + p * ld);
+    const int32_t nvec = (int32_t)(ld >> 2);
+    for (int32_t v = lane; v < nvec; v += 32) D[v] = S[v];
+    if (lane == 0) {
+        F_new[p] = F[from];
+        G_new[p] = G[from];
+    }
+}
+
+size_t trunc_scratch_bytes(int32_t k) { return 64 + 2 * 1024 * sizeof(int32_t) + (size_t)k * sizeof(int32_t); }
+
+// One generation.  pool/pool_next: 4K rows each; F, G: 4K entries (first K valid on entry); on return the
+// survivors are rows 0..K-1 of pool_next with F_next, G_next.  draws: 3K ints.
+cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, int32_t n_jobs,
+                                         double* F, int32_t* G, double* F_next, int32_t* G_next, int32_t* draws,
+                                         Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
+                                         double penalty, void* scratch, cudaStream_t s, int* launches) {
+    const int32_t n = 4 * k;
+    int32_t per_block = ((n + 1023) / 1024 + 255) / 256 * 256;  // rows per block: multiple of 256, <= 1024 blocks
+    const int32_t blocks = (n + per_block - 1) / per_block;
+    TruncPick* pick = reinterpret_cast<TruncPick*>(scratch);
+    int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64);
+    int32_t* kept = bsum + 2 * 1024;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    cudaError_t e;
+    k_trunc_draws<<<(3 * k + 255) / 256, 256, 0, s>>>(k, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
+                                                      counter3(STREAM_SEL_B, gen), counter3(STREAM_PICK, gen), draws);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const int child_blocks = (int)((2 * (int64_t)k + 7) / 8);
+    if (thr16 >= 65536u)
+        k_trunc_children<true><<<child_blocks, 256, 0, s>>>(pool, ld, k, draws, t, keys, (uint32_t)gen,
+                                                            counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32);
+    else
+        k_trunc_children<false><<<child_blocks, 256, 0, s>>>(pool, ld, k, draws, t, keys, (uint32_t)gen,
+                                                             counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_fitness(pool + (int64_t)k * ld, ld, 3 * k, n_jobs, t, capacity, penalty, F + k, G + k, s)) != cudaSuccess)
+        return e;
+    k_trunc_threshold<<<1, 1024, 0, s>>>(F, n, k, pick);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_trunc_count<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_trunc_scan<<<1, 1024, 0, s>>>(bsum, blocks);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_trunc_place<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum, kept);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_trunc_gather<<<(k + 7) / 8, 256, 0, s>>>(pool, pool_next, ld, k, kept, F, G, F_next, G_next);
+    if (launches) *launches += 8;
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Best candidate and its repair to the cluster's capacity: one block.
 // work[0..jpad) exponent, work[jpad..2jpad) GPUs now, work[2jpad..3jpad) GPUs one exponent lower
 // (-1 when the job cannot shrink).

@@ -249,6 +249,38 @@ def test_set_get_population_roundtrip(ones):
     _same_state(g, o)
 
 
+# ---- the paper's truncation selection (originals + crossover children + mutants, best K survive) -------
+@pytest.mark.parametrize("J,N,kw", [(16, 32, {}), (100, 1024, {}), (37, 101, dict(p_mut=1.0)), (5, 3, dict(p_mut=0.0)),
+                                    (130, 257, dict(p_mut=0.02)), (1, 3, {}), (512, 4096, {})])
+def test_truncation_selection_parity(ones, J, N, kw):
+    w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, pinned=J // 5)
+    g, o = _pair(ones, w, flags=4, **kw)
+    g.randomize(2)
+    o.randomize(2)
+    for step in (1, 1, 3):
+        g.evolve(step, 11)
+        o.evolve(step, 11)
+        pg, _ = g.last_parents()
+        po, _ = o.last_parents()
+        assert pg.shape == (N, 2) and (pg == po).all()
+        _same_state(g, o)
+    bg, bo = g.best(True), o.best(True)
+    assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
+
+
+def test_truncation_selection_with_many_ties(ones):
+    # identical candidates: every score ties, survivors are decided by row order alone
+    w = inputs.tiny()
+    g, o = _pair(ones, w, flags=4, p_mut=0.05)
+    rows = np.tile(inputs.random_genomes(w.jobs, 1, seed=5)[0], (w.pop, 1))
+    g.set_population(rows)
+    o.set_population(rows)
+    for _ in range(4):
+        g.evolve(1, 3)
+        o.evolve(1, 3)
+        _same_state(g, o)
+
+
 # ---- a6: best and repair ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "paper", "mid"])
 def test_best_and_repair_parity(ones, name):
