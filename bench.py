@@ -226,6 +226,8 @@ def main():
     ap.add_argument("--no-kernel-events", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling a smaller case)")
+    ap.add_argument("--scheme", default="tournament", choices=["tournament", "truncation"],
+                    help="truncation = the paper's best-K-of-4K selection (ONES_FLAG_TRUNCATION)")
     args = ap.parse_args()
     if args.workload == "online":
         if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
@@ -235,6 +237,9 @@ def main():
     if args.pop:
         import dataclasses
         w = dataclasses.replace(w, pop=args.pop)
+    if args.scheme == "truncation":
+        import dataclasses
+        w = dataclasses.replace(w, params=dataclasses.replace(w.params, flags=w.params.flags | 4))
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -315,7 +320,7 @@ def main():
 
     # ---- the two separate kernels (crossover/mutation, fitness) on the same workload ----
     sep = None
-    if rank == 0 and world == 1 and not args.no_kernel_events:
+    if rank == 0 and world == 1 and not args.no_kernel_events and args.scheme == "tournament":
         import dataclasses
         s.close()
         del s
@@ -353,7 +358,10 @@ def main():
                 "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs)",
                 "best_fitness": out["fitness"]},
     }
-    if stage_n.get("evolve"):
+    if args.scheme == "truncation":
+        line["config"]["scheme"] = "truncation: pool of 4N rows, 3N new candidates scored per generation"
+        line["new_candidates_per_s"] = 3 * line["value"]
+    if stage_n.get("evolve") and args.scheme == "tournament":
         ev_ms = stage_ms["evolve"] / stage_n["evolve"]
         sel_ms = stage_ms["select"] / stage_n["select"] if stage_n.get("select") else 0.0
         # algorithmic bytes per launch: one parent-row read and one child-row write per child gene (8 B),
