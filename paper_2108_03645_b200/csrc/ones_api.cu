@@ -308,6 +308,13 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
         delete c;
         return ONES_ERR_CUDA;
     }
+    if (trunc) {  // the radix search keeps its histogram and counters zero between launches
+        e = cudaMemsetAsync(c->ws + c->L.trunc, 0, trunc_scratch_bytes(pop), c->stream);
+        if (e != cudaSuccess) {
+            delete c;
+            return ONES_ERR_CUDA;
+        }
+    }
     rc = rebuild_tables(c, jobs, n_jobs);
     if (rc == ONES_OK) {
         e = launch_fill_min(c->pop(0), c->ld, c->N, c->J, c->tab, c->stream);

@@ -52,8 +52,6 @@ cudaError_t launch_randomize(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs
                              RoundKeys keys, cudaStream_t s);
 cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
                            int32_t capacity, double penalty, double* F, int32_t* G, cudaStream_t s);
-cudaError_t launch_select(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
-                          uint64_t gen, int32_t* parents, cudaStream_t s);
 // tournaments + top-e in one launch; *done must be 0 at launch (the kernel leaves it 0)
 cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
                                 uint64_t gen, int32_t* parents, int32_t e, int32_t* elites, void* scratch,

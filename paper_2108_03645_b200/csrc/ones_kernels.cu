@@ -338,45 +338,6 @@ cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Tournament selection: one thread per (pair, parent)
-// ---------------------------------------------------------------------------------------------
-__global__ void k_select(const double* __restrict__ F, int32_t n, int32_t tournament, int32_t pairs,
-                         RoundKeys keys, uint32_t gen_lo, uint32_t c3a, uint32_t c3b,
-                         int32_t* __restrict__ parents) {
-    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= 2 * pairs) return;
-    const uint32_t q = (uint32_t)(i >> 1);
-    const uint32_t c3 = (i & 1) ? c3b : c3a;
-    int32_t win = -1;
-    double fwin = 0.0;
-    for (int32_t t0 = 0; t0 < tournament; t0 += 4) {
-        const uint4 w4 = philox((uint32_t)(t0 >> 2), q, gen_lo, c3, keys);
-        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (t0 + u < tournament) {
-                const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
-                const double f = F[idx];
-                if (win < 0 || f > fwin || (f == fwin && idx < win)) {
-                    win = idx;
-                    fwin = f;
-                }
-            }
-        }
-    }
-    parents[i] = win;
-}
-
-cudaError_t launch_select(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
-                          uint64_t gen, int32_t* parents, cudaStream_t s) {
-    if (pairs <= 0) return cudaSuccess;
-    const int grid = (2 * pairs + 127) / 128;
-    k_select<<<grid, 128, 0, s>>>(F, n, tournament, pairs, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
-                                  counter3(STREAM_SEL_B, gen), parents);
-    return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------------------------
 // Top-e selection (score descending, index ascending): per-block partial lists, then one block
 // merges them.  Scores are mapped to order-preserving 64-bit keys; NaN ranks lowest.
 // ---------------------------------------------------------------------------------------------
@@ -1204,43 +1165,57 @@ struct TruncPick {  // result of the selection threshold search
     int32_t pad;
 };
 
-// K-th largest of n score keys by an 8-pass radix search (one CTA)
-__global__ void __launch_bounds__(1024) k_trunc_threshold(const double* __restrict__ F, int32_t n, int32_t k,
-                                                          TruncPick* __restrict__ out) {
+// K-th largest of n score keys by an 8-pass radix search.  One launch per pass: every CTA histograms the
+// current digit of the keys that match the prefix found so far; the last CTA to finish picks the digit
+// that holds the K-th key, narrows the prefix and clears the histogram for the next pass.
+struct TruncState {
+    unsigned long long prefix;
+    int32_t remaining;
+    unsigned int done;
+    unsigned int hist[256];
+};
+
+__global__ void __launch_bounds__(256) k_trunc_radix_pass(const double* __restrict__ F, int32_t n, int32_t k, int pass,
+                                                          TruncState* __restrict__ st, TruncPick* __restrict__ out) {
     __shared__ unsigned int hist[256];
-    __shared__ unsigned long long s_prefix;
-    __shared__ int32_t s_remaining;
-    if (threadIdx.x == 0) {
-        s_prefix = 0ull;
-        s_remaining = k;
+    __shared__ bool s_last;
+    hist[threadIdx.x] = 0u;
+    __syncthreads();
+    const int shift = 56 - 8 * pass;
+    const unsigned long long mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
+    const unsigned long long prefix = pass == 0 ? 0ull : st->prefix;
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const unsigned long long key = score_key(F[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
     }
-    unsigned long long mask = 0ull;
-    for (int pass = 0; pass < 8; ++pass) {
-        const int shift = 56 - 8 * pass;
-        for (int d = threadIdx.x; d < 256; d += blockDim.x) hist[d] = 0u;
-        __syncthreads();
-        const unsigned long long prefix = s_prefix;
-        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
-            const unsigned long long key = score_key(F[i]);
-            if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int32_t above = 0, d = 255;
-            for (; d > 0; --d) {
-                if (above + (int32_t)hist[d] >= s_remaining) break;
-                above += (int32_t)hist[d];
-            }
-            s_remaining -= above;
-            s_prefix = prefix | ((unsigned long long)d << shift);
-        }
-        mask |= 0xFFull << shift;
-        __syncthreads();
-    }
+    __syncthreads();
+    if (hist[threadIdx.x]) atomicAdd(&st->hist[threadIdx.x], hist[threadIdx.x]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&st->done, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    hist[threadIdx.x] = __ldcg(&st->hist[threadIdx.x]);
+    st->hist[threadIdx.x] = 0u;
+    __syncthreads();
     if (threadIdx.x == 0) {
-        out->key = s_prefix;
-        out->quota = s_remaining;
-        out->pad = 0;
+        int32_t remaining = pass == 0 ? k : st->remaining;
+        int32_t above = 0, d = 255;
+        for (; d > 0; --d) {
+            if (above + (int32_t)hist[d] >= remaining) break;
+            above += (int32_t)hist[d];
+        }
+        remaining -= above;
+        const unsigned long long np = prefix | ((unsigned long long)d << shift);
+        st->prefix = np;
+        st->remaining = remaining;
+        st->done = 0u;
+        if (pass == 7) {
+            out->key = np;
+            out->quota = remaining;
+            out->pad = 0;
+        }
     }
 }
 
@@ -1347,7 +1322,9 @@ __global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict_
     }
 }
 
-size_t trunc_scratch_bytes(int32_t k) { return 64 + 2 * 1024 * sizeof(int32_t) + (size_t)k * sizeof(int32_t); }
+size_t trunc_scratch_bytes(int32_t k) {
+    return 64 + sizeof(TruncState) + 2 * 1024 * sizeof(int32_t) + (size_t)k * sizeof(int32_t);
+}
 
 // One generation.  pool/pool_next: 4K rows each; F, G: 4K entries (first K valid on entry); on return the
 // survivors are rows 0..K-1 of pool_next with F_next, G_next.  draws: 3K ints.
@@ -1359,7 +1336,8 @@ cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int6
     int32_t per_block = ((n + 1023) / 1024 + 255) / 256 * 256;  // rows per block: multiple of 256, <= 1024 blocks
     const int32_t blocks = (n + per_block - 1) / per_block;
     TruncPick* pick = reinterpret_cast<TruncPick*>(scratch);
-    int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64);
+    TruncState* state = reinterpret_cast<TruncState*>(reinterpret_cast<char*>(scratch) + 64);
+    int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64 + sizeof(TruncState));
     int32_t* kept = bsum + 2 * 1024;
     const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
     cudaError_t e;
@@ -1376,8 +1354,14 @@ cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int6
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = launch_fitness(pool + (int64_t)k * ld, ld, 3 * k, n_jobs, t, capacity, penalty, F + k, G + k, s)) != cudaSuccess)
         return e;
-    k_trunc_threshold<<<1, 1024, 0, s>>>(F, n, k, pick);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    {
+        int rb = (n + 2047) / 2048;
+        if (rb > kSMs) rb = kSMs;
+        for (int pass = 0; pass < 8; ++pass) {
+            k_trunc_radix_pass<<<rb, 256, 0, s>>>(F, n, k, pass, state, pick);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
+    }
     k_trunc_count<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     k_trunc_scan<<<1, 1024, 0, s>>>(bsum, blocks);
@@ -1385,7 +1369,7 @@ cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int6
     k_trunc_place<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum, kept);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     k_trunc_gather<<<(k + 7) / 8, 256, 0, s>>>(pool, pool_next, ld, k, kept, F, G, F_next, G_next);
-    if (launches) *launches += 8;
+    if (launches) *launches += 15;
     return cudaGetLastError();
 }
 
