@@ -361,6 +361,19 @@ def main():
     if args.scheme == "truncation":
         line["config"]["scheme"] = "truncation: pool of 4N rows, 3N new candidates scored per generation"
         line["new_candidates_per_s"] = 3 * line["value"]
+        if stage_n.get("evolve"):
+            peak, peak_kind = measured_peak()
+            rows = {"children (k_trunc_draws + k_trunc_children)": ("evolve", 6 * N * J * 4),
+                    "k_fitness over the 3N new rows": ("fitness", 3 * N * (4 * J + 12)),
+                    "selection (radix threshold, compaction, k_trunc_gather)": ("select", 2 * N * J * 4 + 4 * N * 8 * 10)}
+            line["kernels"] = {}
+            for name, (stage, nbytes) in rows.items():
+                t_ms = stage_ms[stage] / stage_n[stage]
+                a = nbytes / (t_ms * 1e-3) / 1e9
+                line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
+                                         "bytes_per_generation": nbytes, "ms_per_generation": t_ms}
+            dom = max(line["kernels"].items(), key=lambda kv: kv[1]["ms_per_generation"])
+            line["roofline"] = dict(dom[1], kernel=dom[0], peak_kind=f"of {peak_kind}", traffic=None)
     if stage_n.get("evolve") and args.scheme == "tournament":
         ev_ms = stage_ms["evolve"] / stage_n["evolve"]
         sel_ms = stage_ms["select"] / stage_n["select"] if stage_n.get("select") else 0.0

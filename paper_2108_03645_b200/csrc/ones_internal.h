@@ -83,10 +83,11 @@ cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t
                               int32_t capacity, double penalty, void* scratch, unsigned int* done, cudaStream_t s);
 // The paper's truncation selection over a pool of 4K rows (ONES_FLAG_TRUNCATION)
 size_t trunc_scratch_bytes(int32_t k);
-cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, int32_t n_jobs,
-                                         double* F, int32_t* G, double* F_next, int32_t* G_next, int32_t* draws,
-                                         Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                         double penalty, void* scratch, cudaStream_t s, int* launches);
+cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
+                                  uint64_t gen, uint32_t thr16, cudaStream_t s);  // 2 launches
+cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
+                                const int32_t* G, double* F_next, int32_t* G_next, void* scratch,
+                                cudaStream_t s);  // 12 launches
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,

@@ -1326,24 +1326,14 @@ size_t trunc_scratch_bytes(int32_t k) {
     return 64 + sizeof(TruncState) + 2 * 1024 * sizeof(int32_t) + (size_t)k * sizeof(int32_t);
 }
 
-// One generation.  pool/pool_next: 4K rows each; F, G: 4K entries (first K valid on entry); on return the
-// survivors are rows 0..K-1 of pool_next with F_next, G_next.  draws: 3K ints.
-cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, int32_t n_jobs,
-                                         double* F, int32_t* G, double* F_next, int32_t* G_next, int32_t* draws,
-                                         Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                         double penalty, void* scratch, cudaStream_t s, int* launches) {
-    const int32_t n = 4 * k;
-    int32_t per_block = ((n + 1023) / 1024 + 255) / 256 * 256;  // rows per block: multiple of 256, <= 1024 blocks
-    const int32_t blocks = (n + per_block - 1) / per_block;
-    TruncPick* pick = reinterpret_cast<TruncPick*>(scratch);
-    TruncState* state = reinterpret_cast<TruncState*>(reinterpret_cast<char*>(scratch) + 64);
-    int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64 + sizeof(TruncState));
-    int32_t* kept = bsum + 2 * 1024;
+// Derive the 3K new candidates of one generation into rows K..4K-1 of the pool.  draws: 3K ints.
+cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
+                                  uint64_t gen, uint32_t thr16, cudaStream_t s) {
     const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
-    cudaError_t e;
     k_trunc_draws<<<(3 * k + 255) / 256, 256, 0, s>>>(k, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
                                                       counter3(STREAM_SEL_B, gen), counter3(STREAM_PICK, gen), draws);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     const int child_blocks = (int)((2 * (int64_t)k + 7) / 8);
     if (thr16 >= 65536u)
         k_trunc_children<true><<<child_blocks, 256, 0, s>>>(pool, ld, k, draws, t, keys, (uint32_t)gen,
@@ -1351,16 +1341,26 @@ cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int6
     else
         k_trunc_children<false><<<child_blocks, 256, 0, s>>>(pool, ld, k, draws, t, keys, (uint32_t)gen,
                                                              counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if ((e = launch_fitness(pool + (int64_t)k * ld, ld, 3 * k, n_jobs, t, capacity, penalty, F + k, G + k, s)) != cudaSuccess)
-        return e;
-    {
-        int rb = (n + 2047) / 2048;
-        if (rb > kSMs) rb = kSMs;
-        for (int pass = 0; pass < 8; ++pass) {
-            k_trunc_radix_pass<<<rb, 256, 0, s>>>(F, n, k, pass, state, pick);
-            if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        }
+    return cudaGetLastError();
+}
+
+// Keep the best K of the 4K scored rows: F, G hold 4K entries; the survivors become rows 0..K-1 of
+// pool_next with F_next, G_next.  12 launches.
+cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
+                                const int32_t* G, double* F_next, int32_t* G_next, void* scratch, cudaStream_t s) {
+    const int32_t n = 4 * k;
+    const int32_t per_block = ((n + 1023) / 1024 + 255) / 256 * 256;  // rows per block: multiple of 256, <= 1024 blocks
+    const int32_t blocks = (n + per_block - 1) / per_block;
+    TruncPick* pick = reinterpret_cast<TruncPick*>(scratch);
+    TruncState* state = reinterpret_cast<TruncState*>(reinterpret_cast<char*>(scratch) + 64);
+    int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64 + sizeof(TruncState));
+    int32_t* kept = bsum + 2 * 1024;
+    cudaError_t e;
+    int rb = (n + 2047) / 2048;
+    if (rb > kSMs) rb = kSMs;
+    for (int pass = 0; pass < 8; ++pass) {
+        k_trunc_radix_pass<<<rb, 256, 0, s>>>(F, n, k, pass, state, pick);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     k_trunc_count<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -1369,7 +1369,6 @@ cudaError_t launch_truncation_generation(int32_t* pool, int32_t* pool_next, int6
     k_trunc_place<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum, kept);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     k_trunc_gather<<<(k + 7) / 8, 256, 0, s>>>(pool, pool_next, ld, k, kept, F, G, F_next, G_next);
-    if (launches) *launches += 15;
     return cudaGetLastError();
 }
 
