@@ -1186,7 +1186,12 @@ __global__ void __launch_bounds__(256) k_trunc_radix_pass(const double* __restri
     const unsigned long long prefix = pass == 0 ? 0ull : st->prefix;
     for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         const unsigned long long key = score_key(F[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
+        if ((key & mask) == prefix) {
+            // similar scores share their leading digits: one atomic per distinct digit in the warp
+            const unsigned int digit = (unsigned int)(key >> shift) & 255u;
+            const unsigned int peers = __match_any_sync(__activemask(), digit);
+            if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned int)__popc(peers));
+        }
     }
     __syncthreads();
     if (hist[threadIdx.x]) atomicAdd(&st->hist[threadIdx.x], hist[threadIdx.x]);
