@@ -137,7 +137,10 @@ def oracle_sample(w, pop_sample: int, gens: int):
     return dt
 
 
-def cpu_baseline(w, pop_sample=8192, gens=8):
+def cpu_baseline(w, pop_sample=8192, gens=None):
+    pop_sample = min(pop_sample, w.pop)
+    if gens is None:  # about 1e8 gene evaluations: seconds of single-thread work
+        gens = int(min(2000, max(8, 1.3e8 / (pop_sample * w.n_jobs))))
     dt = oracle_sample(w, pop_sample, gens)
     return {"value": pop_sample * gens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"{gens} generations of a {pop_sample}-candidate population (of {w.pop}), "
@@ -149,7 +152,7 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    pop_sample = 8192
+    pop_sample = min(8192, w.pop)
     for _ in range(min(args.warmup, 1)):
         oracle_sample(w, pop_sample, 1)
     steps = max(1, min(args.steps, 20))
@@ -382,7 +385,8 @@ def main():
         evolve_bytes = 8 * J * (N - E) + 8 * J * E + 8 * ((N - E + 1) // 2) + 4 * E
         fused_bytes = evolve_bytes + 12 * N
         ach = fused_bytes / (ev_ms * 1e-3) / 1e9
-        line["roofline"] = {"kernel": "k_evolve_score", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+        one_launch = launches <= steps  # small shapes run the whole generation in k_generation
+        line["roofline"] = {"kernel": "k_generation" if one_launch else "k_evolve_score", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
                             "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                             "bytes_per_launch": fused_bytes, "ms_per_launch": ev_ms,
                             "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,

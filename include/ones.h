@@ -17,6 +17,8 @@
  *  - Genome tables are row-major int32[n][ld], ld >= number of jobs, ld % 4 == 0,
  *    base address 16-byte aligned.  Columns >= number of jobs are never read as
  *    genes and never written.
+ *  - Calls on a handle make the handle's device current for their duration and restore the
+ *    caller's device before returning.
  *  - All work is enqueued on the CUDA stream given to ones_create.  Calls that
  *    return data to host memory synchronise that stream; the others do not.
  *  - Every function returns ONES_OK (0) or a negative ONES_ERR_* code.  Nothing is

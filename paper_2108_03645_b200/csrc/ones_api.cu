@@ -251,6 +251,18 @@ int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs) {
     return ONES_OK;
 }
 
+// Work of a handle always goes to the device it was created on, whatever device the caller has current.
+struct DeviceScope {
+    int prev = -1;
+    bool changed = false;
+    explicit DeviceScope(const ones_ctx* c) {
+        if (c && cudaGetDevice(&prev) == cudaSuccess && prev != c->device) changed = cudaSetDevice(c->device) == cudaSuccess;
+    }
+    ~DeviceScope() {
+        if (changed) cudaSetDevice(prev);
+    }
+};
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -340,6 +352,7 @@ int ones_destroy(ones_ctx* c) {
 }
 
 int ones_randomize(ones_ctx* c, uint64_t seed) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->J, c->tab, make_round_keys(seed), c->stream));
     c->launches += 1;
@@ -349,6 +362,7 @@ int ones_randomize(ones_ctx* c, uint64_t seed) {
 }
 
 int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_device) {
+    DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
     if (ld < c->J) return ONES_ERR_BAD_PARAM;
     if (on_device) {
@@ -366,6 +380,7 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
 }
 
 int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device) {
+    DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
     if (ld < c->J) return ONES_ERR_BAD_PARAM;
     if (on_device) {
@@ -380,6 +395,7 @@ int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device
 }
 
 int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, double* d_fitness, int32_t* d_gpus) {
+    DeviceScope scope(c);
     if (!c || !d_fitness) return ONES_ERR_NULL;
     if (!d_genomes) {
         if (!c->f_valid) {
@@ -401,6 +417,7 @@ int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, 
 }
 
 int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     if (generations < 0) return ONES_ERR_BAD_PARAM;
     if (generations == 0) return ONES_OK;
@@ -499,6 +516,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
 
 int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_job, double* h_rate_per_job,
               double* fitness, int32_t* total_gpus, int32_t* index) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     int rc;
     if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
@@ -526,6 +544,7 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
 }
 
 int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const int32_t* remap, int32_t capacity) {
+    DeviceScope scope(c);
     if (!c || !jobs || !remap) return ONES_ERR_NULL;
     int rc = check_jobs(jobs, n_jobs);
     if (rc) return rc;
@@ -556,6 +575,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
 }
 
 int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     if (h_parents && c->pairs > 0)
         CU(c, cudaMemcpyAsync(h_parents, c->parents(), (size_t)c->pairs * 8, cudaMemcpyDeviceToHost, c->stream));
@@ -566,6 +586,7 @@ int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
 }
 
 int ones_model_table(ones_ctx* c, double* h_X, int32_t* h_g, int32_t* planes) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     if (planes) *planes = c->tab.k1;
     if (!h_X && !h_g) return ONES_OK;
@@ -624,6 +645,7 @@ int ones_kernel_launches(const ones_ctx* c, uint64_t* launches) {
 }
 
 int ones_set_profiling(ones_ctx* c, int on) {
+    DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
     if (on && c->prof.ev.empty()) {
         const size_t want = 4096;
@@ -646,6 +668,7 @@ int ones_set_profiling(ones_ctx* c, int on) {
 }
 
 int ones_stage_times(ones_ctx* c, double ms[3], uint64_t count[3]) {
+    DeviceScope scope(c);
     if (!c || !ms || !count) return ONES_ERR_NULL;
     int rc = prof_flush(c);
     if (rc) return rc;
