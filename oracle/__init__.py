@@ -53,42 +53,65 @@ def build(force: bool = False) -> str:
 _lib = None
 
 
+def _configure(L: C.CDLL) -> C.CDLL:
+    vp, i32, i64, u32, u64, dbl = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_double
+    L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+    L.oracle_philox4x32_10.restype = None
+    L.oracle_word.argtypes = [u64, u64, u32, u32, u32]
+    L.oracle_word.restype = u32
+    L.oracle_model.argtypes = [vp, i32, vp, vp]
+    L.oracle_term.argtypes = [vp, i32, u32, vp, vp]
+    L.oracle_fitness.argtypes = [vp, i32, i32, dbl, u32, vp, vp, vp]
+    L.oracle_validate_jobs.argtypes = [vp, i32]
+    L.oracle_repair.argtypes = [vp, i32, i32, vp]
+    L.oracle_tournament.argtypes = [vp, i32, i32, u64, u64, u32, u32]
+    L.oracle_tournament.restype = i32
+    L.oracle_top.argtypes = [vp, i32, i32, vp]
+    L.oracle_keep_best.argtypes = [vp, i32, i32, vp]
+    L.oracle_thr16.argtypes = [dbl]
+    L.oracle_thr16.restype = u32
+    L.oracle_create.argtypes = [vp, vp, i32, i32, i32, vp]
+    L.oracle_destroy.argtypes = [vp]
+    L.oracle_randomize.argtypes = [vp, u64]
+    L.oracle_set_population.argtypes = [vp, vp, i64]
+    L.oracle_get_population.argtypes = [vp, vp, i64]
+    L.oracle_evaluate.argtypes = [vp, vp, i64, i32, vp, vp]
+    L.oracle_evolve.argtypes = [vp, i32, u64]
+    L.oracle_best.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp, vp]
+    L.oracle_update_jobs.argtypes = [vp, vp, i32, vp, i32]
+    L.oracle_last_parents.argtypes = [vp, vp, vp]
+    L.oracle_generation.argtypes = [vp, vp]
+    L.oracle_set_generation.argtypes = [vp, u64]
+    L.oracle_pairs.argtypes = [vp]
+    L.oracle_pairs.restype = i32
+    return L
+
+
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
-        vp, i32, i64, u32, u64, dbl = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_double
-        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
-        L.oracle_philox4x32_10.restype = None
-        L.oracle_word.argtypes = [u64, u64, u32, u32, u32]
-        L.oracle_word.restype = u32
-        L.oracle_model.argtypes = [vp, i32, vp, vp]
-        L.oracle_term.argtypes = [vp, i32, u32, vp, vp]
-        L.oracle_fitness.argtypes = [vp, i32, i32, dbl, u32, vp, vp, vp]
-        L.oracle_validate_jobs.argtypes = [vp, i32]
-        L.oracle_repair.argtypes = [vp, i32, i32, vp]
-        L.oracle_tournament.argtypes = [vp, i32, i32, u64, u64, u32, u32]
-        L.oracle_tournament.restype = i32
-        L.oracle_top.argtypes = [vp, i32, i32, vp]
-        L.oracle_keep_best.argtypes = [vp, i32, i32, vp]
-        L.oracle_thr16.argtypes = [dbl]
-        L.oracle_thr16.restype = u32
-        L.oracle_create.argtypes = [vp, vp, i32, i32, i32, vp]
-        L.oracle_destroy.argtypes = [vp]
-        L.oracle_randomize.argtypes = [vp, u64]
-        L.oracle_set_population.argtypes = [vp, vp, i64]
-        L.oracle_get_population.argtypes = [vp, vp, i64]
-        L.oracle_evaluate.argtypes = [vp, vp, i64, i32, vp, vp]
-        L.oracle_evolve.argtypes = [vp, i32, u64]
-        L.oracle_best.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp, vp]
-        L.oracle_update_jobs.argtypes = [vp, vp, i32, vp, i32]
-        L.oracle_last_parents.argtypes = [vp, vp, vp]
-        L.oracle_generation.argtypes = [vp, vp]
-        L.oracle_set_generation.argtypes = [vp, u64]
-        L.oracle_pairs.argtypes = [vp]
-        L.oracle_pairs.restype = i32
-        _lib = L
+        _lib = _configure(C.CDLL(build()))
     return _lib
+
+
+class use_library:
+    """Context manager: run the wrappers of this module against another build of the oracle
+    (the tests use it to show that a planted mistake is caught by the pins)."""
+
+    def __init__(self, path: str):
+        self.path = path
+
+    def __enter__(self):
+        global _lib
+        lib()
+        self.saved = _lib
+        _lib = _configure(C.CDLL(self.path))
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self.saved
+        return False
 
 
 def _jobs_arr(jobs) -> np.ndarray:

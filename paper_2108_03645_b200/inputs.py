@@ -127,7 +127,7 @@ def large(seed: int = 0) -> Workload:
 
 def custom(n_jobs: int, capacity: int, pop: int, generations: int, *, seed: int = 0,
            kmax: int = 7, log_uniform: bool = False, pinned: int = 0,
-           params: SearchParams | None = None, pow2: bool = True) -> Workload:
+           params: SearchParams | None = None, pow2: bool = True, kmin_max: int = 0) -> Workload:
     """A workload of arbitrary shape (ragged J, odd N, ...) for edge-case tests.
 
     ``pow2=False`` draws b0 and max_per_gpu from values that are not powers of
@@ -139,6 +139,8 @@ def custom(n_jobs: int, capacity: int, pop: int, generations: int, *, seed: int 
                       pinned=pinned)
     if not pow2:
         jobs["b0"] = rng.choice(np.array([24, 40, 72, 100], dtype=np.int32), size=n_jobs)
+    if kmin_max > 0:  # lower limits above the smallest batch (never above the job's upper limit)
+        jobs["kmin"] = np.minimum(rng.integers(0, kmin_max + 1, size=n_jobs), jobs["kmax"]).astype(np.int32)
     return Workload("custom", jobs, capacity, pop, generations,
                     params or SearchParams(), seed)
 

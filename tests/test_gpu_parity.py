@@ -88,6 +88,25 @@ def test_fitness_parity(ones, J, n, ld_extra):
     assert Fo[0] == 0.0 and Go[0] == 0
 
 
+def test_fitness_summation_order_case(ones):
+    # 2^53 next to a few ones: the documented order keeps exactly two of them (see the oracle's pin)
+    jobs = np.zeros(16, dtype=inputs.JOB_DTYPE)
+    jobs["b0"] = 128
+    jobs["max_per_gpu"] = 128
+    jobs["a"] = 128.0
+    jobs["a"][0] = 2.0 ** -46
+    jobs["weight"] = 1.0
+    genome = np.full((3, 16), -1, dtype=np.int32)
+    genome[:, [0, 1, 2, 3, 4, 8, 12]] = 0
+    s = ones.Search(jobs, 10 ** 6, 3, inputs.SearchParams(1, 2, 0.1, 1e3))
+    F, G = s.evaluate(torch.from_numpy(genome).cuda())
+    assert F.cpu().tolist() == [2.0 ** 53 + 2.0] * 3 and G.cpu().tolist() == [7, 7, 7]
+    s.set_population(genome)  # the evolve kernels score in the same order
+    s.evolve(1, 0)
+    F2, _ = s.evaluate()
+    assert F2.cpu().tolist()[0] == 2.0 ** 53 + 2.0  # the elite row, copied and scored again
+
+
 def test_fitness_zero_rows_and_sruf(ones):
     w = inputs.paper_scale(1)
     w.jobs["weight"] = np.random.default_rng(0).uniform(1e3, 1e6, w.n_jobs)
@@ -163,7 +182,7 @@ def test_evolve_parity_mid_sampled_generations(ones):
                                 dict(penalty=0.0), dict(penalty=37.5), dict(flags=2), dict(flags=2, p_mut=1.0),
                                 dict(flags=3)])
 def test_evolve_parity_parameter_corners(ones, kw):
-    w = inputs.custom(37, 48, 101, 6, seed=7, kmax=6, pinned=4)
+    w = inputs.custom(37, 48, 101, 6, seed=7, kmax=6, pinned=4, kmin_max=3)
     g, o = _pair(ones, w, **kw)
     g.randomize(5)
     o.randomize(5)
@@ -253,7 +272,7 @@ def test_set_get_population_roundtrip(ones):
 @pytest.mark.parametrize("J,N,kw", [(16, 32, {}), (100, 1024, {}), (37, 101, dict(p_mut=1.0)), (5, 3, dict(p_mut=0.0)),
                                     (130, 257, dict(p_mut=0.02)), (1, 3, {}), (512, 4096, {})])
 def test_truncation_selection_parity(ones, J, N, kw):
-    w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, pinned=J // 5)
+    w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, pinned=J // 5, kmin_max=2)
     g, o = _pair(ones, w, flags=4, **kw)
     g.randomize(2)
     o.randomize(2)

@@ -168,3 +168,26 @@ def test_validation():
     j = jobs.copy()
     j["a"][0] = j["c"][0] = j["d"][0] = 0.0  # t = 0
     assert oracle.validate_jobs(j) < 0
+
+
+def test_summation_order_is_the_documented_one():
+    # 2^53 next to a few ones: which ones survive the rounding depends on the order of the additions.
+    # Documented order: 32 partial sums, job j to partial (j / 4) % 32 in increasing j, then a pairwise
+    # tree with offsets 16, 8, 4, 2, 1.  Jobs 1-3 share partial 0 with the big value and are absorbed one
+    # by one; jobs 4, 8, 12 sit in partials 1, 2, 3: 1 + 1 joins first, then 2^53 + 2 is exact.
+    from paper_2108_03645_b200.inputs import JOB_DTYPE
+    J = 16
+    jobs = np.zeros(J, dtype=JOB_DTYPE)
+    jobs["b0"] = 128
+    jobs["max_per_gpu"] = 128
+    jobs["a"] = 128.0            # X = 128 / a = 1
+    jobs["a"][0] = 2.0 ** -46    # X = 2^53
+    jobs["weight"] = 1.0
+    genome = np.full(J, -1, dtype=np.int32)  # everybody else waits
+    genome[[0, 1, 2, 3, 4, 8, 12]] = 0
+    assert oracle.model(jobs, 0, 0) == (2.0 ** 53, 1) and oracle.model(jobs, 5, 0) == (1.0, 1)
+    F, G = oracle.fitness(jobs, 10 ** 6, 1e3, genome)
+    assert G == 7
+    assert F == 2.0 ** 53 + 2.0
+    # a left-to-right sum loses every one; one partial per job (j % 32) would give 2^53 + 6
+    assert F != 2.0 ** 53 and F != 2.0 ** 53 + 6.0

@@ -289,9 +289,9 @@ def test_update_jobs_remaps_columns():
     s = _search(w)
     s.randomize(0)
     P = s.get_population()
-    # jobs 3 and 7 finished; two jobs arrive (pinned at k=0); job 5's limit drops to 2
+    # jobs 3 and 7 finished; two jobs arrive; job 5's limit drops to 2
     keep = [j for j in range(16) if j not in (3, 7)]
-    new = inputs.custom(2, 16, 32, 1, seed=9, kmax=0).jobs
+    new = inputs.custom(2, 16, 32, 1, seed=9, kmax=3).jobs  # they may grow later, but start at their smallest batch
     jobs2 = np.concatenate([w.jobs[keep], new])
     jobs2["kmax"][keep.index(5)] = 2
     remap = np.array(keep + [-1, -1], dtype=np.int32)
@@ -357,3 +357,19 @@ def test_checkpoint_and_resume():
     c.set_generation(gen)
     c.evolve(5, 3)
     assert (c.get_population() == a.get_population()).all() and c.generation == 9
+
+
+def test_lower_limits_are_respected():
+    w = inputs.custom(40, 10 ** 6, 200, 1, seed=12, kmax=6, kmin_max=4)
+    assert w.jobs["kmin"].max() >= 3
+    s = _search(w, p_mut=0.5)
+    assert (s.get_population() == w.jobs["kmin"][None, :]).all()
+    s.randomize(1)
+    for _ in range(3):
+        P = s.get_population()
+        assert (P >= w.jobs["kmin"][None, :]).all() and (P <= w.jobs["kmax"][None, :]).all()
+        s.evolve(1, 1)
+    # every admissible value of a free job is reached, the lowest and the highest included
+    j = int(np.argmax(w.jobs["kmax"] - w.jobs["kmin"]))
+    seen = set(P[:, j].tolist())
+    assert seen == set(range(int(w.jobs["kmin"][j]), int(w.jobs["kmax"][j]) + 1))
