@@ -13,7 +13,9 @@
  *  - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global
  *    memory of the device that was current at ones_create.  The caller owns every
  *    buffer it passes, including the device workspace; the handle owns only small
- *    host-side state.  Nothing here allocates or frees device memory.
+ *    host-side state (including a few KiB of pinned host memory through which job tables
+ *    are uploaded and the best schedule is downloaded).  Nothing here allocates or frees
+ *    device memory.
  *  - Genome tables are row-major int32[n][ld], ld >= number of jobs, ld % 4 == 0,
  *    base address 16-byte aligned.  Columns >= number of jobs are never read as
  *    genes and never written.
@@ -78,6 +80,11 @@ typedef struct {
  * sized with ones_workspace_bytes_flags (the pool takes 4x the rows).  ones_last_parents then
  * returns [pop][2] parent rows. */
 #define ONES_FLAG_TRUNCATION 4u
+
+/* Small populations normally run all generations of a ones_evolve call in one launch of one
+ * thread-block cluster, with the population in the cluster's shared memory.  This flag keeps the
+ * launch-per-generation sequence instead (same results). */
+#define ONES_FLAG_NO_CLUSTER 8u
 
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
 #define ONES_MAX_ELITES 256   /* elitism <= 256 */

@@ -19,6 +19,7 @@ from .inputs import JOB_DTYPE, SearchParams
 FLAG_SRUF = 1
 FLAG_UNFUSED = 2
 FLAG_TRUNCATION = 4
+FLAG_NO_CLUSTER = 8
 MAX_ELITES = 256
 
 ERRORS = {0: "ONES_OK", -1: "ONES_ERR_NULL", -2: "ONES_ERR_BAD_JOB", -3: "ONES_ERR_BAD_PARAM",

@@ -26,8 +26,8 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, G1, trunc, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs, remap, top, work, out_genome,
-        out_gpus, out_rate, out_rec, exp_X, exp_G, status, total;
+    size_t pop0, pop1, F, F1, G, G1, trunc, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+        status, total;
 };
 
 Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
@@ -57,17 +57,13 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
     L.Gt = take((size_t)kPlanesMax * jp * 4);
     L.kmin = take(jp * 4);
     L.range = take(jp * 4);
-    L.jobs = take((size_t)jmax * sizeof(ones_job));
-    L.remap = take((size_t)jmax * 4);
+    L.jobs_in = take((size_t)jmax * (sizeof(ones_job) + 4));  // job rows, then the remap entries of an update
     {
         const size_t a = top_scratch_bytes(pop, ONES_MAX_ELITES), b = generation_scratch_bytes(ONES_MAX_ELITES);
         L.top = take(a > b ? a : b);
     }
     L.work = take(3 * jp * 4);
-    L.out_genome = take((size_t)jmax * 4);
-    L.out_gpus = take((size_t)jmax * 4);
-    L.out_rate = take((size_t)jmax * 8);
-    L.out_rec = take(sizeof(BestOut));
+    L.out_pack = take(64 + (size_t)jmax * 16);  // BestOut, then rate, genome, gpus of the returned schedule
     L.exp_X = take((size_t)(kPlanesMax - 1) * jmax * 8);
     L.exp_G = take((size_t)(kPlanesMax - 1) * jmax * 4);
     L.status = take(16);
@@ -108,10 +104,13 @@ struct ones_ctx {
     uint64_t gen = 0;
     Tables tab{};
     bool fused = false;  // children are scored inside the evolve kernel
+    ClusterShape cshape{0, 0, 0, 0, 0};  // one-cluster, one-launch path for small populations
     std::vector<ones_job> h_jobs;  // the job table the device tables were built from
     uint64_t launches = 0;
     int last_cuda = 0;
     Prof prof;
+    unsigned char* staging = nullptr;  // small pinned host buffer: uploads and downloads go through it in one copy
+    size_t staging_bytes = 0;
 
     int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
     double* Fbuf(int which) { return reinterpret_cast<double*>(ws + (which ? L.F1 : L.F)); }
@@ -121,12 +120,26 @@ struct ones_ctx {
     int32_t* parents() { return reinterpret_cast<int32_t*>(ws + L.parents); }
     int32_t* elites(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.elites1 : L.elites)); }
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
-    ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs); }
-    int32_t* remap() { return reinterpret_cast<int32_t*>(ws + L.remap); }
+    ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs_in); }
+    int32_t* remap(int32_t n_jobs) { return reinterpret_cast<int32_t*>(ws + L.jobs_in + (size_t)n_jobs * sizeof(ones_job)); }
     int32_t* status() { return reinterpret_cast<int32_t*>(ws + L.status); }
 };
 
 namespace {
+
+int cuda_fail(ones_ctx* c, cudaError_t e);
+
+int ensure_staging(ones_ctx* c, size_t bytes) {
+    if (bytes <= c->staging_bytes) return ONES_OK;
+    if (c->staging) cudaFreeHost(c->staging);
+    c->staging = nullptr;
+    c->staging_bytes = 0;
+    const size_t want = bytes < 4096 ? 4096 : 2 * bytes;
+    cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->staging), want);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->staging_bytes = want;
+    return ONES_OK;
+}
 
 int cuda_fail(ones_ctx* c, cudaError_t e) {
     if (c) c->last_cuda = (int)e;
@@ -184,6 +197,9 @@ void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
         if ((b + m - 1) / m > 65535) narrow = false;
     }
     c->fused = narrow && !(c->prm.flags & ONES_FLAG_UNFUSED) && evolve_score_smem(c->tab) <= (size_t)kMaxSmemPerBlock;
+    c->cshape = ClusterShape{0, 0, 0, 0, 0};
+    if (c->fused && !c->trunc && !(c->prm.flags & ONES_FLAG_NO_CLUSTER))
+        c->cshape = cluster_shape(c->tab, ld_of(n_jobs), c->N, c->prm.elitism, c->pairs);
 }
 
 // ---- per-stage timing with CUDA events on the handle's stream ----
@@ -233,9 +249,14 @@ int run_fitness(ones_ctx* c) {
     return prof_end(c);
 }
 
-int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs) {
+int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const int32_t* h_remap = nullptr) {
+    const size_t jb = sizeof(ones_job) * (size_t)n_jobs, rb = h_remap ? (size_t)n_jobs * 4 : 0;
+    int rc = ensure_staging(c, jb + rb);
+    if (rc) return rc;
+    memcpy(c->staging, h_jobs, jb);
+    if (h_remap) memcpy(c->staging + jb, h_remap, rb);
     CU(c, cudaMemsetAsync(c->status(), 0, 16, c->stream));
-    CU(c, cudaMemcpyAsync(c->jobs(), h_jobs, sizeof(ones_job) * (size_t)n_jobs, cudaMemcpyHostToDevice, c->stream));
+    CU(c, cudaMemcpyAsync(c->jobs(), c->staging, jb + rb, cudaMemcpyHostToDevice, c->stream));
     set_tables(c, h_jobs, n_jobs);
     CU(c, launch_build_tables(c->jobs(), n_jobs, c->prm.flags, c->tab, c->status(), c->stream));
     c->launches += 1;
@@ -262,6 +283,13 @@ struct DeviceScope {
         if (changed) cudaSetDevice(prev);
     }
 };
+
+void free_ctx(ones_ctx* c) {
+    if (!c) return;
+    for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
+    if (c->staging) cudaFreeHost(c->staging);
+    delete c;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -317,13 +345,13 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     c->L = make_layout(c->Jmax, pop, trunc);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) {
-        delete c;
+        free_ctx(c);
         return ONES_ERR_CUDA;
     }
     if (trunc) {  // the radix search keeps its histogram and counters zero between launches
         e = cudaMemsetAsync(c->ws + c->L.trunc, 0, trunc_scratch_bytes(pop), c->stream);
         if (e != cudaSuccess) {
-            delete c;
+            free_ctx(c);
             return ONES_ERR_CUDA;
         }
     }
@@ -334,7 +362,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
         if (e != cudaSuccess) rc = cuda_fail(c, e);
     }
     if (rc != ONES_OK) {
-        delete c;
+        free_ctx(c);
         return rc;
     }
     c->cur = 0;
@@ -346,8 +374,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
 
 int ones_destroy(ones_ctx* c) {
     if (!c) return ONES_OK;
-    for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
-    delete c;
+    free_ctx(c);
     return ONES_OK;
 }
 
@@ -454,6 +481,19 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         return ONES_OK;
     }
     const int32_t E = c->prm.elitism;
+    if (c->cshape.cluster > 0) {
+        // small population: every generation of this call inside one cluster launch
+        if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
+        CU(c, launch_evolve_cluster(c->cshape, c->pop(c->cur), c->ld, c->N, c->J, E, c->pairs, c->prm.tournament, c->F(),
+                                    c->G(), c->parents(), c->elites(0), c->tab, keys, c->gen, generations, c->thr16,
+                                    c->cap, c->prm.penalty, c->stream));
+        c->launches += 1;
+        if ((rc = prof_end(c)) != ONES_OK) return rc;
+        c->gen += (uint64_t)generations;
+        c->elast = 0;
+        c->elites_valid = false;
+        return ONES_OK;
+    }
     unsigned int* done = reinterpret_cast<unsigned int*>(c->status() + 1);
     const GenerationShape shape = c->fused ? generation_shape(c->tab, c->pairs, E) : GenerationShape{0, 0, 0, 0};
     if (shape.blocks > 0) {
@@ -522,21 +562,24 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
     if (!c->f_valid && (rc = run_fitness(c)) != ONES_OK) return rc;
     int nl = 0;
     CU(c, launch_top(c->F(), c->N, 1, c->best_idx(), c->ws + c->L.top, c->stream, &nl));
-    int32_t* d_genome = reinterpret_cast<int32_t*>(c->ws + c->L.out_genome);
-    int32_t* d_gpus = reinterpret_cast<int32_t*>(c->ws + c->L.out_gpus);
-    double* d_rate = reinterpret_cast<double*>(c->ws + c->L.out_rate);
-    BestOut* d_rec = reinterpret_cast<BestOut*>(c->ws + c->L.out_rec);
+    const size_t J = (size_t)c->J;
+    unsigned char* pack = reinterpret_cast<unsigned char*>(c->ws + c->L.out_pack);
+    BestOut* d_rec = reinterpret_cast<BestOut*>(pack);
+    double* d_rate = reinterpret_cast<double*>(pack + 64);
+    int32_t* d_genome = reinterpret_cast<int32_t*>(pack + 64 + J * 8);
+    int32_t* d_gpus = reinterpret_cast<int32_t*>(pack + 64 + J * 12);
     CU(c, launch_best(c->pop(c->cur), c->ld, c->J, c->best_idx(), c->tab, c->cap, c->prm.penalty, repair,
                       reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
     c->launches += (uint64_t)nl + 1;
-    BestOut rec;
-    if (h_genome) CU(c, cudaMemcpyAsync(h_genome, d_genome, (size_t)c->J * 4, cudaMemcpyDeviceToHost, c->stream));
-    if (h_gpus_per_job)
-        CU(c, cudaMemcpyAsync(h_gpus_per_job, d_gpus, (size_t)c->J * 4, cudaMemcpyDeviceToHost, c->stream));
-    if (h_rate_per_job)
-        CU(c, cudaMemcpyAsync(h_rate_per_job, d_rate, (size_t)c->J * 8, cudaMemcpyDeviceToHost, c->stream));
-    CU(c, cudaMemcpyAsync(&rec, d_rec, sizeof rec, cudaMemcpyDeviceToHost, c->stream));
+    const size_t bytes = 64 + J * 16;
+    if ((rc = ensure_staging(c, bytes)) != ONES_OK) return rc;
+    CU(c, cudaMemcpyAsync(c->staging, pack, bytes, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
+    BestOut rec;
+    memcpy(&rec, c->staging, sizeof rec);
+    if (h_rate_per_job) memcpy(h_rate_per_job, c->staging + 64, J * 8);
+    if (h_genome) memcpy(h_genome, c->staging + 64 + J * 8, J * 4);
+    if (h_gpus_per_job) memcpy(h_gpus_per_job, c->staging + 64 + J * 12, J * 4);
     if (fitness) *fitness = rec.fitness;
     if (total_gpus) *total_gpus = rec.total_gpus;
     if (index) *index = rec.index;
@@ -553,8 +596,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
     for (int32_t j = 0; j < n_jobs; ++j)
         if (remap[j] < -1 || remap[j] >= c->J) return ONES_ERR_BAD_PARAM;
     const int64_t old_ld = c->ld;
-    CU(c, cudaMemcpyAsync(c->remap(), remap, (size_t)n_jobs * 4, cudaMemcpyHostToDevice, c->stream));
-    rc = rebuild_tables(c, jobs, n_jobs);
+    rc = rebuild_tables(c, jobs, n_jobs, remap);
     if (rc != ONES_OK) {
         // put the tables of the job set in force back; the population is untouched
         const std::vector<ones_job> keep = c->h_jobs;
@@ -562,7 +604,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
         return rc2 == ONES_OK ? rc : rc2;
     }
     const int64_t new_ld = ld_of(n_jobs);
-    CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(), c->tab.kmin,
+    CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(n_jobs), c->tab.kmin,
                        c->tab.range, c->stream));
     c->launches += 1;
     c->cur ^= 1;

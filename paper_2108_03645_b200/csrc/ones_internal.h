@@ -81,6 +81,18 @@ cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t
                               double* F_new, int32_t* G, int32_t* parents, const int32_t* elites,
                               int32_t* elites_next, Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16,
                               int32_t capacity, double penalty, void* scratch, unsigned int* done, cudaStream_t s);
+// All generations of one call in one launch of one thread-block cluster (population in distributed shared memory)
+struct ClusterShape {
+    int cluster, threads;  // cluster == 0: not applicable
+    int32_t rows_per_cta;
+    int gs;                // lanes per pair of children
+    size_t smem;
+};
+ClusterShape cluster_shape(Tables t, int64_t ld, int32_t n, int32_t elitism, int32_t pairs);
+cudaError_t launch_evolve_cluster(ClusterShape shape, int32_t* pop_io, int64_t ld, int32_t n, int32_t n_jobs,
+                                  int32_t elitism, int32_t pairs, int32_t tournament, double* F_io, int32_t* G_out,
+                                  int32_t* parents_out, int32_t* elites_out, Tables t, RoundKeys keys, uint64_t gen0,
+                                  int32_t generations, uint32_t thr16, int32_t capacity, double penalty, cudaStream_t s);
 // The paper's truncation selection over a pool of 4K rows (ONES_FLAG_TRUNCATION)
 size_t trunc_scratch_bytes(int32_t k);
 cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,

@@ -7,6 +7,7 @@
 //   model tables X (fp64) and G (int32), one plane per exponent, swizzled (see Tables)
 // Nothing here is a dense contraction: the kernels are gathers, adds and a counter-based RNG,
 // bounded by HBM bandwidth (fitness, evolve) or by launch latency (everything else).
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
@@ -1096,6 +1097,303 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
     kern<<<(int)blocks, kThreads, smem, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
                                              (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G);
     return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Small populations: all generations of one ones_evolve call in ONE launch of one thread-block
+// cluster.  Both population buffers, the scores and the model tables live in the shared memory of
+// the cluster's CTAs (CTA r owns rows r*rows_per_cta ...); parents and scores of other CTAs are read,
+// and children that belong to a neighbour written, through distributed shared memory; each CTA copies
+// all scores into its own shared memory once per generation for the tournaments and the elites.  One
+// hardware cluster barrier per generation replaces the kernel boundaries; nothing spins.  Lanes are grouped so that one group of `gs` lanes (gs = int4 per
+// row rounded up to a power of two, at most 32) handles one pair of children: with 6 jobs a warp
+// runs 16 pairs at once.  Draws, operators, summation order and elites are those of the other paths.
+// ---------------------------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+
+struct ClusterSmem {  // byte offsets into dynamic shared memory
+    size_t X, F0, F1, Fall, G16, pop0, pop1, Gc, kmin, range, elit, total;
+};
+
+__host__ __device__ inline ClusterSmem cluster_smem(int32_t planes, int32_t jpad, int64_t ld, int32_t rows,
+                                                    int32_t elitism, int32_t n) {
+    ClusterSmem m;
+    size_t at = 0;
+    const size_t e = (size_t)(elitism > 0 ? elitism : 1);
+#define ONES_TAKE(field, bytes) m.field = at; at = (at + (size_t)(bytes) + 15) & ~(size_t)15
+    ONES_TAKE(X, (size_t)planes * jpad * 8);
+    ONES_TAKE(F0, (size_t)rows * 8);
+    ONES_TAKE(F1, (size_t)rows * 8);
+    ONES_TAKE(Fall, (size_t)n * 8);
+    ONES_TAKE(pop0, (size_t)rows * ld * 4);
+    ONES_TAKE(pop1, (size_t)rows * ld * 4);
+    ONES_TAKE(Gc, (size_t)rows * 4);
+    ONES_TAKE(kmin, (size_t)jpad * 4);
+    ONES_TAKE(range, (size_t)jpad * 4);
+    ONES_TAKE(elit, e * 4);
+    ONES_TAKE(G16, (size_t)planes * jpad * 2);
+#undef ONES_TAKE
+    m.total = (at + 15) & ~(size_t)15;
+    return m;
+}
+
+template <bool ALWAYS>
+__global__ void __launch_bounds__(512, 1)
+k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_jobs, int32_t elitism, int32_t pairs,
+                 int32_t tournament, double* __restrict__ F_io, int32_t* __restrict__ G_out,
+                 int32_t* __restrict__ parents_out, int32_t* __restrict__ elites_out, Tables t, RoundKeys keys,
+                 uint64_t gen0, int32_t generations, uint32_t thr32, int32_t capacity, double penalty,
+                 int32_t rows_per_cta, int32_t gs) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ Rec s_warp[32];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int32_t C = (int32_t)cluster.num_blocks(), me = (int32_t)cluster.block_rank();
+    const int32_t planes = t.k1 + 1, jpad = t.jpad;
+    const ClusterSmem m = cluster_smem(planes, jpad, ld, rows_per_cta, elitism, n);
+    double* sX = reinterpret_cast<double*>(smem_raw + m.X);
+    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + m.G16);
+    double* sF[2] = {reinterpret_cast<double*>(smem_raw + m.F0), reinterpret_cast<double*>(smem_raw + m.F1)};
+    int32_t* sPop[2] = {reinterpret_cast<int32_t*>(smem_raw + m.pop0), reinterpret_cast<int32_t*>(smem_raw + m.pop1)};
+    int32_t* sGc = reinterpret_cast<int32_t*>(smem_raw + m.Gc);
+    int4* sKmin = reinterpret_cast<int4*>(smem_raw + m.kmin);
+    int4* sRange = reinterpret_cast<int4*>(smem_raw + m.range);
+    double* sFall = reinterpret_cast<double*>(smem_raw + m.Fall);  // every candidate's score, copied each generation
+    int32_t* sElit = reinterpret_cast<int32_t*>(smem_raw + m.elit);
+
+    const int32_t lo = me * rows_per_cta, hi = min(n, lo + rows_per_cta), mine = max(0, hi - lo);
+    const int32_t nvec = (int32_t)(ld >> 2);
+    {   // stage tables, my rows and their scores
+        const int32_t cells = planes * jpad;
+        for (int32_t i = threadIdx.x; i < cells; i += blockDim.x) {
+            sX[i] = t.X[i];
+            sG[i] = (uint16_t)t.G[i];
+        }
+        for (int32_t i = threadIdx.x; i < jpad; i += blockDim.x) {
+            reinterpret_cast<int32_t*>(sKmin)[i] = t.kmin[i];
+            reinterpret_cast<int32_t*>(sRange)[i] = t.range[i];
+        }
+        const int4* src = reinterpret_cast<const int4*>(pop_io + (int64_t)lo * ld);
+        for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) reinterpret_cast<int4*>(sPop[0])[i] = src[i];
+        for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) sF[0][i] = F_io[lo + i];
+    }
+    __syncthreads();
+    cluster.sync();  // everybody's rows and scores are staged
+
+    const uint32_t kcap = (uint32_t)t.k1;
+    const int32_t groups = (int32_t)blockDim.x / gs;
+    const int32_t gi = (int32_t)threadIdx.x / gs, gl = (int32_t)threadIdx.x % gs;
+    // child rows owned by this CTA: elite rows r < elitism, then pairs whose even child (row elitism + 2q) is mine
+    const int32_t elite_lo = min(lo, elitism), elite_hi = min(hi, elitism);
+    const int32_t first_child = max(lo, elitism);
+    const int32_t q_lo = (first_child - elitism + 1) >> 1;                    // first q with elitism + 2q >= first_child
+    const int32_t q_hi = hi > elitism ? min(pairs, (hi - elitism + 1) >> 1) : 0;  // first q with elitism + 2q >= hi
+    const int32_t n_items = (elite_hi - elite_lo) + max(0, q_hi - q_lo);
+    const int32_t trips = (n_items + groups - 1) / groups;
+
+    for (int32_t g = 0; g < generations; ++g) {
+        const int cur = g & 1, nxt = cur ^ 1;
+        const uint64_t gen = gen0 + (uint64_t)g;
+        const uint32_t gen_lo = (uint32_t)gen;
+        const uint32_t c3 = counter3(STREAM_MUT, gen), c3a = counter3(STREAM_SEL_A, gen), c3b = counter3(STREAM_SEL_B, gen);
+        // ---- every CTA takes a private copy of all scores, then finds the elites for itself ----
+        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
+            const int32_t owner = i / rows_per_cta;
+            sFall[i] = *cluster.map_shared_rank(sF[cur] + (i - owner * rows_per_cta), (unsigned int)owner);
+        }
+        __syncthreads();
+        if (elitism > 0) {
+            Rec prev;
+            prev.key = 0;
+            prev.idx = -1;
+            prev.pad = 0;
+            for (int32_t r = 0; r < elitism; ++r) {
+                Rec best = block_next_best<0>(sFall, n, 0, r > 0, prev, s_warp);
+                if (threadIdx.x == 0) {
+                    sElit[r] = best.idx;
+                    if (me == 0) elites_out[r] = best.idx;
+                }
+                prev = best;
+            }
+            __syncthreads();
+        }
+        // ---- children ----
+        for (int32_t trip = 0; trip < trips; ++trip) {
+            const int32_t item = trip * groups + gi;
+            const bool live = item < n_items;
+            const bool is_elite = live && item < elite_hi - elite_lo;
+            int32_t pa = 0, pb = 0, slot0 = 0, slot1 = 0;
+            bool has1 = false;
+            uint32_t thr = 0u;
+            if (is_elite) {
+                slot0 = elite_lo + item;
+                pa = pb = sElit[slot0];
+            } else if (live) {
+                const int32_t q = q_lo + (item - (elite_hi - elite_lo));
+                // both tournaments, every lane of the group for itself (same draws, same winner)
+                for (int which = 0; which < 2; ++which) {
+                    int32_t win = -1;
+                    double fwin = 0.0;
+                    for (int32_t t0 = 0; t0 < tournament; t0 += 4) {
+                        const uint4 w4 = philox((uint32_t)(t0 >> 2), (uint32_t)q, gen_lo, which ? c3b : c3a, keys);
+                        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (t0 + u < tournament) {
+                                const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
+                                const double f = sFall[idx];
+                                if (win < 0 || f > fwin || (f == fwin && idx < win)) {
+                                    win = idx;
+                                    fwin = f;
+                                }
+                            }
+                        }
+                    }
+                    if (which) pb = win; else pa = win;
+                }
+                slot0 = elitism + 2 * q;
+                slot1 = slot0 + 1;
+                has1 = slot1 < n;
+                thr = thr32;
+                if (gl == 0) {
+                    parents_out[2 * q] = pa;
+                    parents_out[2 * q + 1] = pb;
+                }
+            }
+            double sum0 = 0.0, sum1 = 0.0;
+            int32_t gp0 = 0, gp1 = 0;
+            if (live) {
+                const int32_t oa = pa / rows_per_cta, ob = pb / rows_per_cta;
+                const int4* A = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pa - oa * rows_per_cta) * ld, (unsigned int)oa));
+                const int4* B = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pb - ob * rows_per_cta) * ld, (unsigned int)ob));
+                const int32_t o0 = slot0 / rows_per_cta, o1 = has1 ? slot1 / rows_per_cta : o0;
+                int4* C0 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)(slot0 - o0 * rows_per_cta) * ld, (unsigned int)o0));
+                int4* C1 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)((has1 ? slot1 : slot0) - o1 * rows_per_cta) * ld, (unsigned int)o1));
+                for (int32_t v = gl; v < nvec; v += gs) {
+                    const int4 a = A[v], b = B[v];
+                    int4 c0 = a, c1 = b;
+                    if (!is_elite) {
+                        const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+                        if (ALWAYS) sibling_int4<true>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
+                        else sibling_int4<false>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
+                    }
+                    C0[v] = c0;
+                    const int32_t base = (v >> 5) * 128 + (v & 31);
+                    score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
+                    if (has1) {
+                        C1[v] = c1;
+                        score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+                    }
+                }
+            }
+            // fixed-order sum over the group's lanes (partials of absent lanes are +0)
+            for (int off = gs >> 1; off >= 1; off >>= 1) {
+                sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
+                gp0 += __shfl_xor_sync(0xFFFFFFFFu, gp0, off);
+                sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
+                gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
+            }
+            if (live && gl == 0) {
+                const int32_t o0 = slot0 / rows_per_cta;
+                const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
+                *cluster.map_shared_rank(sF[nxt] + (slot0 - o0 * rows_per_cta), (unsigned int)o0) =
+                    __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+                *cluster.map_shared_rank(sGc + (slot0 - o0 * rows_per_cta), (unsigned int)o0) = gp0;
+                if (has1) {
+                    const int32_t o1 = slot1 / rows_per_cta;
+                    const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                    *cluster.map_shared_rank(sF[nxt] + (slot1 - o1 * rows_per_cta), (unsigned int)o1) =
+                        __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                    *cluster.map_shared_rank(sGc + (slot1 - o1 * rows_per_cta), (unsigned int)o1) = gp1;
+                }
+            }
+        }
+        cluster.sync();  // all children and their scores written, also those that landed in a neighbour
+    }
+    // ---- write my rows back ----
+    const int fin = generations & 1;
+    int4* dst = reinterpret_cast<int4*>(pop_io + (int64_t)lo * ld);
+    for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) dst[i] = reinterpret_cast<const int4*>(sPop[fin])[i];
+    for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) {
+        F_io[lo + i] = sF[fin][i];
+        G_out[lo + i] = sGc[i];
+    }
+}
+
+template <bool ALWAYS>
+static cudaError_t cluster_config(ClusterShape shape, cudaStream_t s, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr) {
+    auto kern = k_evolve_cluster<ALWAYS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, shape.cluster > 8 ? 1 : 0);
+    if (e != cudaSuccess) return e;
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3((unsigned)shape.cluster, 1, 1);
+    cfg->blockDim = dim3((unsigned)shape.threads, 1, 1);
+    cfg->dynamicSmemBytes = shape.smem;
+    cfg->stream = s;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)shape.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg->attrs = attr;
+    cfg->numAttrs = 1;
+    return cudaSuccess;
+}
+
+// cluster == 0: the population does not fit the shared memory of one cluster that the device can host (or is
+// large enough for the HBM paths).  rows_per_cta >= 32 keeps every CTA busy.
+ClusterShape cluster_shape(Tables t, int64_t ld, int32_t n, int32_t elitism, int32_t pairs) {
+    ClusterShape shape{0, 0, 0, 0, 0};
+    if ((int64_t)pairs + elitism >= (int64_t)kSMs * 16) return shape;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    int gs = 1;
+    while (gs < nvec && gs < 32) gs <<= 1;
+    for (int c = 16; c >= 1; c >>= 1) {
+        const int32_t rows = (n + c - 1) / c;
+        if (c > 1 && rows < 32) continue;
+        const size_t bytes = cluster_smem(t.k1 + 1, t.jpad, ld, rows, elitism, n).total;
+        if (bytes + 2048 > (size_t)kMaxSmemPerBlock) continue;
+        ClusterShape trial{c, 512, rows, gs, bytes};
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[1];
+        int max_clusters = 0;
+        if (cluster_config<false>(trial, nullptr, &cfg, attr) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&max_clusters, k_evolve_cluster<false>, &cfg) != cudaSuccess ||
+            max_clusters < 1) {
+            cudaGetLastError();  // this size cannot be hosted: try a smaller cluster
+            continue;
+        }
+        return trial;
+    }
+    return shape;
+}
+
+template <bool ALWAYS>
+static cudaError_t launch_cluster_t(ClusterShape shape, int32_t* pop_io, int64_t ld, int32_t n, int32_t n_jobs,
+                                    int32_t elitism, int32_t pairs, int32_t tournament, double* F_io, int32_t* G_out,
+                                    int32_t* parents_out, int32_t* elites_out, Tables t, RoundKeys keys, uint64_t gen0,
+                                    int32_t generations, uint32_t thr32, int32_t capacity, double penalty,
+                                    cudaStream_t s) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cudaError_t e = cluster_config<ALWAYS>(shape, s, &cfg, attr);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, k_evolve_cluster<ALWAYS>, pop_io, ld, n, n_jobs, elitism, pairs, tournament, F_io,
+                              G_out, parents_out, elites_out, t, keys, gen0, generations, thr32, capacity, penalty,
+                              shape.rows_per_cta, (int32_t)shape.gs);
+}
+
+cudaError_t launch_evolve_cluster(ClusterShape shape, int32_t* pop_io, int64_t ld, int32_t n, int32_t n_jobs,
+                                  int32_t elitism, int32_t pairs, int32_t tournament, double* F_io, int32_t* G_out,
+                                  int32_t* parents_out, int32_t* elites_out, Tables t, RoundKeys keys, uint64_t gen0,
+                                  int32_t generations, uint32_t thr16, int32_t capacity, double penalty, cudaStream_t s) {
+    if (shape.cluster <= 0) return cudaErrorInvalidConfiguration;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    if (thr16 >= 65536u)
+        return launch_cluster_t<true>(shape, pop_io, ld, n, n_jobs, elitism, pairs, tournament, F_io, G_out, parents_out,
+                                      elites_out, t, keys, gen0, generations, thr32, capacity, penalty, s);
+    return launch_cluster_t<false>(shape, pop_io, ld, n, n_jobs, elitism, pairs, tournament, F_io, G_out, parents_out,
+                                   elites_out, t, keys, gen0, generations, thr32, capacity, penalty, s);
 }
 
 // ---------------------------------------------------------------------------------------------

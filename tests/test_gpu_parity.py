@@ -143,7 +143,8 @@ def test_randomize_parity(ones):
         _same_state(g, o)
 
 
-@pytest.mark.parametrize("name,gens,flags", [("tiny", 10, 0), ("paper", 100, 0), ("paper", 100, 2)])
+@pytest.mark.parametrize("name,gens,flags", [("tiny", 10, 0), ("paper", 100, 0), ("paper", 100, 2), ("tiny", 10, 8),
+                                             ("paper", 100, 8)])  # 0: one cluster launch, 8: launch per generation
 def test_evolve_parity_named_workloads(ones, name, gens, flags):
     w = inputs.WORKLOADS[name]()
     g, o = _pair(ones, w, flags=flags)
@@ -180,7 +181,7 @@ def test_evolve_parity_mid_sampled_generations(ones):
 @pytest.mark.parametrize("kw", [dict(elitism=0), dict(elitism=1), dict(elitism=5, tournament=1),
                                 dict(tournament=9), dict(p_mut=0.0), dict(p_mut=1.0), dict(p_mut=0.02, tournament=8),
                                 dict(penalty=0.0), dict(penalty=37.5), dict(flags=2), dict(flags=2, p_mut=1.0),
-                                dict(flags=3)])
+                                dict(flags=3), dict(flags=8), dict(flags=8, elitism=0), dict(flags=8, p_mut=1.0)])
 def test_evolve_parity_parameter_corners(ones, kw):
     w = inputs.custom(37, 48, 101, 6, seed=7, kmax=6, pinned=4, kmin_max=3)
     g, o = _pair(ones, w, **kw)
@@ -195,10 +196,11 @@ def test_evolve_parity_parameter_corners(ones, kw):
         _same_state(g, o)
 
 
-@pytest.mark.parametrize("J,N", [(1, 2), (2, 3), (5, 4), (127, 33), (129, 64), (260, 1025)])
-def test_evolve_parity_ragged_shapes(ones, J, N):
+@pytest.mark.parametrize("flags", [0, 8])
+@pytest.mark.parametrize("J,N", [(1, 2), (2, 3), (5, 4), (6, 4096), (127, 33), (129, 64), (260, 1025), (700, 2000)])
+def test_evolve_parity_ragged_shapes(ones, J, N, flags):
     w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, params=inputs.SearchParams(1, 3, 0.1, 1e3))
-    g, o = _pair(ones, w)
+    g, o = _pair(ones, w, flags=flags)
     g.randomize(1)
     o.randomize(1)
     g.evolve(4, 2 ** 40 + 17)
