@@ -402,10 +402,20 @@ __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, boo
     __syncthreads();  // s_warp may still be read from the previous round
     if (lane == 0) s_warp[warp] = best;
     __syncthreads();
-    Rec r = s_warp[0];
-    for (int w = 1; w < nwarp; ++w) {
-        const Rec o = s_warp[w];
-        if (o.idx >= 0 && (r.idx < 0 || before(o.key, o.idx, r.key, r.idx))) r = o;
+    // every warp reduces the per-warp winners again (same result everywhere, no third barrier)
+    Rec r;
+    r.key = 0ull;
+    r.idx = -1;
+    r.pad = 0;
+    if (lane < nwarp) r = s_warp[lane];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xFFFFFFFFu, r.key, off);
+        const int32_t oi = __shfl_xor_sync(0xFFFFFFFFu, r.idx, off);
+        if (oi >= 0 && (r.idx < 0 || before(ok, oi, r.key, r.idx))) {
+            r.key = ok;
+            r.idx = oi;
+        }
     }
     return r;
 }
