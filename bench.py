@@ -385,13 +385,18 @@ def main():
         evolve_bytes = 8 * J * (N - E) + 8 * J * E + 8 * ((N - E + 1) // 2) + 4 * E
         fused_bytes = evolve_bytes + 12 * N
         ach = fused_bytes / (ev_ms * 1e-3) / 1e9
-        one_launch = launches <= steps  # small shapes run the whole generation in k_generation
-        line["roofline"] = {"kernel": "k_generation" if one_launch else "k_evolve_score", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+        gens_per_launch = steps if launches < steps else 1  # the cluster path runs a whole call in one launch
+        one_launch = launches <= steps
+        kernel = "k_evolve_cluster" if launches < steps else ("k_generation" if one_launch else "k_evolve_score")
+        ach = fused_bytes * gens_per_launch / (ev_ms * 1e-3) / 1e9
+        line["roofline"] = {"kernel": kernel, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
                             "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
-                            "bytes_per_launch": fused_bytes, "ms_per_launch": ev_ms,
+                            "bytes_per_launch": fused_bytes * gens_per_launch, "ms_per_launch": ev_ms,
+                            "generations_per_launch": gens_per_launch,
                             "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
                             "note": "crossover + mutation + scoring of the children in one pass (dominant kernel of the "
-                                    "generation; k_select_stage precedes it); the unfused kernels are under 'kernels'"}
+                                    "generation); shapes that fit one cluster's shared memory are latency-bound, their "
+                                    "fraction of the HBM rate is informational; the unfused kernels are under 'kernels'"}
         line["kernels"] = {"k_select_stage": {"ms_per_launch": sel_ms}} if sel_ms else {}
         if sep is not None:
             sep_ms, sep_n = sep
