@@ -1153,12 +1153,13 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                  int32_t tournament, double* __restrict__ F_io, int32_t* __restrict__ G_out,
                  int32_t* __restrict__ parents_out, int32_t* __restrict__ elites_out, Tables t, RoundKeys keys,
                  uint64_t gen0, int32_t generations, uint32_t thr32, int32_t capacity, double penalty,
-                 int32_t rows_per_cta, int32_t gs) {
+                 int32_t rows_shift /* rows per CTA = 1 << rows_shift */, int32_t gs) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Rec s_warp[32];
     cg::cluster_group cluster = cg::this_cluster();
     const int32_t C = (int32_t)cluster.num_blocks(), me = (int32_t)cluster.block_rank();
     const int32_t planes = t.k1 + 1, jpad = t.jpad;
+    const int32_t rows_per_cta = 1 << rows_shift, rows_mask = rows_per_cta - 1;
     const ClusterSmem m = cluster_smem(planes, jpad, ld, rows_per_cta, elitism, n);
     double* sX = reinterpret_cast<double*>(smem_raw + m.X);
     uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + m.G16);
@@ -1207,8 +1208,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         const uint32_t c3 = counter3(STREAM_MUT, gen), c3a = counter3(STREAM_SEL_A, gen), c3b = counter3(STREAM_SEL_B, gen);
         // ---- every CTA takes a private copy of all scores, then finds the elites for itself ----
         for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
-            const int32_t owner = i / rows_per_cta;
-            sFall[i] = *cluster.map_shared_rank(sF[cur] + (i - owner * rows_per_cta), (unsigned int)owner);
+            sFall[i] = *cluster.map_shared_rank(sF[cur] + (i & rows_mask), (unsigned int)(i >> rows_shift));
         }
         __syncthreads();
         if (elitism > 0) {
@@ -1272,12 +1272,12 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             double sum0 = 0.0, sum1 = 0.0;
             int32_t gp0 = 0, gp1 = 0;
             if (live) {
-                const int32_t oa = pa / rows_per_cta, ob = pb / rows_per_cta;
-                const int4* A = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pa - oa * rows_per_cta) * ld, (unsigned int)oa));
-                const int4* B = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pb - ob * rows_per_cta) * ld, (unsigned int)ob));
-                const int32_t o0 = slot0 / rows_per_cta, o1 = has1 ? slot1 / rows_per_cta : o0;
-                int4* C0 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)(slot0 - o0 * rows_per_cta) * ld, (unsigned int)o0));
-                int4* C1 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)((has1 ? slot1 : slot0) - o1 * rows_per_cta) * ld, (unsigned int)o1));
+                const int32_t oa = pa >> rows_shift, ob = pb >> rows_shift;
+                const int4* A = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pa & rows_mask) * ld, (unsigned int)oa));
+                const int4* B = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pb & rows_mask) * ld, (unsigned int)ob));
+                const int32_t o0 = slot0 >> rows_shift, o1 = has1 ? slot1 >> rows_shift : o0;
+                int4* C0 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)(slot0 & rows_mask) * ld, (unsigned int)o0));
+                int4* C1 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)((has1 ? slot1 : slot0) & rows_mask) * ld, (unsigned int)o1));
                 for (int32_t v = gl; v < nvec; v += gs) {
                     const int4 a = A[v], b = B[v];
                     int4 c0 = a, c1 = b;
@@ -1303,17 +1303,17 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                 gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
             }
             if (live && gl == 0) {
-                const int32_t o0 = slot0 / rows_per_cta;
+                const int32_t o0 = slot0 >> rows_shift;
                 const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
-                *cluster.map_shared_rank(sF[nxt] + (slot0 - o0 * rows_per_cta), (unsigned int)o0) =
+                *cluster.map_shared_rank(sF[nxt] + (slot0 & rows_mask), (unsigned int)o0) =
                     __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
-                *cluster.map_shared_rank(sGc + (slot0 - o0 * rows_per_cta), (unsigned int)o0) = gp0;
+                *cluster.map_shared_rank(sGc + (slot0 & rows_mask), (unsigned int)o0) = gp0;
                 if (has1) {
-                    const int32_t o1 = slot1 / rows_per_cta;
+                    const int32_t o1 = slot1 >> rows_shift;
                     const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
-                    *cluster.map_shared_rank(sF[nxt] + (slot1 - o1 * rows_per_cta), (unsigned int)o1) =
+                    *cluster.map_shared_rank(sF[nxt] + (slot1 & rows_mask), (unsigned int)o1) =
                         __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
-                    *cluster.map_shared_rank(sGc + (slot1 - o1 * rows_per_cta), (unsigned int)o1) = gp1;
+                    *cluster.map_shared_rank(sGc + (slot1 & rows_mask), (unsigned int)o1) = gp1;
                 }
             }
         }
@@ -1359,8 +1359,9 @@ ClusterShape cluster_shape(Tables t, int64_t ld, int32_t n, int32_t elitism, int
     int gs = 1;
     while (gs < nvec && gs < 32) gs <<= 1;
     for (int c = 16; c >= 1; c >>= 1) {
-        const int32_t rows = (n + c - 1) / c;
-        if (c > 1 && rows < 32) continue;
+        int32_t rows = 1;  // rows per CTA: a power of two (owners and offsets by shift and mask)
+        while (rows < (n + c - 1) / c) rows <<= 1;
+        if (c > 1 && (rows < 32 || (int64_t)rows * (c - 1) >= n)) continue;  // keep every CTA busy
         const size_t bytes = cluster_smem(t.k1 + 1, t.jpad, ld, rows, elitism, n).total;
         if (bytes + 2048 > (size_t)kMaxSmemPerBlock) continue;
         ClusterShape trial{c, 512, rows, gs, bytes};
@@ -1390,7 +1391,7 @@ static cudaError_t launch_cluster_t(ClusterShape shape, int32_t* pop_io, int64_t
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, k_evolve_cluster<ALWAYS>, pop_io, ld, n, n_jobs, elitism, pairs, tournament, F_io,
                               G_out, parents_out, elites_out, t, keys, gen0, generations, thr32, capacity, penalty,
-                              shape.rows_per_cta, (int32_t)shape.gs);
+                              (int32_t)(31 - __builtin_clz((unsigned)shape.rows_per_cta)), (int32_t)shape.gs);
 }
 
 cudaError_t launch_evolve_cluster(ClusterShape shape, int32_t* pop_io, int64_t ld, int32_t n, int32_t n_jobs,
