@@ -18,6 +18,7 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 
 FLAG_SRUF = 1
 FLAG_TRUNCATION = 4
+FLAG_PER_GPU = 16
 STREAM_INIT, STREAM_SEL_A, STREAM_SEL_B, STREAM_MUT = 0, 1, 2, 3
 
 JOB_DTYPE = np.dtype(
@@ -68,6 +69,8 @@ def _configure(L: C.CDLL) -> C.CDLL:
     L.oracle_tournament.restype = i32
     L.oracle_top.argtypes = [vp, i32, i32, vp]
     L.oracle_keep_best.argtypes = [vp, i32, i32, vp]
+    L.oracle_fitness_per_gpu.argtypes = [vp, i32, i32, u32, vp, vp, vp, vp]
+    L.oracle_reorder.argtypes = [vp, i32, i32]
     L.oracle_thr16.argtypes = [dbl]
     L.oracle_thr16.restype = u32
     L.oracle_create.argtypes = [vp, vp, i32, i32, i32, vp]
@@ -197,6 +200,24 @@ def top(F, e: int) -> np.ndarray:
     return idx[:e]
 
 
+def fitness_per_gpu(jobs, slots, flags: int = 0):
+    """(F, GPUs used, per-job exponents) of one per-GPU genome."""
+    a = _jobs_arr(jobs)
+    sl = np.ascontiguousarray(slots, dtype=np.int32)
+    F = C.c_double()
+    G = C.c_int32()
+    ks = np.zeros(a.shape[0], dtype=np.int32)
+    _check(lib().oracle_fitness_per_gpu(_ptr(a), a.shape[0], sl.shape[0], flags, _ptr(sl), C.byref(F), C.byref(G),
+                                        _ptr(ks)), "fitness_per_gpu")
+    return F.value, G.value, ks
+
+
+def reorder(slots, n_jobs: int) -> np.ndarray:
+    sl = np.array(slots, dtype=np.int32)
+    _check(lib().oracle_reorder(_ptr(sl), sl.shape[0], n_jobs), "reorder")
+    return sl
+
+
 def keep_best(F, k: int) -> np.ndarray:
     f = np.ascontiguousarray(F, dtype=np.float64)
     idx = np.zeros(max(k, 1), dtype=np.int32)
@@ -220,6 +241,7 @@ class Search:
         self.J = int(self.jobs.shape[0])
         self.N = int(pop)
         self.E = int(elitism)
+        self.W = int(capacity) if flags & FLAG_PER_GPU else self.J  # genes per candidate
         prm = _Params(elitism, tournament, p_mut, penalty, flags)
         rc = lib().oracle_create(C.byref(self._h), _ptr(self.jobs), self.J, capacity, pop, C.byref(prm))
         if rc != 0:
@@ -242,12 +264,12 @@ class Search:
 
     def set_population(self, genomes: np.ndarray):
         g = np.ascontiguousarray(genomes, dtype=np.int32)
-        assert g.shape[0] == self.N and g.shape[1] >= self.J
+        assert g.shape[0] == self.N and g.shape[1] >= self.W
         _check(lib().oracle_set_population(self._h, _ptr(g), g.shape[1]), "set_population")
 
     def get_population(self) -> np.ndarray:
-        g = np.zeros((self.N, self.J), dtype=np.int32)
-        _check(lib().oracle_get_population(self._h, _ptr(g), self.J), "get_population")
+        g = np.zeros((self.N, self.W), dtype=np.int32)
+        _check(lib().oracle_get_population(self._h, _ptr(g), self.W), "get_population")
         return g
 
     def evaluate(self, genomes: np.ndarray | None = None):

@@ -241,10 +241,66 @@ int oracle_repair(const oracle_job* jobs, int32_t n_jobs, int32_t capacity, int3
 }
 
 /* ------------------------------------------------------------------------- */
+/* Per-GPU genome (the paper's own encoding) and the reorder operation          */
+/* ------------------------------------------------------------------------- */
+int oracle_fitness_per_gpu(const oracle_job* jobs, int32_t n_jobs, int32_t n_gpus, uint32_t flags,
+                           const int32_t* slots, double* F, int32_t* gpus_used, int32_t* exponents) {
+    if (!jobs || !slots || !F) return ORACLE_ERR_NULL;
+    int32_t* count = (int32_t*)calloc((size_t)n_jobs, sizeof(int32_t));
+    if (!count) return ORACLE_ERR_NOMEM;
+    for (int32_t i = 0; i < n_gpus; ++i)
+        if (slots[i] >= 0 && slots[i] < n_jobs) count[slots[i]] += 1; /* c_j = sum_i min(1, b_j^i) */
+    double part[32];
+    for (int l = 0; l < 32; ++l) part[l] = 0.0;
+    int64_t used = 0;
+    for (int32_t j = 0; j < n_jobs; ++j) {
+        int32_t kbest = -1;
+        for (int32_t k = jobs[j].kmin; k <= jobs[j].kmax; ++k) {
+            double X; int32_t g;
+            oracle_model(&jobs[j], k, &X, &g);
+            if (g <= count[j]) kbest = k;
+        }
+        double term = 0.0;
+        int32_t g = 0;
+        if (kbest >= 0) oracle_term(&jobs[j], kbest, flags, &term, &g);
+        part[(j >> 2) & 31] = part[(j >> 2) & 31] + term; /* same summation order as oracle_fitness */
+        used += g;
+        if (exponents) exponents[j] = kbest;
+    }
+    for (int off = 16; off >= 1; off >>= 1)
+        for (int l = 0; l < off; ++l) part[l] = part[l] + part[l + off];
+    *F = part[0];
+    if (gpus_used) *gpus_used = (int32_t)used;
+    free(count);
+    return ORACLE_OK;
+}
+
+int oracle_reorder(int32_t* slots, int32_t n_gpus, int32_t n_jobs) {
+    if (!slots) return ORACLE_ERR_NULL;
+    int32_t* out = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_gpus > 0 ? n_gpus : 1));
+    char* done = (char*)calloc((size_t)(n_jobs > 0 ? n_jobs : 1), 1);
+    if (!out || !done) { free(out); free(done); return ORACLE_ERR_NOMEM; }
+    int32_t at = 0;
+    for (int32_t i = 0; i < n_gpus; ++i) { /* jobs in the order of their first occurrence */
+        int32_t j = slots[i];
+        if (j < 0 || j >= n_jobs || done[j]) continue;
+        done[j] = 1;
+        for (int32_t i2 = i; i2 < n_gpus; ++i2)
+            if (slots[i2] == j) out[at++] = j;
+    }
+    while (at < n_gpus) out[at++] = -1; /* idle GPUs last */
+    memcpy(slots, out, sizeof(int32_t) * (size_t)n_gpus);
+    free(out);
+    free(done);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------- */
 /* The search                                                                  */
 /* ------------------------------------------------------------------------- */
 struct oracle_ctx {
     int32_t J, cap, N, pairs;
+    int32_t W; /* genes per candidate: one per job, or one per GPU with ORACLE_FLAG_PER_GPU */
     oracle_params prm;
     oracle_job* jobs;
     int32_t* pop;   /* N x J */
@@ -257,7 +313,12 @@ struct oracle_ctx {
     int32_t* elites;  /* E of the last generation */
 };
 
+/* admissible values of gene j: the job's exponents, or (per-GPU genome) any job id */
+static int32_t gene_lo(const oracle_ctx* c, int32_t j) { return (c->prm.flags & ORACLE_FLAG_PER_GPU) ? 0 : c->jobs[j].kmin; }
+static int32_t gene_hi(const oracle_ctx* c, int32_t j) { return (c->prm.flags & ORACLE_FLAG_PER_GPU) ? c->J - 1 : c->jobs[j].kmax; }
+
 static int check_params(const oracle_params* p, int32_t pop) {
+    if ((p->flags & ORACLE_FLAG_PER_GPU) && (p->flags & ORACLE_FLAG_TRUNCATION)) return ORACLE_ERR_BAD_PARAM;
     if (p->elitism < 0 || p->tournament < 1) return ORACLE_ERR_BAD_PARAM;
     if (pop < p->elitism + 1) return ORACLE_ERR_BAD_PARAM;
     if (!(p->p_mut >= 0.0 && p->p_mut <= 1.0)) return ORACLE_ERR_BAD_PARAM;
@@ -285,8 +346,9 @@ int oracle_create(oracle_ctx** out, const oracle_job* jobs, int32_t n_jobs, int3
     oracle_ctx* c = (oracle_ctx*)calloc(1, sizeof *c);
     if (!c) return ORACLE_ERR_NOMEM;
     c->J = n_jobs; c->cap = capacity; c->N = pop; c->prm = p;
+    c->W = (p.flags & ORACLE_FLAG_PER_GPU) ? capacity : n_jobs;
     c->pairs = (p.flags & ORACLE_FLAG_TRUNCATION) ? pop : (pop - p.elitism + 1) / 2;
-    size_t cells = (size_t)pop * (size_t)n_jobs;
+    size_t cells = (size_t)pop * (size_t)c->W;
     c->jobs = (oracle_job*)malloc(sizeof(oracle_job) * (size_t)n_jobs);
     c->pop = (int32_t*)malloc(sizeof(int32_t) * cells);
     c->next = (int32_t*)malloc(sizeof(int32_t) * cells);
@@ -301,7 +363,8 @@ int oracle_create(oracle_ctx** out, const oracle_job* jobs, int32_t n_jobs, int3
     memcpy(c->jobs, jobs, sizeof(oracle_job) * (size_t)n_jobs);
     /* initial population G_0 of simple solutions: every job at its smallest batch */
     for (int32_t i = 0; i < pop; ++i)
-        for (int32_t j = 0; j < n_jobs; ++j) c->pop[(size_t)i * n_jobs + j] = jobs[j].kmin;
+        for (int32_t j = 0; j < c->W; ++j)
+            c->pop[(size_t)i * c->W + j] = (p.flags & ORACLE_FLAG_PER_GPU) ? -1 : jobs[j].kmin; /* per GPU: all idle */
     c->f_valid = 0;
     c->gen_abs = 0;
     *out = c;
@@ -316,12 +379,11 @@ int oracle_destroy(oracle_ctx* c) {
 int oracle_randomize(oracle_ctx* c, uint64_t seed) {
     if (!c) return ORACLE_ERR_NULL;
     for (int32_t i = 0; i < c->N; ++i)
-        for (int32_t j = 0; j < c->J; ++j) {
-            const oracle_job* q = &c->jobs[j];
-            int32_t k = q->kmin; /* candidate 0 stays the all-minimum schedule */
+        for (int32_t j = 0; j < c->W; ++j) {
+            int32_t k = gene_lo(c, j); /* candidate 0 stays the all-minimum schedule */
             if (i > 0) k = draw_gene(oracle_word(seed, 0, (uint32_t)i, (uint32_t)j, ORACLE_STREAM_INIT),
-                                     q->kmin, q->kmax);
-            c->pop[(size_t)i * c->J + j] = k;
+                                     gene_lo(c, j), gene_hi(c, j));
+            c->pop[(size_t)i * c->W + j] = k;
         }
     c->f_valid = 0;
     return ORACLE_OK;
@@ -329,25 +391,30 @@ int oracle_randomize(oracle_ctx* c, uint64_t seed) {
 
 int oracle_set_population(oracle_ctx* c, const int32_t* genomes, int64_t ld) {
     if (!c || !genomes) return ORACLE_ERR_NULL;
-    if (ld < c->J) return ORACLE_ERR_BAD_PARAM;
+    if (ld < c->W) return ORACLE_ERR_BAD_PARAM;
     for (int32_t i = 0; i < c->N; ++i)
-        memcpy(&c->pop[(size_t)i * c->J], &genomes[(size_t)i * (size_t)ld], sizeof(int32_t) * (size_t)c->J);
+        memcpy(&c->pop[(size_t)i * c->W], &genomes[(size_t)i * (size_t)ld], sizeof(int32_t) * (size_t)c->W);
     c->f_valid = 0;
     return ORACLE_OK;
 }
 
 int oracle_get_population(oracle_ctx* c, int32_t* genomes, int64_t ld) {
     if (!c || !genomes) return ORACLE_ERR_NULL;
-    if (ld < c->J) return ORACLE_ERR_BAD_PARAM;
+    if (ld < c->W) return ORACLE_ERR_BAD_PARAM;
     for (int32_t i = 0; i < c->N; ++i)
-        memcpy(&genomes[(size_t)i * (size_t)ld], &c->pop[(size_t)i * c->J], sizeof(int32_t) * (size_t)c->J);
+        memcpy(&genomes[(size_t)i * (size_t)ld], &c->pop[(size_t)i * c->W], sizeof(int32_t) * (size_t)c->W);
     return ORACLE_OK;
 }
 
+static void score_row(const oracle_ctx* c, const int32_t* row, double* F, int32_t* G) {
+    if (c->prm.flags & ORACLE_FLAG_PER_GPU)
+        oracle_fitness_per_gpu(c->jobs, c->J, c->cap, c->prm.flags, row, F, G, NULL);
+    else
+        oracle_fitness(c->jobs, c->J, c->cap, c->prm.penalty, c->prm.flags, row, F, G);
+}
+
 static void score_population(oracle_ctx* c) {
-    for (int32_t i = 0; i < c->N; ++i)
-        oracle_fitness(c->jobs, c->J, c->cap, c->prm.penalty, c->prm.flags,
-                       &c->pop[(size_t)i * c->J], &c->F[i], &c->G[i]);
+    for (int32_t i = 0; i < c->N; ++i) score_row(c, &c->pop[(size_t)i * c->W], &c->F[i], &c->G[i]);
     c->f_valid = 1;
 }
 
@@ -360,10 +427,12 @@ int oracle_evaluate(oracle_ctx* c, const int32_t* genomes, int64_t ld, int32_t n
         if (gpus) memcpy(gpus, c->G, sizeof(int32_t) * (size_t)c->N);
         return ORACLE_OK;
     }
-    if (ld < c->J || n < 0) return ORACLE_ERR_BAD_PARAM;
-    for (int32_t i = 0; i < n; ++i)
-        oracle_fitness(c->jobs, c->J, c->cap, c->prm.penalty, c->prm.flags,
-                       &genomes[(size_t)i * (size_t)ld], &fitness[i], gpus ? &gpus[i] : NULL);
+    if (ld < c->W || n < 0) return ORACLE_ERR_BAD_PARAM;
+    for (int32_t i = 0; i < n; ++i) {
+        int32_t g;
+        score_row(c, &genomes[(size_t)i * (size_t)ld], &fitness[i], &g);
+        if (gpus) gpus[i] = g;
+    }
     return ORACLE_OK;
 }
 
@@ -475,7 +544,7 @@ int oracle_evolve(oracle_ctx* c, int32_t generations, uint64_t seed) {
         }
         return ORACLE_OK;
     }
-    const int32_t N = c->N, J = c->J, E = c->prm.elitism, T = c->prm.tournament;
+    const int32_t N = c->N, J = c->W /* genes per candidate */, E = c->prm.elitism, T = c->prm.tournament;
     const uint32_t thr = oracle_thr16(c->prm.p_mut);
     if (!c->f_valid) score_population(c);
     for (int32_t it = 0; it < generations; ++it) {
@@ -494,19 +563,21 @@ int oracle_evolve(oracle_ctx* c, int32_t generations, uint64_t seed) {
             const int32_t* A = &c->pop[(size_t)pa * J];
             const int32_t* B = &c->pop[(size_t)pb * J];
             for (int32_t j = 0; j < J; ++j) {
-                const oracle_job* jb = &c->jobs[j];
+                const int32_t lo = gene_lo(c, j), hi = gene_hi(c, j);
                 uint32_t W = oracle_word(seed, gen, (uint32_t)slot0, (uint32_t)j, ORACLE_STREAM_MUT);
                 int flip = (int)(W & 1u); /* which child inherits the first parent's gene */
                 int32_t child0 = flip ? B[j] : A[j];
                 int32_t child1 = flip ? A[j] : B[j];
-                if ((W & 0xFFFFu) < thr) child0 = draw_gene(even_fraction(W), jb->kmin, jb->kmax);
+                if ((W & 0xFFFFu) < thr) child0 = draw_gene(even_fraction(W), lo, hi);
                 c->next[(size_t)slot0 * J + j] = child0;
                 if (slot1 < N) {
-                    if ((W >> 16) < thr) child1 = draw_gene(odd_fraction(W), jb->kmin, jb->kmax);
+                    if ((W >> 16) < thr) child1 = draw_gene(odd_fraction(W), lo, hi);
                     c->next[(size_t)slot1 * J + j] = child1;
                 }
             }
         }
+        if (c->prm.flags & ORACLE_FLAG_PER_GPU) /* "Reorder": pack each job's workers, every new candidate */
+            for (int32_t i = 0; i < N; ++i) oracle_reorder(&c->next[(size_t)i * J], J, c->J);
         int32_t* tmp = c->pop; c->pop = c->next; c->next = tmp;
         c->gen_abs = gen + 1;
         score_population(c);
@@ -522,14 +593,19 @@ int oracle_best(oracle_ctx* c, int repair, int32_t* genome, int32_t* gpus_per_jo
     oracle_top(c->F, c->N, 1, &best);
     int32_t* row = (int32_t*)malloc(sizeof(int32_t) * (size_t)c->J);
     if (!row) return ORACLE_ERR_NOMEM;
-    memcpy(row, &c->pop[(size_t)best * c->J], sizeof(int32_t) * (size_t)c->J);
     int rc = ORACLE_OK;
     double F = c->F[best];
     int32_t G = c->G[best];
-    if (repair) {
-        rc = oracle_repair(c->jobs, c->J, c->cap, row);
-        /* score of the repaired schedule: no penalty is left when it fits */
-        oracle_fitness(c->jobs, c->J, c->cap, c->prm.penalty, c->prm.flags, row, &F, &G);
+    if (c->prm.flags & ORACLE_FLAG_PER_GPU) {
+        /* the schedule as per-job exponents: what each job can run on the GPUs it holds; always fits */
+        oracle_fitness_per_gpu(c->jobs, c->J, c->cap, c->prm.flags, &c->pop[(size_t)best * c->W], &F, &G, row);
+    } else {
+        memcpy(row, &c->pop[(size_t)best * c->J], sizeof(int32_t) * (size_t)c->J);
+        if (repair) {
+            rc = oracle_repair(c->jobs, c->J, c->cap, row);
+            /* score of the repaired schedule: no penalty is left when it fits */
+            oracle_fitness(c->jobs, c->J, c->cap, c->prm.penalty, c->prm.flags, row, &F, &G);
+        }
     }
     for (int32_t j = 0; j < c->J; ++j) {
         double X; int32_t g;
@@ -548,6 +624,7 @@ int oracle_best(oracle_ctx* c, int repair, int32_t* genome, int32_t* gpus_per_jo
 int oracle_update_jobs(oracle_ctx* c, const oracle_job* jobs, int32_t n_jobs, const int32_t* remap,
                        int32_t capacity) {
     if (!c || !jobs || !remap) return ORACLE_ERR_NULL;
+    if (c->prm.flags & ORACLE_FLAG_PER_GPU) return ORACLE_ERR_BAD_PARAM; /* job ids would need relabelling */
     int rc = oracle_validate_jobs(jobs, n_jobs);
     if (rc) return rc;
     if (capacity <= 0) return ORACLE_ERR_BAD_PARAM;
@@ -573,7 +650,7 @@ int oracle_update_jobs(oracle_ctx* c, const oracle_job* jobs, int32_t n_jobs, co
         }
     free(c->pop); free(c->next); free(c->jobs);
     c->pop = np; c->next = nn; c->jobs = nj;
-    c->J = n_jobs; c->cap = capacity;
+    c->J = n_jobs; c->W = n_jobs; c->cap = capacity;
     c->f_valid = 0;
     return ORACLE_OK;
 }

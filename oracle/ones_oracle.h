@@ -42,6 +42,9 @@ typedef struct {
 /* bit 2 (value 2) only selects a launch sequence in the CUDA library; it means nothing here */
 #define ORACLE_FLAG_TRUNCATION 4u /* the paper's selection: best K of K originals + 2K crossover children + K mutants */
 
+/* bit 8 means nothing here either (launch sequence) */
+#define ORACLE_FLAG_PER_GPU 16u /* the paper's own genome: one slot per GPU holding a job id (Eq. 1-2, Fig. 1) */
+
 enum {
     ORACLE_OK = 0,
     ORACLE_ERR_NULL = -1,
@@ -76,6 +79,15 @@ int32_t oracle_tournament(const double* F, int32_t n, int32_t tournament, uint64
                           uint64_t gen_abs, uint32_t q, uint32_t stream);
 /* indices of the e best candidates (F descending, index ascending) */
 int oracle_top(const double* F, int32_t n, int32_t e, int32_t* idx);
+/* per-GPU genome: `slots` holds one job id per GPU (anything outside [0, n_jobs) = idle).  Job j holds
+ * c_j = the number of its slots (Eq. 2) and runs at the largest admissible batch whose GPU need fits:
+ * the largest k in [kmin_j, kmax_j] with ceil(b0 << k / max_per_gpu) <= c_j; with none it waits.
+ * exponents (nullable) receives that k per job, or -1. */
+int oracle_fitness_per_gpu(const oracle_job* jobs, int32_t n_jobs, int32_t n_gpus, uint32_t flags,
+                           const int32_t* slots, double* F, int32_t* gpus_used, int32_t* exponents);
+/* "Reorder": the workers of a job become neighbours, jobs in the order of their first occurrence,
+ * idle GPUs last */
+int oracle_reorder(int32_t* slots, int32_t n_gpus, int32_t n_jobs);
 /* the k best of n scores, as ascending indices (truncation selection, order preserved) */
 int oracle_keep_best(const double* F, int32_t n, int32_t k, int32_t* kept);
 /* mutation threshold on the 16-bit decision field for probability p */

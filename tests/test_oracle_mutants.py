@@ -16,6 +16,7 @@ import test_oracle_model as M
 import test_oracle_rng as R
 import test_oracle_search as S
 import test_oracle_truncation as T
+import test_oracle_per_gpu as P
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "ones_oracle.c")
 
@@ -79,6 +80,21 @@ CASES = [
      [S.test_update_jobs_remaps_columns]),
     ("truncation keeps the worst", "for (int32_t r = 0; r < k; ++r) keep[order[r]] = 1;", "for (int32_t r = 0; r < k; ++r) keep[order[n - 1 - r]] = 1;",
      [T.test_keep_best_against_sorted]),
+    ("per-GPU: the smallest batch that fits instead of the largest", "if (g <= count[j]) kbest = k;", "if (g <= count[j] && kbest < 0) kbest = k;",
+     [P.test_fitness_counts_gpus_and_picks_the_largest_batch_that_fits]),
+    ("per-GPU: a job may use more GPUs than it holds", "if (g <= count[j]) kbest = k;", "if (g <= count[j] + 1) kbest = k;",
+     [P.test_fitness_counts_gpus_and_picks_the_largest_batch_that_fits]),
+    ("per-GPU: lower limit ignored", "for (int32_t k = jobs[j].kmin; k <= jobs[j].kmax; ++k) {\n            double X; int32_t g;\n            oracle_model(&jobs[j], k, &X, &g);\n            if (g <= count[j]) kbest = k;",
+     "for (int32_t k = 0; k <= jobs[j].kmax; ++k) {\n            double X; int32_t g;\n            oracle_model(&jobs[j], k, &X, &g);\n            if (g <= count[j]) kbest = k;",
+     [P.test_fitness_counts_gpus_and_picks_the_largest_batch_that_fits]),
+    ("reorder: idle GPUs first", "    int32_t at = 0;\n    for (int32_t i = 0; i < n_gpus; ++i) { /* jobs in the order of their first occurrence */",
+     "    int32_t at = 0;\n    for (int32_t i = 0; i < n_gpus; ++i) if (slots[i] < 0 || slots[i] >= n_jobs) out[at++] = -1;\n    for (int32_t i = 0; i < n_gpus; ++i) { /* jobs in the order of their first occurrence */",
+     [P.test_reorder_examples]),
+    ("reorder: jobs by id, not by first occurrence", "for (int32_t i = 0; i < n_gpus; ++i) { /* jobs in the order of their first occurrence */\n        int32_t j = slots[i];",
+     "for (int32_t i = 0; i < n_gpus; ++i) { /* jobs in the order of their first occurrence */\n        int32_t j = i < n_jobs ? i : -1;",
+     [P.test_reorder_examples]),
+    ("per-GPU search skips the reorder", "for (int32_t i = 0; i < N; ++i) oracle_reorder(&c->next[(size_t)i * J], J, c->J);", "(void)0;",
+     [P.test_search_on_the_per_gpu_genome]),
     ("mutants take the parents' stream", "(uint32_t)m, (uint32_t)j, ORACLE_STREAM_MUTANT);", "(uint32_t)m, (uint32_t)j, ORACLE_STREAM_MUT);",
      [T.test_generation_is_best_k_of_originals_children_and_mutants]),
 ]
