@@ -229,8 +229,9 @@ def main():
     ap.add_argument("--no-kernel-events", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling a smaller case)")
-    ap.add_argument("--scheme", default="tournament", choices=["tournament", "truncation"],
-                    help="truncation = the paper's best-K-of-4K selection (ONES_FLAG_TRUNCATION)")
+    ap.add_argument("--scheme", default="tournament", choices=["tournament", "truncation", "per_gpu"],
+                    help="truncation = the paper's best-K-of-4K selection (ONES_FLAG_TRUNCATION); per_gpu = the "
+                         "paper's one-slot-per-GPU genome with the reorder operation (ONES_FLAG_PER_GPU)")
     args = ap.parse_args()
     if args.workload == "online":
         if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
@@ -240,9 +241,10 @@ def main():
     if args.pop:
         import dataclasses
         w = dataclasses.replace(w, pop=args.pop)
-    if args.scheme == "truncation":
+    if args.scheme != "tournament":
         import dataclasses
-        w = dataclasses.replace(w, params=dataclasses.replace(w.params, flags=w.params.flags | 4))
+        bit = 4 if args.scheme == "truncation" else 16
+        w = dataclasses.replace(w, params=dataclasses.replace(w.params, flags=w.params.flags | bit))
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -296,7 +298,7 @@ def main():
 
     # ---- end to end: every step uploads the job table and reads the best schedule back ----
     J, N, E = w.n_jobs, w.pop, w.params.elitism
-    e2e_steps = 0 if args.no_e2e else min(steps, 100)
+    e2e_steps = 0 if (args.no_e2e or args.scheme == "per_gpu") else min(steps, 100)
     identity = np.arange(J, dtype=np.int32)
     jobs_pinned = torch.from_numpy(w.jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
     jobs_host = jobs_pinned.numpy().view(inputs.JOB_DTYPE)
@@ -361,6 +363,22 @@ def main():
                 "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs)",
                 "best_fitness": out["fitness"]},
     }
+    if args.scheme == "per_gpu":
+        Wg = w.capacity
+        line["config"]["scheme"] = f"per-GPU genome: {Wg} slots per candidate, reorder after crossover and mutation"
+        if stage_n.get("evolve"):
+            peak, peak_kind = measured_peak()
+            rows = {"k_evolve": ("evolve", 8 * Wg * N),
+                    "k_per_gpu<reorder, score>": ("fitness", N * (8 * Wg + 12)),
+                    "k_select_stage": ("select", 8 * N)}
+            line["kernels"] = {}
+            for name, (stage, nbytes) in rows.items():
+                t_ms = stage_ms[stage] / stage_n[stage]
+                a = nbytes / (t_ms * 1e-3) / 1e9
+                line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
+                                         "bytes_per_generation": nbytes, "ms_per_generation": t_ms}
+            dom = max(line["kernels"].items(), key=lambda kv: kv[1]["ms_per_generation"])
+            line["roofline"] = dict(dom[1], kernel=dom[0], peak_kind=f"of {peak_kind}", traffic=None)
     if args.scheme == "truncation":
         line["config"]["scheme"] = "truncation: pool of 4N rows, 3N new candidates scored per generation"
         line["new_candidates_per_s"] = 3 * line["value"]

@@ -86,6 +86,19 @@ typedef struct {
  * launch-per-generation sequence instead (same results). */
 #define ONES_FLAG_NO_CLUSTER 8u
 
+/* The paper's own genome (Eq. 1-2, Fig. 1): a candidate is one int32 per GPU of the cluster holding the
+ * id of the job that runs there (anything outside [0, n_jobs) = idle), so genome tables are
+ * int32[n][ld] with ld >= capacity.  Job j holds c_j = the number of its GPUs and runs at the largest
+ * exponent in [kmin_j, kmax_j] whose GPU need fits into c_j; with none it waits.  The score is the sum
+ * over jobs as before (no penalty: a candidate cannot exceed the cluster).  Crossover acts per GPU,
+ * mutation puts a uniformly drawn job on a GPU with rate p_mut, and every new candidate goes through
+ * the paper's "Reorder" (the workers of a job become neighbours, jobs in the order of their first
+ * occurrence, idle GPUs last).  ones_create starts from an idle cluster.  ones_best returns the best
+ * candidate as per-job exponents (h_genome[n_jobs], -1 = waits); the per-GPU rows come from
+ * ones_get_population.  ones_update_jobs is not available; not combinable with ONES_FLAG_TRUNCATION.
+ * Size the workspace with ones_workspace_bytes_per_gpu. */
+#define ONES_FLAG_PER_GPU 16u
+
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
 #define ONES_MAX_ELITES 256   /* elitism <= 256 */
 
@@ -107,6 +120,8 @@ enum {
 size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop);
 /* The same for a handle created with `flags` (ONES_FLAG_TRUNCATION needs room for its candidate pool). */
 size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flags);
+/* The same for a handle with ONES_FLAG_PER_GPU (rows hold `capacity` genes). */
+size_t ones_workspace_bytes_per_gpu(int32_t n_jobs, int32_t pop, int32_t capacity);
 
 /* Create a search over `n_jobs` jobs on a cluster of `capacity` GPUs with a
  * population of `pop` candidates (Section 3.2.2 "Initialization": the population

@@ -308,6 +308,7 @@ class Search:
         _check(lib().oracle_update_jobs(self._h, _ptr(a), a.shape[0], _ptr(r), capacity), "update_jobs")
         self.jobs = a
         self.J = int(a.shape[0])
+        self.W = self.J
 
     def last_parents(self):
         pairs = int(lib().oracle_pairs(self._h))

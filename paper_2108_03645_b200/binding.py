@@ -20,6 +20,7 @@ FLAG_SRUF = 1
 FLAG_UNFUSED = 2
 FLAG_TRUNCATION = 4
 FLAG_NO_CLUSTER = 8
+FLAG_PER_GPU = 16
 MAX_ELITES = 256
 
 ERRORS = {0: "ONES_OK", -1: "ONES_ERR_NULL", -2: "ONES_ERR_BAD_JOB", -3: "ONES_ERR_BAD_PARAM",
@@ -44,6 +45,7 @@ _lib = None
 _SIGNATURES = {
     "ones_workspace_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
     "ones_workspace_bytes_flags": (C.c_size_t, [C.c_int32, C.c_int32, C.c_uint32]),
+    "ones_workspace_bytes_per_gpu": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
     "ones_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                               C.c_size_t, C.c_void_p]),
     "ones_destroy": (C.c_int, [C.c_void_p]),
@@ -149,7 +151,11 @@ class Search:
         self.J = int(jobs.shape[0])
         self.capacity = int(capacity)
         nmax = max(self.J, int(n_jobs_max or 0))
-        nbytes = workspace_bytes(nmax, pop, p.flags)
+        self.W = int(capacity) if p.flags & FLAG_PER_GPU else self.J  # genes per candidate
+        if p.flags & FLAG_PER_GPU:
+            nbytes = int(lib().ones_workspace_bytes_per_gpu(self.J, pop, capacity))
+        else:
+            nbytes = workspace_bytes(nmax, pop, p.flags)
         if nbytes == 0:
             raise OnesError(-3, "ones_workspace_bytes")
         self.device = torch.device("cuda", torch.cuda.current_device())
@@ -196,7 +202,7 @@ class Search:
         self._check(rc, "ones_set_population")
 
     def get_population(self, on_device: bool = False, ld: int | None = None):
-        ld = self.J if ld is None else ld
+        ld = self.W if ld is None else ld
         if on_device:
             out = torch.zeros((self.N, ld), dtype=torch.int32, device=self.device)
             rc = lib().ones_get_population(self._h, _t_ptr(out), ld, 1)
@@ -245,6 +251,7 @@ class Search:
         self._check(lib().ones_update_jobs(self._h, _np_ptr(jobs), jobs.shape[0], _np_ptr(r), capacity),
                     "ones_update_jobs")
         self.J = int(jobs.shape[0])
+        self.W = self.J
         self.capacity = int(capacity)
 
     # -- inspection ---------------------------------------------------------------

@@ -26,11 +26,11 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, G1, trunc, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
         status, total;
 };
 
-Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
+Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus = 0 /* > 0: per-GPU genome */) {
     Layout L;
     size_t at = 0;
     auto take = [&](size_t bytes) {
@@ -38,7 +38,8 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
         at = up(at + bytes, kAlign);
         return here;
     };
-    const size_t ldm = (size_t)ld_of(jmax), jp = (size_t)jpad_of(jmax);
+    const size_t ldm = (size_t)ld_of(gpus > 0 ? gpus : jmax), jp = (size_t)jpad_of(jmax);
+    const size_t sp = (size_t)jpad_of(gpus > 0 ? gpus : 1);  // slot limits of the per-GPU genome
     // the truncation scheme keeps a pool of 4 * pop rows (originals, crossover children, mutants)
     const size_t rows = trunc ? 4 * (size_t)pop : (size_t)pop;
     const size_t pairs = trunc ? 3 * (size_t)pop : ((size_t)pop + 1) / 2;  // 2K parents + K mutant sources
@@ -49,6 +50,8 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false) {
     L.G = take(rows * 4);
     L.G1 = take(rows * 4);
     L.trunc = take(trunc ? trunc_scratch_bytes(pop) : 16);
+    L.slot_kmin = take(sp * 4);
+    L.slot_range = take(sp * 4);
     L.parents = take(pairs * 2 * 4);
     L.elites = take((size_t)ONES_MAX_ELITES * 4);
     L.elites1 = take((size_t)ONES_MAX_ELITES * 4);
@@ -97,6 +100,9 @@ struct ones_ctx {
     int fcur = 0;           // score buffer in force
     int gcur = 0;           // GPU-count buffer in force (only the truncation scheme alternates it)
     bool trunc = false;     // ONES_FLAG_TRUNCATION
+    bool per_gpu = false;   // ONES_FLAG_PER_GPU: one gene per GPU (a job id) instead of one per job
+    int32_t W = 0;          // genes per candidate
+    Tables tabS{};          // as tab, with the limits of a slot (any job id) for the shared operators
     int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
     int elast = 0;          // elites buffer used by the last generation
     bool elites_valid = false;
@@ -197,6 +203,12 @@ void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
         if ((b + m - 1) / m > 65535) narrow = false;
     }
     c->fused = narrow && !(c->prm.flags & ONES_FLAG_UNFUSED) && evolve_score_smem(c->tab) <= (size_t)kMaxSmemPerBlock;
+    c->tabS = c->tab;
+    if (c->per_gpu) {
+        c->tabS.kmin = reinterpret_cast<int32_t*>(c->ws + c->L.slot_kmin);
+        c->tabS.range = reinterpret_cast<int32_t*>(c->ws + c->L.slot_range);
+        c->fused = false;  // scoring a per-GPU candidate needs its job counts: separate kernel
+    }
     c->cshape = ClusterShape{0, 0, 0, 0, 0};
     if (c->fused && !c->trunc && !(c->prm.flags & ONES_FLAG_NO_CLUSTER))
         c->cshape = cluster_shape(c->tab, ld_of(n_jobs), c->N, c->prm.elitism, c->pairs);
@@ -241,8 +253,11 @@ int prof_end(ones_ctx* c) {
 int run_fitness(ones_ctx* c) {
     int rc = prof_begin(c, 0);
     if (rc) return rc;
-    CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
-                         c->stream));
+    if (c->per_gpu)
+        CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->jobs(), c->F(), c->G(), c->stream));
+    else
+        CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
+                             c->stream));
     c->launches += 1;
     c->f_valid = true;
     c->elites_valid = false;
@@ -303,7 +318,13 @@ size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flag
     if (n_jobs_max <= 0 || n_jobs_max > kJobsLimit || pop <= 0 || pop > kPopLimit) return 0;
     const bool trunc = (flags & ONES_FLAG_TRUNCATION) != 0;
     if (trunc && pop > kPopLimit / 4) return 0;
+    if (flags & ONES_FLAG_PER_GPU) return 0;  // needs the cluster size: ones_workspace_bytes_per_gpu
     return make_layout(n_jobs_max, pop, trunc).total;
+}
+
+size_t ones_workspace_bytes_per_gpu(int32_t n_jobs, int32_t pop, int32_t capacity) {
+    if (n_jobs <= 0 || n_jobs > kJobsLimit || pop <= 0 || pop > kPopLimit || capacity <= 0 || capacity > kJobsLimit) return 0;
+    return make_layout(n_jobs, pop, false, capacity).total;
 }
 
 int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t capacity, int32_t pop,
@@ -320,11 +341,14 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     if (rc) return rc;
     if ((reinterpret_cast<uintptr_t>(d_workspace) & (kAlign - 1)) != 0) return ONES_ERR_ALIGN;
     const bool trunc = (p.flags & ONES_FLAG_TRUNCATION) != 0;
-    if (trunc && pop > kPopLimit / 4) return ONES_ERR_BAD_PARAM;
-    if (workspace_bytes < make_layout(n_jobs, pop, trunc).total) return ONES_ERR_WORKSPACE;
+    const bool per_gpu = (p.flags & ONES_FLAG_PER_GPU) != 0;
+    if (trunc && (pop > kPopLimit / 4 || per_gpu)) return ONES_ERR_BAD_PARAM;
+    if (per_gpu && capacity > kJobsLimit) return ONES_ERR_BAD_PARAM;
+    const int32_t gpus = per_gpu ? capacity : 0;
+    if (workspace_bytes < make_layout(n_jobs, pop, trunc, gpus).total) return ONES_ERR_WORKSPACE;
     // the largest job count this workspace can hold
     int32_t lo = n_jobs, hi = kJobsLimit;
-    while (lo < hi) {
+    while (lo < hi && !per_gpu) {  // (the per-GPU genome has no job-set updates: nothing to grow into)
         const int32_t mid = lo + (hi - lo + 1) / 2;
         if (make_layout(mid, pop, trunc).total <= workspace_bytes) lo = mid;
         else hi = mid - 1;
@@ -333,16 +357,18 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     if (!c) return ONES_ERR_NOMEM;
     c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     c->J = n_jobs;
-    c->Jmax = lo;
+    c->Jmax = per_gpu ? n_jobs : lo;
+    c->per_gpu = per_gpu;
+    c->W = per_gpu ? capacity : n_jobs;
     c->N = pop;
     c->cap = capacity;
     c->prm = p;
     c->thr16 = threshold16(p.p_mut);
     c->trunc = trunc;
     c->pairs = trunc ? pop : (pop - p.elitism + 1) / 2;
-    c->ld = ld_of(n_jobs);
+    c->ld = ld_of(c->W);
     c->ws = reinterpret_cast<char*>(d_workspace);
-    c->L = make_layout(c->Jmax, pop, trunc);
+    c->L = make_layout(c->Jmax, pop, trunc, gpus);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) {
         free_ctx(c);
@@ -357,7 +383,13 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     }
     rc = rebuild_tables(c, jobs, n_jobs);
     if (rc == ONES_OK) {
-        e = launch_fill_min(c->pop(0), c->ld, c->N, c->J, c->tab, c->stream);
+        if (per_gpu) {  // an idle cluster: every slot -1; slot limits for the shared operators
+            e = cudaMemsetAsync(c->pop(0), 0xFF, (size_t)c->N * c->ld * 4, c->stream);
+            if (e == cudaSuccess)
+                e = launch_fill_slot_limits(c->tabS.kmin, c->tabS.range, jpad_of(c->W), c->W, c->J, c->stream);
+        } else {
+            e = launch_fill_min(c->pop(0), c->ld, c->N, c->J, c->tab, c->stream);
+        }
         c->launches += 1;
         if (e != cudaSuccess) rc = cuda_fail(c, e);
     }
@@ -381,7 +413,7 @@ int ones_destroy(ones_ctx* c) {
 int ones_randomize(ones_ctx* c, uint64_t seed) {
     DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
-    CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->J, c->tab, make_round_keys(seed), c->stream));
+    CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->W, c->tabS, make_round_keys(seed), c->stream));
     c->launches += 1;
     c->f_valid = false;
     c->elites_valid = false;
@@ -391,13 +423,13 @@ int ones_randomize(ones_ctx* c, uint64_t seed) {
 int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_device) {
     DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
-    if (ld < c->J) return ONES_ERR_BAD_PARAM;
+    if (ld < c->W) return ONES_ERR_BAD_PARAM;
     if (on_device) {
-        CU(c, launch_copy_rows(genomes, ld, c->pop(c->cur), c->ld, c->N, c->J, 1, c->stream));
+        CU(c, launch_copy_rows(genomes, ld, c->pop(c->cur), c->ld, c->N, c->W, 1, c->stream));
         c->launches += 1;
     } else {
-        if (c->ld != c->J) CU(c, cudaMemsetAsync(c->pop(c->cur), 0, (size_t)c->N * c->ld * 4, c->stream));
-        CU(c, cudaMemcpy2DAsync(c->pop(c->cur), (size_t)c->ld * 4, genomes, (size_t)ld * 4, (size_t)c->J * 4,
+        if (c->ld != c->W) CU(c, cudaMemsetAsync(c->pop(c->cur), 0, (size_t)c->N * c->ld * 4, c->stream));
+        CU(c, cudaMemcpy2DAsync(c->pop(c->cur), (size_t)c->ld * 4, genomes, (size_t)ld * 4, (size_t)c->W * 4,
                                 (size_t)c->N, cudaMemcpyHostToDevice, c->stream));
         CU(c, cudaStreamSynchronize(c->stream));
     }
@@ -409,12 +441,12 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
 int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device) {
     DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
-    if (ld < c->J) return ONES_ERR_BAD_PARAM;
+    if (ld < c->W) return ONES_ERR_BAD_PARAM;
     if (on_device) {
-        CU(c, launch_copy_rows(c->pop(c->cur), c->ld, genomes, ld, c->N, c->J, 0, c->stream));
+        CU(c, launch_copy_rows(c->pop(c->cur), c->ld, genomes, ld, c->N, c->W, 0, c->stream));
         c->launches += 1;
     } else {
-        CU(c, cudaMemcpy2DAsync(genomes, (size_t)ld * 4, c->pop(c->cur), (size_t)c->ld * 4, (size_t)c->J * 4,
+        CU(c, cudaMemcpy2DAsync(genomes, (size_t)ld * 4, c->pop(c->cur), (size_t)c->ld * 4, (size_t)c->W * 4,
                                 (size_t)c->N, cudaMemcpyDeviceToHost, c->stream));
         CU(c, cudaStreamSynchronize(c->stream));
     }
@@ -433,12 +465,15 @@ int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, 
         if (d_gpus) CU(c, cudaMemcpyAsync(d_gpus, c->G(), (size_t)c->N * 4, cudaMemcpyDeviceToDevice, c->stream));
         return ONES_OK;
     }
-    if (n < 0 || ld < c->J) return ONES_ERR_BAD_PARAM;
+    if (n < 0 || ld < c->W) return ONES_ERR_BAD_PARAM;
     if ((ld & 3) != 0 || !aligned16(d_genomes)) return ONES_ERR_ALIGN;
     if (n == 0) return ONES_OK;
     int rc = prof_begin(c, 0);
     if (rc) return rc;
-    CU(c, launch_fitness(d_genomes, ld, n, c->J, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
+    if (c->per_gpu)
+        CU(c, launch_fitness_per_gpu(d_genomes, ld, n, c->W, c->J, c->tab, c->jobs(), d_fitness, d_gpus, c->stream));
+    else
+        CU(c, launch_fitness(d_genomes, ld, n, c->J, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
     c->launches += 1;
     return prof_end(c);
 }
@@ -540,15 +575,24 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
                                       c->parents(), c->elites(0), c->tab, keys, c->gen, c->thr16, c->cap,
                                       c->prm.penalty, c->F(), c->G(), c->stream));
         } else {
-            CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs, c->parents(),
-                                c->elites(0), c->tab, keys, c->gen, c->thr16, c->stream));
+            CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->W, E, c->pairs, c->parents(),
+                                c->elites(0), c->tabS, keys, c->gen, c->thr16, c->stream));
         }
         c->launches += 1;
         if ((rc = prof_end(c)) != ONES_OK) return rc;
 
         c->cur ^= 1;
         c->gen += 1;
-        if (!c->fused && (rc = run_fitness(c)) != ONES_OK) return rc;
+        if (c->per_gpu) {
+            // "Reorder" packs each job's workers in every new candidate; the same pass scores it
+            if ((rc = prof_begin(c, 0)) != ONES_OK) return rc;
+            CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->jobs(), c->F(), c->G(), c->stream));
+            c->launches += 1;
+            c->f_valid = true;
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+        } else if (!c->fused && (rc = run_fitness(c)) != ONES_OK) {
+            return rc;
+        }
     }
     c->prof.sample = true;
     return ONES_OK;
@@ -568,8 +612,13 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
     double* d_rate = reinterpret_cast<double*>(pack + 64);
     int32_t* d_genome = reinterpret_cast<int32_t*>(pack + 64 + J * 8);
     int32_t* d_gpus = reinterpret_cast<int32_t*>(pack + 64 + J * 12);
-    CU(c, launch_best(c->pop(c->cur), c->ld, c->J, c->best_idx(), c->tab, c->cap, c->prm.penalty, repair,
-                      reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
+    if (c->per_gpu)
+        CU(c, launch_best_per_gpu(c->pop(c->cur), c->ld, c->W, c->J, c->best_idx(), c->tab,
+                                  reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec,
+                                  c->stream));
+    else
+        CU(c, launch_best(c->pop(c->cur), c->ld, c->J, c->best_idx(), c->tab, c->cap, c->prm.penalty, repair,
+                          reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
     c->launches += (uint64_t)nl + 1;
     const size_t bytes = 64 + J * 16;
     if ((rc = ensure_staging(c, bytes)) != ONES_OK) return rc;
@@ -589,6 +638,7 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
 int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const int32_t* remap, int32_t capacity) {
     DeviceScope scope(c);
     if (!c || !jobs || !remap) return ONES_ERR_NULL;
+    if (c->per_gpu) return ONES_ERR_BAD_PARAM;  // job ids inside the genomes would need relabelling
     int rc = check_jobs(jobs, n_jobs);
     if (rc) return rc;
     if (capacity <= 0) return ONES_ERR_BAD_PARAM;
@@ -609,6 +659,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
     c->launches += 1;
     c->cur ^= 1;
     c->J = n_jobs;
+    c->W = n_jobs;
     c->ld = new_ld;
     c->cap = capacity;
     c->f_valid = false;

@@ -1687,6 +1687,291 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
 }
 
 // ---------------------------------------------------------------------------------------------
+// The paper's own genome (Eq. 1-2, Fig. 1): one slot per GPU holding a job id (anything outside
+// [0, n_jobs) = idle).  Job j holds c_j = the number of its slots and runs at the largest exponent in
+// [kmin_j, kmax_j] whose GPU need g_j(k) fits into c_j; with none it waits.  Scores are summed over jobs
+// in the same fixed order as everywhere else.
+// ---------------------------------------------------------------------------------------------
+// per job: the exponent it can run at on `count` GPUs (-1: waits).  g_j(k) does not decrease with k, so
+// the search stops at the first exponent that needs more GPUs than the job holds.
+__device__ __forceinline__ int32_t exponent_that_fits(const Tables& t, int32_t j, int32_t count) {
+    const int32_t lo = t.kmin[j], hi = lo + t.range[j] - 1;
+    const int32_t at = slot_of(j);
+    int32_t best = -1;
+    for (int32_t k = lo; k <= hi; ++k) {
+        if (t.G[(int64_t)k * t.jpad + at] > count) break;
+        best = k;
+    }
+    return best;
+}
+
+// The same from the job's own limits, without the table: ceil((b0 << k) / m) <= count exactly when
+// (b0 << k) <= count * m, so the largest such k is floor(log2(count * m / b0)), found from the leading bits.
+__device__ __forceinline__ int32_t exponent_that_fits(int32_t b0, int32_t m, int32_t kmin, int32_t kmax, int32_t count) {
+    const unsigned long long room = (unsigned long long)count * (unsigned long long)m;
+    if (room < (unsigned long long)b0) return -1;
+    int32_t k = (63 - __clzll((long long)room)) - (31 - __clz(b0));
+    if (((unsigned long long)b0 << k) > room) --k;
+    k = min(k, kmax);
+    return k >= kmin ? k : -1;
+}
+
+// Count the GPUs of every job in one row held in shared memory.  A thread walks a contiguous piece of
+// the row and adds a whole run of equal ids at once: after "Reorder" the workers of a job are neighbours,
+// so one atomic per run instead of one per GPU.  FIRST also records each job's first slot.
+template <bool FIRST>
+__device__ __forceinline__ void count_runs(const int32_t* __restrict__ rowbuf, int32_t from, int32_t to, int32_t n_jobs,
+                                           int32_t* __restrict__ count, int32_t* __restrict__ first) {
+    int32_t run_id = -1, run_len = 0, run_at = 0;
+    for (int32_t i = from; i < to; ++i) {
+        const int32_t id = rowbuf[i];
+        if (id != run_id) {
+            if (run_id >= 0) {
+                atomicAdd(&count[run_id], run_len);
+                if (FIRST) atomicMin(&first[run_id], run_at);
+            }
+            run_id = (uint32_t)id < (uint32_t)n_jobs ? id : -1;
+            run_len = 0;
+            run_at = i;
+        }
+        ++run_len;
+    }
+    if (run_id >= 0) {
+        atomicAdd(&count[run_id], run_len);
+        if (FIRST) atomicMin(&first[run_id], run_at);
+    }
+}
+
+// Per-GPU candidates, one CTA per candidate.  SCORE: the candidate's fitness and GPU demand from the
+// job counts.  REORDER: the row rewritten with every job's workers side by side, jobs in order of first
+// occurrence, idle GPUs last; the counts do not change, so both come from one counting pass.
+// Shared memory: count[J] | first[J] start[J] (later the per-job terms, fp64) | the row.
+template <bool REORDER, bool SCORE>
+__global__ void __launch_bounds__(256)
+k_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+          const ones_job* __restrict__ jobs, double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int32_t s_warp[8];
+    __shared__ int32_t s_used;
+    const int32_t jpad4 = (n_jobs + 3) & ~3;
+    int32_t* count = reinterpret_cast<int32_t*>(smem_raw);
+    int32_t* first = count + jpad4;
+    int32_t* start = first + jpad4;
+    double* term = reinterpret_cast<double*>(first);
+    int32_t* rowbuf = start + jpad4;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t piece = ((n_gpus + 255) / 256) | 1;  // odd: neighbouring threads' pieces start in different banks
+    const int32_t from = min(n_gpus, tid * piece), to = min(n_gpus, (tid + 1) * piece);
+    for (int64_t cand = blockIdx.x; cand < n; cand += gridDim.x) {
+        int32_t* row = slots + cand * ld;
+        for (int32_t j = tid; j < n_jobs; j += 256) {
+            count[j] = 0;
+            if (REORDER) first[j] = 0x7FFFFFFF;
+        }
+        if (tid == 0) s_used = 0;
+        for (int32_t i = tid; i < n_gpus; i += 256) rowbuf[i] = row[i];
+        __syncthreads();
+        count_runs<REORDER>(rowbuf, from, to, n_jobs, count, first);
+        __syncthreads();
+        if (REORDER) {
+            // a job's run starts where the runs of the jobs that occurred earlier end: scan over the slots
+            int32_t mine = 0;
+            for (int32_t i = from; i < to; ++i) {
+                const int32_t id = rowbuf[i];
+                if ((uint32_t)id < (uint32_t)n_jobs && first[id] == i) mine += count[id];
+            }
+            int32_t incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            int32_t offset = incl - mine, total = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                const int32_t v = s_warp[w];
+                if (w < warp) offset += v;
+                total += v;
+            }
+            for (int32_t i = from; i < to; ++i) {
+                const int32_t id = rowbuf[i];
+                if ((uint32_t)id < (uint32_t)n_jobs && first[id] == i) {
+                    start[id] = offset;
+                    offset += count[id];
+                }
+            }
+            __syncthreads();
+            // fill: job j occupies [start, start + count); idle GPUs after the last run
+            for (int32_t i = total + tid; i < n_gpus; i += 256) rowbuf[i] = -1;
+            for (int32_t j = tid; j < n_jobs; j += 256) {
+                const int32_t c = count[j];
+                if (c > 0) {
+                    const int32_t s0 = start[j];
+                    for (int32_t u = 0; u < c; ++u) rowbuf[s0 + u] = j;
+                }
+            }
+            __syncthreads();
+            for (int32_t i = tid; i < n_gpus; i += 256) row[i] = rowbuf[i];
+        }
+        if (SCORE) {
+            int32_t used = 0;
+            for (int32_t j0 = tid; j0 < jpad4; j0 += 4 * 256) {
+                // four jobs at a time: their limits first, then the table entries, so the loads overlap
+                int64_t at[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int32_t j = j0 + u * 256;
+                    at[u] = -1;
+                    if (j < n_jobs && count[j] > 0) {
+                        const int4 q = *reinterpret_cast<const int4*>(jobs + j);  // b0, max_per_gpu, kmin, kmax
+                        const int32_t k = exponent_that_fits(q.x, q.y, q.z, q.w, count[j]);
+                        if (k >= 0) at[u] = (int64_t)k * t.jpad + slot_of(j);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int32_t j = j0 + u * 256;
+                    double x = 0.0;
+                    if (at[u] >= 0) {
+                        x = t.X[at[u]];
+                        used += t.G[at[u]];
+                    }
+                    if (j < jpad4) term[j] = x;
+                }
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) used += __shfl_xor_sync(0xFFFFFFFFu, used, off);
+            if (lane == 0 && used) atomicAdd(&s_used, used);
+            __syncthreads();
+            if (warp == 0) {
+                // fixed summation order: lane l adds jobs 4l..4l+3 of every block of 128 jobs in turn,
+                // then the 32 partial sums pairwise; a waiting job adds +0.0, which changes nothing
+                double sum = 0.0;
+                for (int32_t v = lane; 4 * v < jpad4; v += 32) {
+                    const double4 q = *reinterpret_cast<const double4*>(term + 4 * v);
+                    sum = __dadd_rn(__dadd_rn(__dadd_rn(__dadd_rn(sum, q.x), q.y), q.z), q.w);
+                }
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+                if (lane == 0) {
+                    F[cand] = sum;
+                    if (G) G[cand] = s_used;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+static size_t per_gpu_smem(int32_t n_gpus, int32_t n_jobs) {
+    return ((size_t)3 * ((n_jobs + 3) & ~3) + n_gpus) * 4;
+}
+
+template <bool REORDER, bool SCORE>
+static cudaError_t launch_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+                                  const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const size_t smem = per_gpu_smem(n_gpus, n_jobs);
+    if (smem > (size_t)kMaxSmemPerBlock - 2048) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaFuncSetAttribute(k_per_gpu<REORDER, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = n;
+    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    k_per_gpu<REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, jobs, F, G);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fitness_per_gpu(const int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs,
+                                   Tables t, const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<false, true>(const_cast<int32_t*>(slots), ld, n, n_gpus, n_jobs, t, jobs, F, G, s);
+}
+
+cudaError_t launch_reorder(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, cudaStream_t s) {
+    Tables none{};
+    return launch_per_gpu<true, false>(slots, ld, n, n_gpus, n_jobs, none, nullptr, nullptr, nullptr, s);
+}
+
+cudaError_t launch_reorder_score(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+                                 const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<true, true>(slots, ld, n, n_gpus, n_jobs, t, jobs, F, G, s);
+}
+
+// admissible values of a slot: any job id (kmin 0, range n_jobs), for the shared operators
+__global__ void k_fill_slot_limits(int32_t* __restrict__ kmin, int32_t* __restrict__ range, int32_t len, int32_t n_gpus,
+                                   int32_t n_jobs) {
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < len; i += gridDim.x * blockDim.x) {
+        kmin[i] = 0;
+        range[i] = i < n_gpus ? n_jobs : 1;
+    }
+}
+
+cudaError_t launch_fill_slot_limits(int32_t* kmin, int32_t* range, int32_t len, int32_t n_gpus, int32_t n_jobs,
+                                    cudaStream_t s) {
+    k_fill_slot_limits<<<(len + 255) / 256, 256, 0, s>>>(kmin, range, len, n_gpus, n_jobs);
+    return cudaGetLastError();
+}
+
+// best candidate of a per-GPU population as per-job exponents (one CTA); work: n_jobs counters
+__global__ void __launch_bounds__(256)
+k_best_per_gpu(const int32_t* __restrict__ pop, int64_t ld, int32_t n_gpus, int32_t n_jobs,
+               const int32_t* __restrict__ best_index, Tables t, int32_t* __restrict__ work,
+               int32_t* __restrict__ genome_out, int32_t* __restrict__ gpus_out, double* __restrict__ rate_out,
+               BestOut* __restrict__ out) {
+    const int32_t best = best_index[0];
+    const int32_t* row = pop + (int64_t)best * ld;
+    for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) work[j] = 0;
+    __syncthreads();
+    for (int32_t i = threadIdx.x; i < n_gpus; i += blockDim.x) {
+        const int32_t id = row[i];
+        if ((uint32_t)id < (uint32_t)n_jobs) atomicAdd(&work[id], 1);
+    }
+    __syncthreads();
+    for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) {
+        const int32_t k = exponent_that_fits(t, j, work[j]);
+        const int64_t at = (int64_t)(k >= 0 ? k : t.k1) * t.jpad + slot_of(j);
+        genome_out[j] = k;
+        gpus_out[j] = t.G[at];
+        rate_out[j] = t.X[at];
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        double sum = 0.0;
+        int32_t used = 0;
+        const int32_t nvec = (n_jobs + 3) >> 2;
+        for (int32_t v = lane; v < nvec; v += 32)
+            for (int s = 0; s < 4; ++s) {
+                const int32_t j = 4 * v + s;
+                if (j < n_jobs) {
+                    sum = __dadd_rn(sum, rate_out[j]);
+                    used += gpus_out[j];
+                }
+            }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            used += __shfl_xor_sync(0xFFFFFFFFu, used, off);
+        }
+        if (lane == 0) {
+            out->fitness = sum;
+            out->total_gpus = used;
+            out->index = best;
+            out->status = 0;
+            out->steps = 0;
+        }
+    }
+}
+
+cudaError_t launch_best_per_gpu(const int32_t* pop, int64_t ld, int32_t n_gpus, int32_t n_jobs, const int32_t* best_index,
+                                Tables t, int32_t* work, int32_t* genome_out, int32_t* gpus_out, double* rate_out,
+                                BestOut* out, cudaStream_t s) {
+    k_best_per_gpu<<<1, 256, 0, s>>>(pop, ld, n_gpus, n_jobs, best_index, t, work, genome_out, gpus_out, rate_out, out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Best candidate and its repair to the cluster's capacity: one block.
 // work[0..jpad) exponent, work[jpad..2jpad) GPUs now, work[2jpad..3jpad) GPUs one exponent lower
 // (-1 when the job cannot shrink).

@@ -302,6 +302,41 @@ def test_truncation_selection_with_many_ties(ones):
         _same_state(g, o)
 
 
+# ---- the paper's per-GPU genome with the reorder operation -------------------------------------------
+@pytest.mark.parametrize("J,gpus,N,kw", [(6, 12, 64, {}), (100, 64, 1024, {}), (37, 130, 101, dict(p_mut=1.0)),
+                                         (5, 3, 4, dict(p_mut=0.0)), (300, 257, 129, dict(elitism=0)),
+                                         (2048, 4096, 300, dict(p_mut=0.02, tournament=8))])
+def test_per_gpu_genome_parity(ones, J, gpus, N, kw):
+    w = inputs.custom(J, gpus, N, 4, seed=J + N, kmax=6, kmin_max=1)
+    g, o = _pair(ones, w, flags=16, **kw)
+    assert (g.get_population() == -1).all() and g.get_population().shape == (N, gpus)
+    _same_state(g, o)  # an idle cluster scores 0
+    g.randomize(3)
+    o.randomize(3)
+    _same_state(g, o)
+    for step in (1, 2):
+        g.evolve(step, 13)
+        o.evolve(step, 13)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+    bg, bo = g.best(), o.best()
+    for key in ("genome", "gpus_per_job", "rate_per_job"):
+        assert (bg[key] == bo[key]).all(), key
+    assert bg["fitness"] == bo["fitness"] and bg["total_gpus"] == bo["total_gpus"] <= gpus
+    # scoring rows from outside, with idle and invalid ids and padding columns
+    rng = np.random.default_rng(J)
+    ld = (gpus + 3) // 4 * 4 + 4
+    rows = np.full((50, ld), 0x7F7F7F7F, dtype=np.int32)
+    rows[:, :gpus] = rng.integers(-2, J + 2, size=(50, gpus))
+    Fg, Gg = g.evaluate(torch.from_numpy(rows).cuda())
+    Fo, Go = o.evaluate(rows)
+    assert (Fg.cpu().numpy() == Fo).all() and (Gg.cpu().numpy() == Go).all()
+    with pytest.raises(ones.OnesError):
+        g.update_jobs(w.jobs, np.arange(J, dtype=np.int32), gpus)
+
+
 # ---- a6: best and repair ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "paper", "mid"])
 def test_best_and_repair_parity(ones, name):
