@@ -26,7 +26,7 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
         status, total;
 };
 
@@ -52,6 +52,7 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus =
     L.trunc = take(trunc ? trunc_scratch_bytes(pop) : 16);
     L.slot_kmin = take(sp * 4);
     L.slot_range = take(sp * 4);
+    L.fit = take(gpus > 0 ? jp * 16 : 16);  // per-GPU genome: the jobs' limits in the tables' job order
     L.parents = take(pairs * 2 * 4);
     L.elites = take((size_t)ONES_MAX_ELITES * 4);
     L.elites1 = take((size_t)ONES_MAX_ELITES * 4);
@@ -127,6 +128,7 @@ struct ones_ctx {
     int32_t* elites(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.elites1 : L.elites)); }
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
     ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs_in); }
+    int4* fit() { return reinterpret_cast<int4*>(ws + L.fit); }
     int32_t* remap(int32_t n_jobs) { return reinterpret_cast<int32_t*>(ws + L.jobs_in + (size_t)n_jobs * sizeof(ones_job)); }
     int32_t* status() { return reinterpret_cast<int32_t*>(ws + L.status); }
 };
@@ -254,7 +256,7 @@ int run_fitness(ones_ctx* c) {
     int rc = prof_begin(c, 0);
     if (rc) return rc;
     if (c->per_gpu)
-        CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->jobs(), c->F(), c->G(), c->stream));
+        CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->F(), c->G(), c->stream));
     else
         CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
                              c->stream));
@@ -386,7 +388,8 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
         if (per_gpu) {  // an idle cluster: every slot -1; slot limits for the shared operators
             e = cudaMemsetAsync(c->pop(0), 0xFF, (size_t)c->N * c->ld * 4, c->stream);
             if (e == cudaSuccess)
-                e = launch_fill_slot_limits(c->tabS.kmin, c->tabS.range, jpad_of(c->W), c->W, c->J, c->stream);
+                e = launch_fill_slot_limits(c->tabS.kmin, c->tabS.range, jpad_of(c->W), c->W, c->J, c->jobs(), c->fit(),
+                                            c->tab.jpad, c->stream);
         } else {
             e = launch_fill_min(c->pop(0), c->ld, c->N, c->J, c->tab, c->stream);
         }
@@ -471,7 +474,7 @@ int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, 
     int rc = prof_begin(c, 0);
     if (rc) return rc;
     if (c->per_gpu)
-        CU(c, launch_fitness_per_gpu(d_genomes, ld, n, c->W, c->J, c->tab, c->jobs(), d_fitness, d_gpus, c->stream));
+        CU(c, launch_fitness_per_gpu(d_genomes, ld, n, c->W, c->J, c->tab, c->fit(), d_fitness, d_gpus, c->stream));
     else
         CU(c, launch_fitness(d_genomes, ld, n, c->J, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
     c->launches += 1;
@@ -586,7 +589,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         if (c->per_gpu) {
             // "Reorder" packs each job's workers in every new candidate; the same pass scores it
             if ((rc = prof_begin(c, 0)) != ONES_OK) return rc;
-            CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->jobs(), c->F(), c->G(), c->stream));
+            CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->F(), c->G(), c->stream));
             c->launches += 1;
             c->f_valid = true;
             if ((rc = prof_end(c)) != ONES_OK) return rc;

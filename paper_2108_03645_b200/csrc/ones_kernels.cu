@@ -1716,6 +1716,52 @@ __device__ __forceinline__ int32_t exponent_that_fits(int32_t b0, int32_t m, int
     return k >= kmin ? k : -1;
 }
 
+// Per-job terms of one per-GPU candidate from its job counts (shared memory), 256 threads.  A thread
+// takes jobs 4v..4v+3: their counts are one int4, and for each of the four the lanes of a warp read
+// neighbouring entries of the limits and of the model tables (the tables' job order).  Returns the GPUs used.
+__device__ __forceinline__ int32_t per_gpu_terms(const int32_t* __restrict__ count, double* __restrict__ term,
+                                                 int32_t jpad4, const Tables& t, const int4* __restrict__ fit) {
+    int32_t used = 0;
+    for (int32_t v0 = threadIdx.x; 4 * v0 < jpad4; v0 += 2 * 256) {
+        // eight jobs per step: all their limits first, then all their table entries, so the loads overlap
+        int32_t c[8], at[8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int32_t v = v0 + 256 * h;
+            int4 cnt = make_int4(0, 0, 0, 0);
+            if (4 * v < jpad4) cnt = *reinterpret_cast<const int4*>(count + 4 * v);
+            c[4 * h + 0] = cnt.x; c[4 * h + 1] = cnt.y; c[4 * h + 2] = cnt.z; c[4 * h + 3] = cnt.w;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int32_t v = v0 + 256 * (e >> 2);
+            const int32_t entry = ((4 * v) & ~127) + (v & 31) + 32 * (e & 3);
+            at[e] = -1;
+            if (c[e] > 0) {
+                const int4 q = __ldg(fit + entry);  // b0, max_per_gpu, kmin, kmax
+                const int32_t k = exponent_that_fits(q.x, q.y, q.z, q.w, c[e]);
+                if (k >= 0) at[e] = k * t.jpad + entry;
+            }
+        }
+        double x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            x[e] = 0.0;
+            if (at[e] >= 0) {
+                x[e] = __ldg(t.X + at[e]);
+                used += __ldg(t.G + at[e]);
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int32_t v = v0 + 256 * h;
+            if (4 * v < jpad4)
+                *reinterpret_cast<double4*>(term + 4 * v) = make_double4(x[4 * h], x[4 * h + 1], x[4 * h + 2], x[4 * h + 3]);
+        }
+    }
+    return used;
+}
+
 // Count the GPUs of every job in one row held in shared memory.  A thread walks a contiguous piece of
 // the row and adds a whole run of equal ids at once: after "Reorder" the workers of a job are neighbours,
 // so one atomic per run instead of one per GPU.  FIRST also records each job's first slot.
@@ -1749,7 +1795,7 @@ __device__ __forceinline__ void count_runs(const int32_t* __restrict__ rowbuf, i
 template <bool REORDER, bool SCORE>
 __global__ void __launch_bounds__(256)
 k_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-          const ones_job* __restrict__ jobs, double* __restrict__ F, int32_t* __restrict__ G) {
+          const int4* __restrict__ fit, double* __restrict__ F, int32_t* __restrict__ G) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int32_t s_warp[8];
     __shared__ int32_t s_used;
@@ -1816,31 +1862,7 @@ k_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, in
             for (int32_t i = tid; i < n_gpus; i += 256) row[i] = rowbuf[i];
         }
         if (SCORE) {
-            int32_t used = 0;
-            for (int32_t j0 = tid; j0 < jpad4; j0 += 4 * 256) {
-                // four jobs at a time: their limits first, then the table entries, so the loads overlap
-                int64_t at[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int32_t j = j0 + u * 256;
-                    at[u] = -1;
-                    if (j < n_jobs && count[j] > 0) {
-                        const int4 q = *reinterpret_cast<const int4*>(jobs + j);  // b0, max_per_gpu, kmin, kmax
-                        const int32_t k = exponent_that_fits(q.x, q.y, q.z, q.w, count[j]);
-                        if (k >= 0) at[u] = (int64_t)k * t.jpad + slot_of(j);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int32_t j = j0 + u * 256;
-                    double x = 0.0;
-                    if (at[u] >= 0) {
-                        x = t.X[at[u]];
-                        used += t.G[at[u]];
-                    }
-                    if (j < jpad4) term[j] = x;
-                }
-            }
+            int32_t used = per_gpu_terms(count, term, jpad4, t, fit);
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) used += __shfl_xor_sync(0xFFFFFFFFu, used, off);
             if (lane == 0 && used) atomicAdd(&s_used, used);
@@ -1865,27 +1887,179 @@ k_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, in
     }
 }
 
+// The same for rows of at most 256 * PIECE slots: every thread keeps its PIECE neighbouring slots in
+// registers, so the row is read once from global memory and walked without loops over shared memory.
+// Shared memory: count[J] | first[J] | the reordered row, later the per-job terms (fp64).
+template <int PIECE, bool REORDER, bool SCORE>
+__global__ void __launch_bounds__(256, 4)
+k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+               const int4* __restrict__ fit, double* __restrict__ F, int32_t* __restrict__ G) {
+    static_assert(PIECE % 4 == 0, "a thread's slots are whole int4");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int32_t s_warp[8];
+    __shared__ int32_t s_used;
+    const int32_t jpad4 = (n_jobs + 3) & ~3;
+    int32_t* count = reinterpret_cast<int32_t*>(smem_raw);
+    int32_t* first = count + jpad4;
+    int32_t* out = first + jpad4;
+    double* term = reinterpret_cast<double*>(out);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t from = tid * PIECE;
+    int32_t id[PIECE];
+    // this thread's slots of one row (rows are padded to int4); the next row is fetched while the current
+    // one is still being worked on
+    auto fetch = [&](int64_t cand) {
+        const int32_t* src = slots + cand * ld + from;
+#pragma unroll
+        for (int q = 0; q < PIECE / 4; ++q) {
+            int4 v = make_int4(-1, -1, -1, -1);
+            if (from + 4 * q < n_gpus) v = __ldcs(reinterpret_cast<const int4*>(src + 4 * q));
+            id[4 * q + 0] = v.x; id[4 * q + 1] = v.y; id[4 * q + 2] = v.z; id[4 * q + 3] = v.w;
+        }
+    };
+    if (blockIdx.x < n) fetch(blockIdx.x);
+    for (int64_t cand = blockIdx.x; cand < n; cand += gridDim.x) {
+        int32_t* row = slots + cand * ld;
+#pragma unroll
+        for (int u = 0; u < PIECE; ++u)
+            if (from + u >= n_gpus || (uint32_t)id[u] >= (uint32_t)n_jobs) id[u] = -1;  // idle
+        for (int32_t j = 4 * tid; j < jpad4; j += 4 * 256) {
+            *reinterpret_cast<int4*>(count + j) = make_int4(0, 0, 0, 0);
+            if (REORDER) *reinterpret_cast<int4*>(first + j) = make_int4(0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF);
+        }
+        if (tid == 0) s_used = 0;
+        __syncthreads();
+        {   // one atomic per run of equal ids
+            int32_t run_id = -1, run_len = 0, run_at = 0;
+#pragma unroll
+            for (int u = 0; u <= PIECE; ++u) {
+                const int32_t v = u < PIECE ? id[u] : -2;
+                if (v != run_id) {
+                    if (run_id >= 0) {
+                        atomicAdd(&count[run_id], run_len);
+                        if (REORDER) atomicMin(&first[run_id], run_at);
+                    }
+                    run_id = v;
+                    run_len = 0;
+                    run_at = from + u;
+                }
+                ++run_len;
+            }
+        }
+        __syncthreads();
+        if (REORDER) {
+            // a job's run starts where the runs of the jobs that occurred earlier end: scan over the slots
+            int32_t c[PIECE];
+            int32_t mine = 0;
+#pragma unroll
+            for (int u = 0; u < PIECE; ++u) {
+                c[u] = 0;
+                if (id[u] >= 0 && first[id[u]] == from + u) c[u] = count[id[u]];
+                mine += c[u];
+            }
+            int32_t incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            int32_t offset = incl - mine, total = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                const int32_t v = s_warp[w];
+                if (w < warp) offset += v;
+                total += v;
+            }
+#pragma unroll
+            for (int u = 0; u < PIECE; ++u) {
+                for (int32_t r = 0; r < c[u]; ++r) out[offset + r] = id[u];
+                offset += c[u];
+            }
+            for (int32_t i = total + tid; i < n_gpus; i += 256) out[i] = -1;  // idle GPUs last
+            if (cand + gridDim.x < n) fetch(cand + gridDim.x);
+            __syncthreads();
+            for (int32_t i = 4 * tid; i < n_gpus; i += 4 * 256) {
+                if (i + 3 < n_gpus) {
+                    *reinterpret_cast<int4*>(row + i) = *reinterpret_cast<const int4*>(out + i);
+                } else {
+                    for (int32_t r = i; r < n_gpus; ++r) row[r] = out[r];
+                }
+            }
+            if (SCORE) __syncthreads();  // the terms take the row's place
+        }
+        if (!REORDER && cand + gridDim.x < n) fetch(cand + gridDim.x);
+        if (SCORE) {
+            int32_t used = per_gpu_terms(count, term, jpad4, t, fit);
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) used += __shfl_xor_sync(0xFFFFFFFFu, used, off);
+            if (lane == 0 && used) atomicAdd(&s_used, used);
+            __syncthreads();
+            if (warp == 0) {
+                // fixed summation order: lane l adds jobs 4l..4l+3 of every block of 128 jobs in turn,
+                // then the 32 partial sums pairwise; a waiting job adds +0.0, which changes nothing
+                double sum = 0.0;
+                for (int32_t v = lane; 4 * v < jpad4; v += 32) {
+                    const double4 q = *reinterpret_cast<const double4*>(term + 4 * v);
+                    sum = __dadd_rn(__dadd_rn(__dadd_rn(__dadd_rn(sum, q.x), q.y), q.z), q.w);
+                }
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+                if (lane == 0) {
+                    F[cand] = sum;
+                    if (G) G[cand] = s_used;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+static size_t per_gpu_regs_smem(int32_t n_gpus, int32_t n_jobs) {
+    const size_t jpad4 = (size_t)((n_jobs + 3) & ~3), wpad = (size_t)((n_gpus + 3) & ~3);
+    const size_t tail = wpad * 4 > jpad4 * 8 ? wpad * 4 : jpad4 * 8;
+    return 2 * jpad4 * 4 + tail;
+}
+
+template <int PIECE, bool REORDER, bool SCORE>
+static cudaError_t launch_per_gpu_regs(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+                                       const int4* fit, double* F, int32_t* G, cudaStream_t s) {
+    const size_t smem = per_gpu_regs_smem(n_gpus, n_jobs);
+    cudaError_t e = cudaFuncSetAttribute(k_per_gpu_regs<PIECE, REORDER, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = n;
+    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    k_per_gpu_regs<PIECE, REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G);
+    return cudaGetLastError();
+}
+
 static size_t per_gpu_smem(int32_t n_gpus, int32_t n_jobs) {
     return ((size_t)3 * ((n_jobs + 3) & ~3) + n_gpus) * 4;
 }
 
 template <bool REORDER, bool SCORE>
 static cudaError_t launch_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                  const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
+                                  const int4* fit, double* F, int32_t* G, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
+    if (per_gpu_regs_smem(n_gpus, n_jobs) <= (size_t)kMaxSmemPerBlock - 2048) {
+        if (n_gpus <= 256 * 4) return launch_per_gpu_regs<4, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+        if (n_gpus <= 256 * 16) return launch_per_gpu_regs<16, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+    }
     const size_t smem = per_gpu_smem(n_gpus, n_jobs);
     if (smem > (size_t)kMaxSmemPerBlock - 2048) return cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(k_per_gpu<REORDER, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int64_t blocks = n;
     if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
-    k_per_gpu<REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, jobs, F, G);
+    k_per_gpu<REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G);
     return cudaGetLastError();
 }
 
 cudaError_t launch_fitness_per_gpu(const int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs,
-                                   Tables t, const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
-    return launch_per_gpu<false, true>(const_cast<int32_t*>(slots), ld, n, n_gpus, n_jobs, t, jobs, F, G, s);
+                                   Tables t, const int4* fit, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<false, true>(const_cast<int32_t*>(slots), ld, n, n_gpus, n_jobs, t, fit, F, G, s);
 }
 
 cudaError_t launch_reorder(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, cudaStream_t s) {
@@ -1894,22 +2068,29 @@ cudaError_t launch_reorder(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus
 }
 
 cudaError_t launch_reorder_score(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                 const ones_job* jobs, double* F, int32_t* G, cudaStream_t s) {
-    return launch_per_gpu<true, true>(slots, ld, n, n_gpus, n_jobs, t, jobs, F, G, s);
+                                 const int4* fit, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<true, true>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
 }
 
-// admissible values of a slot: any job id (kmin 0, range n_jobs), for the shared operators
+// admissible values of a slot: any job id (kmin 0, range n_jobs), for the shared operators; and the
+// jobs' limits (b0, max_per_gpu, kmin, kmax) in the model tables' job order, for the exponent search
 __global__ void k_fill_slot_limits(int32_t* __restrict__ kmin, int32_t* __restrict__ range, int32_t len, int32_t n_gpus,
-                                   int32_t n_jobs) {
+                                   int32_t n_jobs, const ones_job* __restrict__ jobs, int4* __restrict__ fit, int32_t jpad) {
     for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < len; i += gridDim.x * blockDim.x) {
         kmin[i] = 0;
         range[i] = i < n_gpus ? n_jobs : 1;
     }
+    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < jpad; j += gridDim.x * blockDim.x) {
+        int4 q = make_int4(1, 1, 1, 0);  // no job: no exponent fits
+        if (j < n_jobs) q = make_int4(jobs[j].b0, jobs[j].max_per_gpu, jobs[j].kmin, jobs[j].kmax);
+        fit[slot_of(j)] = q;
+    }
 }
 
 cudaError_t launch_fill_slot_limits(int32_t* kmin, int32_t* range, int32_t len, int32_t n_gpus, int32_t n_jobs,
-                                    cudaStream_t s) {
-    k_fill_slot_limits<<<(len + 255) / 256, 256, 0, s>>>(kmin, range, len, n_gpus, n_jobs);
+                                    const ones_job* jobs, int4* fit, int32_t jpad, cudaStream_t s) {
+    const int32_t most = len > jpad ? len : jpad;
+    k_fill_slot_limits<<<(most + 255) / 256, 256, 0, s>>>(kmin, range, len, n_gpus, n_jobs, jobs, fit, jpad);
     return cudaGetLastError();
 }
 

@@ -305,7 +305,8 @@ def test_truncation_selection_with_many_ties(ones):
 # ---- the paper's per-GPU genome with the reorder operation -------------------------------------------
 @pytest.mark.parametrize("J,gpus,N,kw", [(6, 12, 64, {}), (100, 64, 1024, {}), (37, 130, 101, dict(p_mut=1.0)),
                                          (5, 3, 4, dict(p_mut=0.0)), (300, 257, 129, dict(elitism=0)),
-                                         (2048, 4096, 300, dict(p_mut=0.02, tournament=8))])
+                                         (2048, 4096, 300, dict(p_mut=0.02, tournament=8)), (40, 4100, 33, {}),
+                                         (1500, 1027, 40, {})])
 def test_per_gpu_genome_parity(ones, J, gpus, N, kw):
     w = inputs.custom(J, gpus, N, 4, seed=J + N, kmax=6, kmin_max=1)
     g, o = _pair(ones, w, flags=16, **kw)
