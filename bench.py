@@ -139,6 +139,9 @@ def oracle_sample(w, pop_sample: int, gens: int):
 
 def cpu_baseline(w, pop_sample=8192, gens=None):
     pop_sample = min(pop_sample, w.pop)
+    if w.params.flags & 16:
+        # per-GPU genome: the oracle's reorder costs slots x jobs per row (about 3.5 ms at 4096 x 2048)
+        pop_sample, gens = min(pop_sample, 1024), 4
     if gens is None:  # about 1e8 gene evaluations: seconds of single-thread work
         gens = int(min(2000, max(8, 1.3e8 / (pop_sample * w.n_jobs))))
     dt = oracle_sample(w, pop_sample, gens)

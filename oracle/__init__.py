@@ -71,6 +71,7 @@ def _configure(L: C.CDLL) -> C.CDLL:
     L.oracle_keep_best.argtypes = [vp, i32, i32, vp]
     L.oracle_fitness_per_gpu.argtypes = [vp, i32, i32, u32, vp, vp, vp, vp]
     L.oracle_reorder.argtypes = [vp, i32, i32]
+    L.oracle_refresh.argtypes = [vp, i32, u32, vp, i32, vp, vp, i32]
     L.oracle_thr16.argtypes = [dbl]
     L.oracle_thr16.restype = u32
     L.oracle_create.argtypes = [vp, vp, i32, i32, i32, vp]
@@ -218,6 +219,18 @@ def reorder(slots, n_jobs: int) -> np.ndarray:
     return sl
 
 
+def refresh(jobs, slots, inv, is_new, flags: int = 0) -> np.ndarray:
+    """One per-GPU candidate refreshed for a new job table (not packed: see `reorder`)."""
+    a = _jobs_arr(jobs)
+    sl = np.array(slots, dtype=np.int32)
+    iv = np.ascontiguousarray(inv, dtype=np.int32)
+    nw = np.ascontiguousarray(is_new, dtype=np.int8)
+    assert nw.shape[0] == a.shape[0]
+    _check(lib().oracle_refresh(_ptr(a), a.shape[0], flags, _ptr(iv), iv.shape[0], _ptr(nw), _ptr(sl), sl.shape[0]),
+           "refresh")
+    return sl
+
+
 def keep_best(F, k: int) -> np.ndarray:
     f = np.ascontiguousarray(F, dtype=np.float64)
     idx = np.zeros(max(k, 1), dtype=np.int32)
@@ -242,6 +255,7 @@ class Search:
         self.N = int(pop)
         self.E = int(elitism)
         self.W = int(capacity) if flags & FLAG_PER_GPU else self.J  # genes per candidate
+        self.flags = int(flags)
         prm = _Params(elitism, tournament, p_mut, penalty, flags)
         rc = lib().oracle_create(C.byref(self._h), _ptr(self.jobs), self.J, capacity, pop, C.byref(prm))
         if rc != 0:
@@ -308,7 +322,8 @@ class Search:
         _check(lib().oracle_update_jobs(self._h, _ptr(a), a.shape[0], _ptr(r), capacity), "update_jobs")
         self.jobs = a
         self.J = int(a.shape[0])
-        self.W = self.J
+        if not self.flags & FLAG_PER_GPU:
+            self.W = self.J
 
     def last_parents(self):
         pairs = int(lib().oracle_pairs(self._h))

@@ -295,6 +295,82 @@ int oracle_reorder(int32_t* slots, int32_t n_gpus, int32_t n_jobs) {
     return ORACLE_OK;
 }
 
+/* "Refresh" of one per-GPU candidate at a change of the job set (Section 3.2.2).
+ * inv[o] = new id of old job o, or -1 when it has finished; is_new[j] != 0 for a job that was not there. */
+int oracle_refresh(const oracle_job* jobs, int32_t n_jobs, uint32_t flags, const int32_t* inv, int32_t n_jobs_old,
+                   const char* is_new, int32_t* slots, int32_t n_gpus) {
+    if (!jobs || !inv || !is_new || !slots) return ORACLE_ERR_NULL;
+    int32_t* count = (int32_t*)calloc((size_t)(n_jobs > 0 ? n_jobs : 1), sizeof(int32_t));
+    int32_t* limit = (int32_t*)calloc((size_t)(n_jobs > 0 ? n_jobs : 1), sizeof(int32_t));
+    if (!count || !limit) { free(count); free(limit); return ORACLE_ERR_NOMEM; }
+    /* (1) GPUs of finished jobs become idle; surviving jobs are known by their new ids */
+    for (int32_t i = 0; i < n_gpus; ++i) {
+        int32_t o = slots[i];
+        slots[i] = (o >= 0 && o < n_jobs_old) ? inv[o] : -1;
+        if (slots[i] >= 0) count[slots[i]] += 1;
+    }
+    /* (2) scale down: a job gives up the GPUs beyond those its batch-size limit needs, last ones first */
+    for (int32_t j = 0; j < n_jobs; ++j) {
+        double X;
+        oracle_model(&jobs[j], jobs[j].kmax, &X, &limit[j]);
+    }
+    for (int32_t i = n_gpus - 1; i >= 0; --i) {
+        int32_t j = slots[i];
+        if (j >= 0 && count[j] > limit[j]) { slots[i] = -1; count[j] -= 1; }
+    }
+    /* (3) every new job gets the GPUs of its smallest batch: idle GPUs first (lowest first), then the
+     * last GPU of the job that has been here longest (lowest index) among those that still hold one */
+    for (int32_t j = 0; j < n_jobs; ++j) {
+        if (!is_new[j]) continue;
+        double X; int32_t want;
+        oracle_model(&jobs[j], jobs[j].kmin, &X, &want);
+        for (int32_t u = 0; u < want; ++u) {
+            int32_t at = -1;
+            for (int32_t i = 0; i < n_gpus && at < 0; ++i) if (slots[i] < 0) at = i;
+            if (at < 0) {
+                int32_t v = -1;
+                for (int32_t q = 0; q < n_jobs && v < 0; ++q) if (!is_new[q] && count[q] > 0) v = q;
+                if (v < 0) break;
+                for (int32_t i = n_gpus - 1; i >= 0 && at < 0; --i) if (slots[i] == v) at = i;
+                count[v] -= 1;
+            }
+            slots[at] = j;
+            count[j] += 1;
+        }
+    }
+    /* (4) fill the idle GPUs: the job whose score term gains most from growing to its limit goes first
+     * (ties: lower index) and takes what it needs for that, or what is left */
+    for (;;) {
+        int32_t idle = 0;
+        for (int32_t i = 0; i < n_gpus; ++i) idle += slots[i] < 0;
+        if (idle == 0) break;
+        int32_t pick = -1;
+        double best = 0.0;
+        for (int32_t j = 0; j < n_jobs; ++j) {
+            if (count[j] >= limit[j]) continue;
+            int32_t know = -1, g;
+            for (int32_t k = jobs[j].kmin; k <= jobs[j].kmax; ++k) {
+                double X;
+                oracle_model(&jobs[j], k, &X, &g);
+                if (g <= count[j]) know = k;
+            }
+            double now = 0.0, top;
+            if (know >= 0) oracle_term(&jobs[j], know, flags, &now, &g);
+            oracle_term(&jobs[j], jobs[j].kmax, flags, &top, &g);
+            double gain = top - now;
+            if (pick < 0 || gain > best) { pick = j; best = gain; }
+        }
+        if (pick < 0) break;
+        int32_t take = limit[pick] - count[pick];
+        if (take > idle) take = idle;
+        for (int32_t i = 0; i < n_gpus && take > 0; ++i)
+            if (slots[i] < 0) { slots[i] = pick; count[pick] += 1; take -= 1; }
+    }
+    free(count);
+    free(limit);
+    return ORACLE_OK;
+}
+
 /* ------------------------------------------------------------------------- */
 /* The search                                                                  */
 /* ------------------------------------------------------------------------- */
@@ -624,18 +700,39 @@ int oracle_best(oracle_ctx* c, int repair, int32_t* genome, int32_t* gpus_per_jo
 int oracle_update_jobs(oracle_ctx* c, const oracle_job* jobs, int32_t n_jobs, const int32_t* remap,
                        int32_t capacity) {
     if (!c || !jobs || !remap) return ORACLE_ERR_NULL;
-    if (c->prm.flags & ORACLE_FLAG_PER_GPU) return ORACLE_ERR_BAD_PARAM; /* job ids would need relabelling */
     int rc = oracle_validate_jobs(jobs, n_jobs);
     if (rc) return rc;
     if (capacity <= 0) return ORACLE_ERR_BAD_PARAM;
     for (int32_t j = 0; j < n_jobs; ++j)
         if (remap[j] < -1 || remap[j] >= c->J) return ORACLE_ERR_BAD_PARAM;
+    oracle_job* nj = (oracle_job*)malloc(sizeof(oracle_job) * (size_t)n_jobs);
+    if (!nj) return ORACLE_ERR_NOMEM;
+    memcpy(nj, jobs, sizeof(oracle_job) * (size_t)n_jobs);
+    if (c->prm.flags & ORACLE_FLAG_PER_GPU) {
+        /* the cluster keeps its size; every candidate is refreshed and packed again */
+        if (capacity != c->cap) { free(nj); return ORACLE_ERR_BAD_PARAM; }
+        int32_t* inv = (int32_t*)malloc(sizeof(int32_t) * (size_t)c->J);
+        char* is_new = (char*)calloc((size_t)n_jobs, 1);
+        if (!inv || !is_new) { free(inv); free(is_new); free(nj); return ORACLE_ERR_NOMEM; }
+        for (int32_t o = 0; o < c->J; ++o) inv[o] = -1;
+        for (int32_t j = 0; j < n_jobs; ++j) {
+            if (remap[j] >= 0) inv[remap[j]] = j; else is_new[j] = 1;
+        }
+        for (int32_t i = 0; i < c->N; ++i) {
+            int32_t* row = &c->pop[(size_t)i * c->W];
+            oracle_refresh(jobs, n_jobs, c->prm.flags, inv, c->J, is_new, row, c->W);
+            oracle_reorder(row, c->W, n_jobs);
+        }
+        free(inv); free(is_new); free(c->jobs);
+        c->jobs = nj;
+        c->J = n_jobs;
+        c->f_valid = 0;
+        return ORACLE_OK;
+    }
     size_t cells = (size_t)c->N * (size_t)n_jobs;
     int32_t* np = (int32_t*)malloc(sizeof(int32_t) * cells);
     int32_t* nn = (int32_t*)malloc(sizeof(int32_t) * cells);
-    oracle_job* nj = (oracle_job*)malloc(sizeof(oracle_job) * (size_t)n_jobs);
-    if (!np || !nn || !nj) { free(np); free(nn); free(nj); return ORACLE_ERR_NOMEM; }
-    memcpy(nj, jobs, sizeof(oracle_job) * (size_t)n_jobs);
+    if (!np || !nn) { free(np); free(nn); free(nj); return ORACLE_ERR_NOMEM; }
     /* refresh: finished jobs' columns vanish, surviving jobs keep their gene
      * (clamped into the new limits), new jobs start at their smallest batch */
     for (int32_t i = 0; i < c->N; ++i)

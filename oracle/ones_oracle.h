@@ -88,6 +88,16 @@ int oracle_fitness_per_gpu(const oracle_job* jobs, int32_t n_jobs, int32_t n_gpu
 /* "Reorder": the workers of a job become neighbours, jobs in the order of their first occurrence,
  * idle GPUs last */
 int oracle_reorder(int32_t* slots, int32_t n_gpus, int32_t n_jobs);
+/* "Refresh" of one per-GPU candidate when the job set changes (Section 3.2.2, Fig. 5), in four steps:
+ * (1) slots of finished jobs become idle and surviving jobs take their new ids (inv[old id] = new id or -1);
+ * (2) a job holding more GPUs than its batch-size limit needs gives up the surplus, last slots first;
+ * (3) each new job (is_new) gets the GPUs of its smallest batch: the lowest idle slots, else the last slot of
+ *     the lowest-index (longest present) surviving job that still holds one;
+ * (4) while a GPU is idle: the job below its limit whose score term gains most from growing to the limit
+ *     (ties: lower index) takes the GPUs it needs for that, or what is left, lowest idle slots first.
+ * The row is not packed here (see oracle_reorder). */
+int oracle_refresh(const oracle_job* jobs, int32_t n_jobs, uint32_t flags, const int32_t* inv, int32_t n_jobs_old,
+                   const char* is_new, int32_t* slots, int32_t n_gpus);
 /* the k best of n scores, as ascending indices (truncation selection, order preserved) */
 int oracle_keep_best(const double* F, int32_t n, int32_t k, int32_t* kept);
 /* mutation threshold on the 16-bit decision field for probability p */

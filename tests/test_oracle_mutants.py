@@ -17,6 +17,7 @@ import test_oracle_rng as R
 import test_oracle_search as S
 import test_oracle_truncation as T
 import test_oracle_per_gpu as P
+import test_oracle_refresh as RF
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "ones_oracle.c")
 
@@ -95,6 +96,30 @@ CASES = [
      [P.test_reorder_examples]),
     ("per-GPU search skips the reorder", "for (int32_t i = 0; i < N; ++i) oracle_reorder(&c->next[(size_t)i * J], J, c->J);", "(void)0;",
      [P.test_search_on_the_per_gpu_genome]),
+    ("refresh: surplus GPUs freed from the front", "for (int32_t i = n_gpus - 1; i >= 0; --i) {\n        int32_t j = slots[i];\n        if (j >= 0 && count[j] > limit[j])",
+     "for (int32_t i = 0; i < n_gpus; ++i) {\n        int32_t j = slots[i];\n        if (j >= 0 && count[j] > limit[j])",
+     [RF.test_scale_down_frees_the_last_gpus_beyond_the_limit]),
+    ("refresh: no scale-down", "if (j >= 0 && count[j] > limit[j]) { slots[i] = -1; count[j] -= 1; }", "(void)j;",
+     [RF.test_scale_down_frees_the_last_gpus_beyond_the_limit]),
+    ("refresh: GPUs taken from the newest job", "for (int32_t q = 0; q < n_jobs && v < 0; ++q) if (!is_new[q] && count[q] > 0) v = q;",
+     "for (int32_t q = n_jobs - 1; q >= 0 && v < 0; --q) if (!is_new[q] && count[q] > 0) v = q;",
+     [RF.test_new_job_takes_the_last_gpu_of_the_longest_present_job_when_nothing_is_idle]),
+    ("refresh: the victim's first GPU instead of its last", "for (int32_t i = n_gpus - 1; i >= 0 && at < 0; --i) if (slots[i] == v) at = i;",
+     "for (int32_t i = 0; i < n_gpus && at < 0; ++i) if (slots[i] == v) at = i;",
+     [RF.test_new_job_takes_the_last_gpu_of_the_longest_present_job_when_nothing_is_idle]),
+    ("refresh: one GPU per new job whatever its smallest batch needs", "oracle_model(&jobs[j], jobs[j].kmin, &X, &want);",
+     "oracle_model(&jobs[j], jobs[j].kmin, &X, &want); want = 1;",
+     [RF.test_new_job_takes_the_last_gpu_of_the_longest_present_job_when_nothing_is_idle]),
+    ("refresh: the smallest gain goes first", "if (pick < 0 || gain > best) { pick = j; best = gain; }",
+     "if (pick < 0 || gain < best) { pick = j; best = gain; }", [RF.test_fig5_like_example_finished_job_new_job_and_refill]),
+    ("refresh: ties to the higher index", "if (pick < 0 || gain > best) { pick = j; best = gain; }",
+     "if (pick < 0 || gain >= best) { pick = j; best = gain; }", [RF.test_fig5_like_example_finished_job_new_job_and_refill]),
+    ("refresh: the gain ignores what the job runs at now", "double gain = top - now;", "double gain = top;",
+     [RF.test_refresh_against_the_python_restatement_and_invariants]),
+    ("refresh: new jobs wait behind the refill", "if (!is_new[j]) continue;", "if (1) continue;",
+     [RF.test_fig5_like_example_finished_job_new_job_and_refill]),
+    ("a job-set change skips the refresh", "oracle_refresh(jobs, n_jobs, c->prm.flags, inv, c->J, is_new, row, c->W);", "(void)0;",
+     [RF.test_search_refreshes_every_candidate_at_a_job_set_change]),
     ("mutants take the parents' stream", "(uint32_t)m, (uint32_t)j, ORACLE_STREAM_MUTANT);", "(uint32_t)m, (uint32_t)j, ORACLE_STREAM_MUT);",
      [T.test_generation_is_best_k_of_originals_children_and_mutants]),
 ]

@@ -92,4 +92,4 @@ def test_search_on_the_per_gpu_genome():
     assert got["total_gpus"] <= 12 and got["gpus_per_job"].sum() == got["total_gpus"]
     assert got["fitness"] == pytest.approx(math.fsum(got["rate_per_job"]), rel=1e-13)
     with pytest.raises(oracle.OracleError):
-        s.update_jobs(w.jobs, np.arange(6, dtype=np.int32), 12)
+        s.update_jobs(w.jobs, np.arange(6, dtype=np.int32), 13)   # the cluster keeps its size
