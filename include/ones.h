@@ -95,8 +95,8 @@ typedef struct {
  * the paper's "Reorder" (the workers of a job become neighbours, jobs in the order of their first
  * occurrence, idle GPUs last).  ones_create starts from an idle cluster.  ones_best returns the best
  * candidate as per-job exponents (h_genome[n_jobs], -1 = waits); the per-GPU rows come from
- * ones_get_population.  ones_update_jobs is not available; not combinable with ONES_FLAG_TRUNCATION.
- * Size the workspace with ones_workspace_bytes_per_gpu. */
+ * ones_get_population.  ones_update_jobs runs the paper's "Refresh" on every candidate (see there).
+ * Not combinable with ONES_FLAG_TRUNCATION.  Size the workspace with ones_workspace_bytes_per_gpu. */
 #define ONES_FLAG_PER_GPU 16u
 
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
@@ -120,8 +120,9 @@ enum {
 size_t ones_workspace_bytes(int32_t n_jobs_max, int32_t pop);
 /* The same for a handle created with `flags` (ONES_FLAG_TRUNCATION needs room for its candidate pool). */
 size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flags);
-/* The same for a handle with ONES_FLAG_PER_GPU (rows hold `capacity` genes). */
-size_t ones_workspace_bytes_per_gpu(int32_t n_jobs, int32_t pop, int32_t capacity);
+/* The same for a handle with ONES_FLAG_PER_GPU (rows hold `capacity` genes); n_jobs_max is the largest job
+ * set that ones_update_jobs will be given. */
+size_t ones_workspace_bytes_per_gpu(int32_t n_jobs_max, int32_t pop, int32_t capacity);
 
 /* Create a search over `n_jobs` jobs on a cluster of `capacity` GPUs with a
  * population of `pop` candidates (Section 3.2.2 "Initialization": the population
@@ -188,7 +189,22 @@ int ones_best(ones_ctx* ctx, int repair, int32_t* h_genome, int32_t* h_gpus_per_
  * jobs leave, new jobs arrive, limits R_j move).  Column j of the new population is
  * column remap[j] of the old one clamped into the new [kmin_j, kmax_j], or kmin_j
  * when remap[j] == -1; the model tables are rebuilt.  jobs, remap: host, n_jobs
- * entries; n_jobs must fit the workspace.  Asynchronous apart from argument checks. */
+ * entries; n_jobs must fit the workspace.  Asynchronous apart from argument checks.
+ *
+ * With ONES_FLAG_PER_GPU the candidates hold job ids, and every candidate goes through the four steps of
+ * "Refresh" (Fig. 5) and then "Reorder":
+ *   (1) the GPUs of finished jobs (old ids that no remap[j] names) become idle, surviving jobs take their
+ *       new ids (should several new rows name one old job, the highest j keeps its GPUs);
+ *   (2) a job holding more GPUs than its batch-size limit b0 << kmax needs gives up the surplus, its last
+ *       GPUs first;
+ *   (3) every new job (remap[j] == -1), in index order, gets the GPUs of its smallest batch: the lowest idle
+ *       GPUs, and when none is idle the last GPU of the lowest-index (longest present) surviving job that
+ *       still holds one;
+ *   (4) while a GPU is idle, the job below its limit whose score term gains most from growing to the limit
+ *       (ties: lower index) takes the GPUs it needs for that, or what is left, lowest idle GPUs first.
+ * capacity must equal the cluster size of ones_create (ONES_ERR_BAD_PARAM otherwise).  The step keeps one
+ * candidate and its per-job lists in the shared memory of a thread block: 8 * capacity + 40 * n_jobs bytes
+ * (n_jobs rounded up to a power of two) must stay below 226 KiB, else ONES_ERR_WORKSPACE. */
 int ones_update_jobs(ones_ctx* ctx, const ones_job* jobs, int32_t n_jobs, const int32_t* remap,
                      int32_t capacity);
 

@@ -153,7 +153,7 @@ class Search:
         nmax = max(self.J, int(n_jobs_max or 0))
         self.W = int(capacity) if p.flags & FLAG_PER_GPU else self.J  # genes per candidate
         if p.flags & FLAG_PER_GPU:
-            nbytes = int(lib().ones_workspace_bytes_per_gpu(self.J, pop, capacity))
+            nbytes = int(lib().ones_workspace_bytes_per_gpu(nmax, pop, capacity))
         else:
             nbytes = workspace_bytes(nmax, pop, p.flags)
         if nbytes == 0:
@@ -251,7 +251,8 @@ class Search:
         self._check(lib().ones_update_jobs(self._h, _np_ptr(jobs), jobs.shape[0], _np_ptr(r), capacity),
                     "ones_update_jobs")
         self.J = int(jobs.shape[0])
-        self.W = self.J
+        if not self.params.flags & FLAG_PER_GPU:
+            self.W = self.J
         self.capacity = int(capacity)
 
     # -- inspection ---------------------------------------------------------------

@@ -26,7 +26,7 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, refresh, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
         status, total;
 };
 
@@ -53,6 +53,7 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus =
     L.slot_kmin = take(sp * 4);
     L.slot_range = take(sp * 4);
     L.fit = take(gpus > 0 ? jp * 16 : 16);  // per-GPU genome: the jobs' limits in the tables' job order
+    L.refresh = take(gpus > 0 ? (2 * (size_t)jmax + 2) * 4 : 16);  // per-GPU genome: old -> new ids, new jobs' needs
     L.parents = take(pairs * 2 * 4);
     L.elites = take((size_t)ONES_MAX_ELITES * 4);
     L.elites1 = take((size_t)ONES_MAX_ELITES * 4);
@@ -129,6 +130,8 @@ struct ones_ctx {
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
     ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs_in); }
     int4* fit() { return reinterpret_cast<int4*>(ws + L.fit); }
+    int32_t* refresh_inv() { return reinterpret_cast<int32_t*>(ws + L.refresh); }
+    int32_t* refresh_cum() { return refresh_inv() + Jmax; }
     int32_t* remap(int32_t n_jobs) { return reinterpret_cast<int32_t*>(ws + L.jobs_in + (size_t)n_jobs * sizeof(ones_job)); }
     int32_t* status() { return reinterpret_cast<int32_t*>(ws + L.status); }
 };
@@ -350,16 +353,16 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     if (workspace_bytes < make_layout(n_jobs, pop, trunc, gpus).total) return ONES_ERR_WORKSPACE;
     // the largest job count this workspace can hold
     int32_t lo = n_jobs, hi = kJobsLimit;
-    while (lo < hi && !per_gpu) {  // (the per-GPU genome has no job-set updates: nothing to grow into)
+    while (lo < hi) {
         const int32_t mid = lo + (hi - lo + 1) / 2;
-        if (make_layout(mid, pop, trunc).total <= workspace_bytes) lo = mid;
+        if (make_layout(mid, pop, trunc, gpus).total <= workspace_bytes) lo = mid;
         else hi = mid - 1;
     }
     ones_ctx* c = new (std::nothrow) ones_ctx();
     if (!c) return ONES_ERR_NOMEM;
     c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     c->J = n_jobs;
-    c->Jmax = per_gpu ? n_jobs : lo;
+    c->Jmax = lo;
     c->per_gpu = per_gpu;
     c->W = per_gpu ? capacity : n_jobs;
     c->N = pop;
@@ -641,20 +644,37 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
 int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const int32_t* remap, int32_t capacity) {
     DeviceScope scope(c);
     if (!c || !jobs || !remap) return ONES_ERR_NULL;
-    if (c->per_gpu) return ONES_ERR_BAD_PARAM;  // job ids inside the genomes would need relabelling
     int rc = check_jobs(jobs, n_jobs);
     if (rc) return rc;
     if (capacity <= 0) return ONES_ERR_BAD_PARAM;
     if (n_jobs > c->Jmax) return ONES_ERR_WORKSPACE;
     for (int32_t j = 0; j < n_jobs; ++j)
         if (remap[j] < -1 || remap[j] >= c->J) return ONES_ERR_BAD_PARAM;
+    if (c->per_gpu) {
+        if (capacity != c->cap) return ONES_ERR_BAD_PARAM;  // a candidate has one gene per GPU of the cluster
+        if (refresh_smem(c->W, n_jobs) > (size_t)kMaxSmemPerBlock - 1024) return ONES_ERR_WORKSPACE;
+    }
     const int64_t old_ld = c->ld;
+    const int32_t old_J = c->J;
     rc = rebuild_tables(c, jobs, n_jobs, remap);
     if (rc != ONES_OK) {
         // put the tables of the job set in force back; the population is untouched
         const std::vector<ones_job> keep = c->h_jobs;
         int rc2 = rebuild_tables(c, keep.data(), (int32_t)keep.size());
         return rc2 == ONES_OK ? rc : rc2;
+    }
+    if (c->per_gpu) {
+        // every candidate is refreshed in place (finished jobs leave, limits, new jobs, refill) and packed again
+        CU(c, launch_fill_slot_limits(c->tabS.kmin, c->tabS.range, jpad_of(c->W), c->W, n_jobs, c->jobs(), c->fit(),
+                                      c->tab.jpad, c->stream));
+        CU(c, launch_refresh_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, old_J, n_jobs, c->tab, c->fit(), c->remap(n_jobs),
+                                     c->refresh_inv(), c->refresh_cum(), c->stream));
+        CU(c, launch_reorder(c->pop(c->cur), c->ld, c->N, c->W, n_jobs, c->stream));
+        c->launches += 4;
+        c->J = n_jobs;
+        c->f_valid = false;
+        c->elites_valid = false;
+        return ONES_OK;
     }
     const int64_t new_ld = ld_of(n_jobs);
     CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(n_jobs), c->tab.kmin,

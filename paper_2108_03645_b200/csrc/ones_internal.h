@@ -112,6 +112,13 @@ cudaError_t launch_fill_slot_limits(int32_t* kmin, int32_t* range, int32_t len, 
 cudaError_t launch_best_per_gpu(const int32_t* pop, int64_t ld, int32_t n_gpus, int32_t n_jobs, const int32_t* best_index,
                                 Tables t, int32_t* work, int32_t* genome_out, int32_t* gpus_out, double* rate_out,
                                 BestOut* out, cudaStream_t s);
+// "Refresh" of every per-GPU candidate at a job-set change (tables, fit and remap are those of the new job
+// set, n_old the size of the old one); inv: n_old entries, newcum: n_jobs + 1 entries of scratch.  Two launches.
+// Needs refresh_smem(n_gpus, n_jobs) <= kMaxSmemPerBlock - 1024 bytes of shared memory per CTA.
+size_t refresh_smem(int32_t n_gpus, int32_t n_jobs);
+cudaError_t launch_refresh_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_old, int32_t n_jobs,
+                                   Tables t, const int4* fit, const int32_t* remap, int32_t* inv, int32_t* newcum,
+                                   cudaStream_t s);
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,

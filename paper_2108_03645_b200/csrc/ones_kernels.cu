@@ -2153,6 +2153,317 @@ cudaError_t launch_best_per_gpu(const int32_t* pop, int64_t ld, int32_t n_gpus, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// "Refresh" of per-GPU candidates when the job set changes (Section 3.2.2, Fig. 5), one CTA per candidate:
+//   (1) GPUs of finished jobs become idle, surviving jobs take their new ids (inv[old id] = new id or -1);
+//   (2) a job holding more GPUs than its batch-size limit needs gives up the surplus, last GPUs first;
+//   (3) every new job, in index order, gets the GPUs of its smallest batch: the lowest idle GPUs, and once
+//       none is idle the last GPU of the lowest-index surviving job that still holds one;
+//   (4) the idle GPUs that remain go to the jobs below their limit in the order of the score they would
+//       gain by growing to it (ties: lower index), each taking what it needs for that, lowest GPUs first.
+// Each step is a sequential rule; here every GPU slot decides on its own from three numbers: its rank among
+// the slots of its job (which of them are "last"), its rank among the idle slots (which are "lowest"), and
+// prefix sums over the jobs in the order they are served ("unit" u of step (3) belongs to the new job whose
+// range of the running sum of smallest-batch needs holds u; units beyond the idle GPUs are taken from the
+// surviving jobs in index order, each job's GPUs from its last one down).  Step (4) serves every job at most
+// once and a job's gain does not change while others are served, so it is one sort by gain.
+// The row is not packed here: "Reorder" runs afterwards.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kScanSat = 1u << 30;  // prefix sums saturate here (far above any GPU count)
+
+__device__ __forceinline__ int32_t sat_add(int32_t a, int32_t b) {
+    return (int32_t)min((uint32_t)a + (uint32_t)b, kScanSat);
+}
+
+// Exclusive prefix sums of the non-negative a[0..n) in shared memory, in place, by a block of 256 threads;
+// returns the total to every thread.
+__device__ int32_t block_scan_excl(int32_t* __restrict__ a, int32_t n, int32_t* __restrict__ s_warp) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t chunk = ((n + 255) / 256) | 1;
+    const int32_t from = min(n, tid * chunk), to = min(n, from + chunk);
+    int32_t mine = 0;
+    for (int32_t i = from; i < to; ++i) mine = sat_add(mine, a[i]);
+    int32_t incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl = sat_add(incl, up);
+    }
+    int32_t excl = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
+    if (lane == 0) excl = 0;
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int32_t offset = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const int32_t v = s_warp[w];
+        if (w < warp) offset = sat_add(offset, v);
+        total = sat_add(total, v);
+    }
+    int32_t run = sat_add(offset, excl);
+    for (int32_t i = from; i < to; ++i) {
+        const int32_t v = a[i];
+        a[i] = run;
+        run = sat_add(run, v);
+    }
+    __syncthreads();
+    return total;
+}
+
+// largest p in [0, n) with a[p] <= v, for non-decreasing a with a[0] <= v
+__device__ __forceinline__ int32_t last_at_most(const int32_t* __restrict__ a, int32_t n, int32_t v) {
+    int32_t lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) >> 1;
+        if (a[mid] <= v) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Once per job-set change: inv[old id] = the new id of a surviving job (the highest, should several claim
+// one old job) or -1, and newcum[j] = the GPUs that the new jobs before j need for their smallest batch
+// (newcum[n_jobs] = all of them), capped at the cluster's size: needs beyond it can never be met.
+__global__ void __launch_bounds__(256)
+k_refresh_prepare(const int32_t* __restrict__ remap, int32_t n_old, int32_t n_jobs, const int4* __restrict__ fit,
+                  int32_t n_gpus, int32_t* __restrict__ inv, int32_t* __restrict__ newcum) {
+    __shared__ int32_t s_warp[8];
+    __shared__ int32_t s_carry;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int32_t o = tid; o < n_old; o += 256) inv[o] = -1;
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int32_t j = tid; j < n_jobs; j += 256) {
+        const int32_t r = remap[j];
+        if (r >= 0 && r < n_old) atomicMax(&inv[r], j);
+    }
+    for (int32_t base = 0; base < n_jobs; base += 256) {
+        const int32_t j = base + tid;
+        int32_t want = 0;
+        if (j < n_jobs && remap[j] < 0) {
+            const int4 q = fit[slot_of(j)];  // b0, max_per_gpu, kmin, kmax
+            const long long b = (long long)q.x << q.z, m = q.y;
+            const long long g = (b + m - 1) / m;
+            want = (int32_t)(g < (long long)n_gpus ? g : (long long)n_gpus);
+        }
+        int32_t incl = want;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl = sat_add(incl, up);
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        int32_t offset = s_carry, total = s_carry;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const int32_t v = s_warp[w];
+            if (w < warp) offset = sat_add(offset, v);
+            total = sat_add(total, v);
+        }
+        const int32_t before = sat_add(offset, incl - want);  // incl - want is exact unless incl saturated,
+        if (j < n_jobs) newcum[j] = min(before, n_gpus);      // and then both exceed the cap anyway
+        __syncthreads();
+        if (tid == 0) s_carry = total;
+        __syncthreads();
+    }
+    if (tid == 0) newcum[n_jobs] = min(s_carry, n_gpus);
+}
+
+static int32_t refresh_sort_len(int32_t n_jobs) {
+    int32_t j2 = 2;
+    while (j2 < n_jobs) j2 <<= 1;
+    return j2;
+}
+
+size_t refresh_smem(int32_t n_gpus, int32_t n_jobs) {
+    const size_t jp = (size_t)((n_jobs + 3) & ~3), wp = (size_t)((n_gpus + 3) & ~3), j2 = (size_t)refresh_sort_len(n_jobs);
+    return 12 * j2 + 4 * (j2 + 4) + 4 * (4 * jp + 2 * wp);
+}
+
+__global__ void __launch_bounds__(256)
+k_refresh_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_old, int32_t n_jobs,
+                  Tables t, const int4* __restrict__ fit, const int32_t* __restrict__ remap,
+                  const int32_t* __restrict__ inv, const int32_t* __restrict__ newcum, int32_t j2) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int32_t s_warp[8];
+    const int32_t jp = (n_jobs + 3) & ~3, wp = (n_gpus + 3) & ~3;
+    double* key = reinterpret_cast<double*>(smem_raw);  // step (4): gain of the job at this place of the order
+    int32_t* sj = reinterpret_cast<int32_t*>(key + j2);  //           and the job itself
+    int32_t* cum = sj + j2;                              // prefix sums over jobs (j2 + 4 entries)
+    int32_t* count = cum + j2 + 4;                       // GPUs held by each job
+    int32_t* first = count + jp;                         // its first and last slot
+    int32_t* last = first + jp;
+    int32_t* lim = last + jp;                            // GPUs its batch-size limit needs
+    int32_t* row = lim + jp;                             // the candidate
+    int32_t* rk = row + wp;                              // occupied slot: rank among its job's slots; idle: among the idle
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t U = newcum[n_jobs];
+    const int32_t chunk = ((n_gpus + 255) / 256) | 1;
+    const int32_t from = min(n_gpus, tid * chunk), to = min(n_gpus, from + chunk);
+    for (int32_t j = tid; j < n_jobs; j += 256) {
+        const int32_t at = slot_of(j);
+        lim[j] = t.G[(int64_t)fit[at].w * t.jpad + at];
+    }
+    for (int64_t cand = blockIdx.x; cand < n; cand += gridDim.x) {
+        int32_t* grow = slots + cand * ld;
+        for (int32_t j = tid; j < n_jobs; j += 256) {
+            count[j] = 0;
+            first[j] = 0x7FFFFFFF;
+            last[j] = -1;
+        }
+        __syncthreads();
+        // (1) new ids; GPUs, first and last slot of every job
+        for (int32_t i = tid; i < n_gpus; i += 256) {
+            const int32_t o = grow[i];
+            const int32_t id = (uint32_t)o < (uint32_t)n_old ? __ldg(inv + o) : -1;
+            row[i] = id;
+            if (id >= 0) {
+                atomicAdd(&count[id], 1);
+                atomicMin(&first[id], i);
+                atomicMax(&last[id], i);
+            }
+        }
+        __syncthreads();
+        // rank of a slot among the slots of its job: the distance from the first one when they are neighbours
+        // (every row this library writes is packed), else counted by one thread per such job
+        for (int32_t i = tid; i < n_gpus; i += 256) {
+            const int32_t id = row[i];
+            rk[i] = id >= 0 ? i - first[id] : 0;
+        }
+        __syncthreads();
+        for (int32_t j = tid; j < n_jobs; j += 256) {
+            const int32_t c = count[j];
+            if (c > 0 && last[j] - first[j] + 1 != c) {
+                int32_t r = 0;
+                for (int32_t i = first[j]; i <= last[j]; ++i)
+                    if (row[i] == j) rk[i] = r++;
+            }
+        }
+        __syncthreads();
+        // (2) scale down to the limit: the slots of rank >= limit are the last ones
+        for (int32_t i = tid; i < n_gpus; i += 256) {
+            const int32_t id = row[i];
+            if (id >= 0 && rk[i] >= lim[id]) row[i] = -1;
+        }
+        for (int32_t j = tid; j < n_jobs; j += 256) {
+            const int32_t kept = min(count[j], lim[j]);
+            count[j] = kept;
+            cum[j] = __ldg(remap + j) < 0 ? 0 : kept;  // what step (3) may take from the jobs before j
+        }
+        __syncthreads();
+        const int32_t V = block_scan_excl(cum, n_jobs, s_warp);
+        // rank of every idle slot among the idle ones
+        int32_t idle_mine = 0;
+        for (int32_t i = from; i < to; ++i) idle_mine += row[i] < 0;
+        int32_t incl = idle_mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        int32_t idle_before = incl - idle_mine, n_idle = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const int32_t v = s_warp[w];
+            if (w < warp) idle_before += v;
+            n_idle += v;
+        }
+        for (int32_t i = from; i < to; ++i)
+            if (row[i] < 0) rk[i] = idle_before++;
+        __syncthreads();
+        // (3) the new jobs' units: u < n_idle is the u-th idle slot, the others are taken from surviving jobs
+        const int32_t granted = min(U, n_idle + V);
+        const int32_t taken = max(0, granted - n_idle);
+        for (int32_t i = tid; i < n_gpus; i += 256) {
+            const int32_t id = row[i];
+            int32_t unit = -1;
+            if (id < 0) {
+                if (rk[i] < U) unit = rk[i];
+            } else if (__ldg(remap + id) >= 0) {
+                const int32_t turn = cum[id] + (count[id] - 1 - rk[i]);  // its place in the order GPUs are taken
+                if (turn < taken) unit = n_idle + turn;
+            }
+            if (unit >= 0) row[i] = last_at_most(newcum, n_jobs + 1, unit);
+        }
+        __syncthreads();
+        for (int32_t j = tid; j < n_jobs; j += 256) {
+            if (__ldg(remap + j) < 0) count[j] = min(newcum[j + 1], granted) - min(newcum[j], granted);
+            else count[j] -= min(max(taken - cum[j], 0), count[j]);
+        }
+        __syncthreads();
+        // (4) refill what is still idle (block-uniform condition)
+        if (n_idle > U) {
+            for (int32_t s = tid; s < j2; s += 256) {
+                double gain = -CUDART_INF;
+                int32_t who = 0x40000000 + s;
+                if (s < n_jobs && count[s] < lim[s]) {
+                    const int32_t at = slot_of(s);
+                    const int4 q = __ldg(fit + at);
+                    const int32_t k = count[s] > 0 ? exponent_that_fits(q.x, q.y, q.z, q.w, count[s]) : -1;
+                    const double now = k >= 0 ? t.X[(int64_t)k * t.jpad + at] : 0.0;
+                    gain = __dsub_rn(t.X[(int64_t)q.w * t.jpad + at], now);
+                    who = s;
+                }
+                key[s] = gain;
+                sj[s] = who;
+            }
+            __syncthreads();
+            for (int32_t k = 2; k <= j2; k <<= 1)
+                for (int32_t d = k >> 1; d > 0; d >>= 1) {
+                    for (int32_t s = tid; s < j2; s += 256) {
+                        const int32_t p = s ^ d;
+                        if (p > s) {
+                            const double ka = key[s], kb = key[p];
+                            const int32_t ja = sj[s], jb = sj[p];
+                            const bool b_first = kb > ka || (kb == ka && jb < ja);  // p's job is served before s's
+                            const bool a_first = ka > kb || (ka == kb && ja < jb);
+                            if (((s & k) == 0) ? b_first : a_first) {
+                                key[s] = kb; key[p] = ka;
+                                sj[s] = jb; sj[p] = ja;
+                            }
+                        }
+                    }
+                    __syncthreads();
+                }
+            for (int32_t s = tid; s < j2; s += 256) {
+                const int32_t j = sj[s];
+                cum[s] = j < n_jobs ? min(lim[j] - count[j], n_gpus) : 0;
+            }
+            __syncthreads();
+            const int32_t wanted = block_scan_excl(cum, j2, s_warp);
+            for (int32_t i = tid; i < n_gpus; i += 256) {
+                if (row[i] < 0) {
+                    const int32_t r = rk[i] - U;
+                    if (r >= 0 && r < wanted) row[i] = sj[last_at_most(cum, j2, r)];
+                }
+            }
+            __syncthreads();
+        }
+        for (int32_t i = tid; i < n_gpus; i += 256) grow[i] = row[i];
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_refresh_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_old, int32_t n_jobs,
+                                   Tables t, const int4* fit, const int32_t* remap, int32_t* inv, int32_t* newcum,
+                                   cudaStream_t s) {
+    const size_t smem = refresh_smem(n_gpus, n_jobs);
+    if (smem > (size_t)kMaxSmemPerBlock - 1024) return cudaErrorInvalidConfiguration;
+    k_refresh_prepare<<<1, 256, 0, s>>>(remap, n_old, n_jobs, fit, n_gpus, inv, newcum);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || n <= 0) return e;
+    e = cudaFuncSetAttribute(k_refresh_per_gpu, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = n;
+    if (blocks > (int64_t)kSMs * 4) blocks = (int64_t)kSMs * 4;
+    k_refresh_per_gpu<<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_old, n_jobs, t, fit, remap, inv, newcum,
+                                                      refresh_sort_len(n_jobs));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Best candidate and its repair to the cluster's capacity: one block.
 // work[0..jpad) exponent, work[jpad..2jpad) GPUs now, work[2jpad..3jpad) GPUs one exponent lower
 // (-1 when the job cannot shrink).

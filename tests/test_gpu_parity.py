@@ -335,7 +335,77 @@ def test_per_gpu_genome_parity(ones, J, gpus, N, kw):
     Fo, Go = o.evaluate(rows)
     assert (Fg.cpu().numpy() == Fo).all() and (Gg.cpu().numpy() == Go).all()
     with pytest.raises(ones.OnesError):
-        g.update_jobs(w.jobs, np.arange(J, dtype=np.int32), gpus)
+        g.update_jobs(w.jobs, np.arange(J, dtype=np.int32), gpus + 1)  # the cluster keeps its size
+
+
+def _changed_job_set(rng, jobs, n_leave, n_new, seed, kmax_new=0, shuffle=False):
+    """Some jobs finish, limits move by -1..+1 exponents, new jobs join; returns (jobs, remap)."""
+    J = jobs.shape[0]
+    keep = sorted(rng.choice(J, size=J - n_leave, replace=False).tolist())
+    fresh = inputs.custom(max(n_new, 1), 8, 4, 1, seed=seed, kmax=kmax_new, kmin_max=min(1, kmax_new)).jobs[:n_new]
+    new = np.concatenate([jobs[keep], fresh])
+    new["kmax"][:len(keep)] = np.clip(new["kmax"][:len(keep)] + rng.integers(-1, 2, len(keep)), 0, 7)
+    new["kmin"] = np.minimum(new["kmin"], new["kmax"])
+    remap = np.array(keep + [-1] * n_new, dtype=np.int32)
+    if shuffle:  # new jobs anywhere in the table
+        order = rng.permutation(new.shape[0])
+        new, remap = new[order], remap[order]
+    return new, remap
+
+
+@pytest.mark.parametrize("J,gpus,N,leave,arrive,kw", [
+    (6, 12, 64, 2, 2, {}),                                   # small: finished jobs, new jobs, refill
+    (100, 64, 300, 13, 20, {}),                              # more new jobs than GPUs free up: GPUs are taken
+    (37, 130, 101, 5, 3, dict(flags=1)),                     # SRUF terms: gains of either sign
+    (5, 3, 9, 1, 6, {}),                                     # more new jobs than GPUs
+    (300, 257, 129, 0, 0, {}),                               # only the limits move
+    (64, 1027, 40, 60, 1, {}),                               # the cluster empties: one big refill
+    (2048, 4096, 150, 200, 150, dict(p_mut=0.02)),           # benchmark shape
+    (40, 4100, 33, 7, 9, {}),                                # rows above 4096 slots
+])
+def test_per_gpu_refresh_parity(ones, J, gpus, N, leave, arrive, kw):
+    """ones_update_jobs on per-GPU candidates = the oracle's Refresh + Reorder, row by row."""
+    flags = 16 | kw.pop("flags", 0)
+    w = inputs.custom(J, gpus, N, 4, seed=J + N, kmax=6, kmin_max=1)
+    p = inputs.SearchParams(flags=flags, **kw)
+    g = ones.Search(w.jobs, gpus, N, p, n_jobs_max=J + 3 * arrive + 8)
+    o = oracle.Search(w.jobs, gpus, N, elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut, penalty=p.penalty,
+                      flags=flags)
+    g.randomize(3)
+    o.randomize(3)
+    g.evolve(2, 13)
+    o.evolve(2, 13)
+    rng = np.random.default_rng(J + gpus)
+    jobs = w.jobs
+    for rnd in range(3):
+        if rnd == 1:
+            # rows from outside: unpacked, with idle and out-of-range ids (ranks are then counted, not derived)
+            rows = rng.integers(-2, jobs.shape[0] + 2, size=(N, gpus)).astype(np.int32)
+            rows[: N // 3] = np.sort(rows[: N // 3], axis=1)
+            g.set_population(rows)
+            o.set_population(rows)
+        jobs2, remap = _changed_job_set(rng, jobs, min(leave, jobs.shape[0] - 1), arrive, seed=50 + rnd,
+                                        kmax_new=rnd, shuffle=rnd == 2)
+        g.update_jobs(jobs2, remap, gpus)
+        o.update_jobs(jobs2, remap, gpus)
+        assert (g.get_population() == o.get_population()).all(), rnd
+        _same_state(g, o)
+        g.evolve(2, rnd)
+        o.evolve(2, rnd)
+        _same_state(g, o)
+        jobs = jobs2
+    bg, bo = g.best(), o.best()
+    assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
+
+
+def test_per_gpu_refresh_limits(ones):
+    w = inputs.custom(6, 12, 8, 1, seed=1, kmax=3)
+    g = ones.Search(w.jobs, 12, 8, inputs.SearchParams(flags=16), n_jobs_max=8)
+    with pytest.raises(ones.OnesError) as err:   # more jobs than the workspace was sized for
+        g.update_jobs(np.concatenate([w.jobs] * 4), np.full(24, -1, dtype=np.int32), 12)
+    assert err.value.code == -5
+    g.update_jobs(w.jobs[:4], np.array([0, 1, 1, -1], dtype=np.int32), 12)   # two rows claim old job 1
+    assert ((g.get_population() >= -1) & (g.get_population() < 4)).all()
 
 
 # ---- a6: best and repair ---------------------------------------------------------------------------
