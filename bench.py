@@ -220,6 +220,16 @@ def run_online(args):
     print(json.dumps(line))
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of this
+# benchmark's default workload at its full population (profiles/dram_traffic_large_pop65536.md).  They belong
+# to the kernels as they were when the capture was taken: set an entry to None when its kernel changes.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("large", 65536, "k_evolve_score"): 403.6e6 + 485.2e6,
+    ("large", 65536, "k_evolve"): 401.6e6 + 483.0e6,
+    ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
+}
+
+
 # ----------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -411,7 +421,8 @@ def main():
         kernel = "k_evolve_cluster" if launches < steps else ("k_generation" if one_launch else "k_evolve_score")
         ach = fused_bytes * gens_per_launch / (ev_ms * 1e-3) / 1e9
         line["roofline"] = {"kernel": kernel, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                            "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                            "frac": ach / peak, "peak_kind": f"of {peak_kind}",
+                            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, N, kernel)),
                             "bytes_per_launch": fused_bytes * gens_per_launch, "ms_per_launch": ev_ms,
                             "generations_per_launch": gens_per_launch,
                             "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
@@ -428,6 +439,7 @@ def main():
                 a = nbytes / (t_ms * 1e-3) / 1e9
                 line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
                                          "bytes_per_launch": nbytes, "ms_per_launch": t_ms,
+                                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, N, name)),
                                          "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
                                          "how": "same workload with ONES_FLAG_UNFUSED (separate scoring pass)"}
     if base is not None:
