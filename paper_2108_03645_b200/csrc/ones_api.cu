@@ -103,6 +103,7 @@ struct ones_ctx {
     int gcur = 0;           // GPU-count buffer in force (only the truncation scheme alternates it)
     bool trunc = false;     // ONES_FLAG_TRUNCATION
     bool per_gpu = false;   // ONES_FLAG_PER_GPU: one gene per GPU (a job id) instead of one per job
+    bool narrow = false;    // per-GPU genome: capacity * max_per_gpu < 2^31 for every job (32-bit exponent search)
     int32_t W = 0;          // genes per candidate
     Tables tabS{};          // as tab, with the limits of a slot (any job id) for the shared operators
     int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
@@ -210,6 +211,9 @@ void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
     c->fused = narrow && !(c->prm.flags & ONES_FLAG_UNFUSED) && evolve_score_smem(c->tab) <= (size_t)kMaxSmemPerBlock;
     c->tabS = c->tab;
     if (c->per_gpu) {
+        c->narrow = true;
+        for (int32_t j = 0; j < n_jobs; ++j)
+            if ((int64_t)c->W * jobs[j].max_per_gpu >= ((int64_t)1 << 31)) c->narrow = false;
         c->tabS.kmin = reinterpret_cast<int32_t*>(c->ws + c->L.slot_kmin);
         c->tabS.range = reinterpret_cast<int32_t*>(c->ws + c->L.slot_range);
         c->fused = false;  // scoring a per-GPU candidate needs its job counts: separate kernel
@@ -259,7 +263,7 @@ int run_fitness(ones_ctx* c) {
     int rc = prof_begin(c, 0);
     if (rc) return rc;
     if (c->per_gpu)
-        CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->F(), c->G(), c->stream));
+        CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->narrow, c->F(), c->G(), c->stream));
     else
         CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
                              c->stream));
@@ -477,7 +481,7 @@ int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, 
     int rc = prof_begin(c, 0);
     if (rc) return rc;
     if (c->per_gpu)
-        CU(c, launch_fitness_per_gpu(d_genomes, ld, n, c->W, c->J, c->tab, c->fit(), d_fitness, d_gpus, c->stream));
+        CU(c, launch_fitness_per_gpu(d_genomes, ld, n, c->W, c->J, c->tab, c->fit(), c->narrow, d_fitness, d_gpus, c->stream));
     else
         CU(c, launch_fitness(d_genomes, ld, n, c->J, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
     c->launches += 1;
@@ -592,7 +596,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         if (c->per_gpu) {
             // "Reorder" packs each job's workers in every new candidate; the same pass scores it
             if ((rc = prof_begin(c, 0)) != ONES_OK) return rc;
-            CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->F(), c->G(), c->stream));
+            CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->narrow, c->F(), c->G(), c->stream));
             c->launches += 1;
             c->f_valid = true;
             if ((rc = prof_end(c)) != ONES_OK) return rc;

@@ -101,12 +101,13 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
                                 const int32_t* G, double* F_next, int32_t* G_next, void* scratch,
                                 cudaStream_t s);  // 12 launches
 // The paper's per-GPU genome (ONES_FLAG_PER_GPU): scoring, the reorder operation, slot limits, best
+// narrow: n_gpus * max_per_gpu < 2^31 for every job, so the exponent search may use 32-bit arithmetic
 cudaError_t launch_fitness_per_gpu(const int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs,
-                                   Tables t, const int4* fit, double* F, int32_t* G, cudaStream_t s);
+                                   Tables t, const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s);
 cudaError_t launch_reorder(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, cudaStream_t s);
 // reorder and score in one pass over the rows
 cudaError_t launch_reorder_score(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                 const int4* fit, double* F, int32_t* G, cudaStream_t s);
+                                 const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s);
 cudaError_t launch_fill_slot_limits(int32_t* kmin, int32_t* range, int32_t len, int32_t n_gpus, int32_t n_jobs,
                                     const ones_job* jobs, int4* fit, int32_t jpad, cudaStream_t s);
 cudaError_t launch_best_per_gpu(const int32_t* pop, int64_t ld, int32_t n_gpus, int32_t n_jobs, const int32_t* best_index,

@@ -61,6 +61,31 @@ __host__ __device__ __forceinline__ int32_t slot_of(int32_t j) {
     return (j & ~127) + ((j & 3) << 5) + ((j >> 2) & 31);
 }
 
+// Programmatic dependent launch.  A kernel launched with launch_after_previous() may become resident while
+// the kernel before it in the stream is still running; everything it does before grid_dependency_wait()
+// (staging the model tables, which no kernel of the generation loop writes) overlaps that kernel, and
+// nothing written by it is touched until the wait returns, which is when the previous kernel has completed
+// and its writes are visible.  grid_dependency_release() lets the next kernel's CTAs become resident early in
+// the same way.  Launched normally, a kernel passes the wait at once.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... Params, typename... Args>
+static cudaError_t launch_after_previous(void (*kernel)(Params...), int blocks, int threads, size_t smem, cudaStream_t s,
+                                         Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Model tables: X_j(k), g_j(k) for every job and exponent (throughput model of the job table)
 // ---------------------------------------------------------------------------------------------
@@ -516,6 +541,7 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
                uint32_t gen_lo, uint32_t c3a, uint32_t c3b, int32_t* __restrict__ parents, int32_t e,
                int32_t top_blocks, int32_t per_block, Rec* __restrict__ partial, int32_t* __restrict__ elites,
                unsigned int* __restrict__ done) {
+    grid_dependency_wait();  // the scores come from the kernel before
     if ((int32_t)blockIdx.x >= top_blocks) {
         const int32_t i = ((int32_t)blockIdx.x - top_blocks) * blockDim.x + threadIdx.x;
         if (i < 2 * pairs) tournament_thread(F, n, tournament, i, keys, gen_lo, (i & 1) ? c3b : c3a, parents);
@@ -539,6 +565,9 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
             break;
         }
     }
+    // from here on only the merging CTA still works: the next kernel's CTAs may take the other SMs (they
+    // arrive once every tournament CTA has ended and every top-e CTA is here)
+    grid_dependency_release();
     __threadfence();  // every thread's records before the CTA is counted as finished
     __syncthreads();
     if (threadIdx.x == 0) s_last = atomicAdd(done, 1u) == (unsigned int)(top_blocks - 1);
@@ -562,10 +591,9 @@ cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, 
     const int sel_b = (2 * pairs + 255) / 256;
     if (top_b + sel_b == 0) return cudaSuccess;
     const int32_t per_block = top_b ? (n + top_b - 1) / top_b : 0;
-    k_select_stage<<<top_b + sel_b, 256, 0, s>>>(F, n, tournament, pairs, keys, (uint32_t)gen,
-                                                 counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), parents, e,
-                                                 top_b, per_block, reinterpret_cast<Rec*>(scratch), elites, done);
-    return cudaGetLastError();
+    return launch_after_previous(k_select_stage, top_b + sel_b, 256, 0, s, F, n, tournament, pairs, keys, (uint32_t)gen,
+                                 counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), parents, e, (int32_t)top_b,
+                                 per_block, reinterpret_cast<Rec*>(scratch), elites, done);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -726,6 +754,10 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
         }
         __syncthreads();
     }
+    // parents and elites come from the selection stage, the rows from the generation before.  No early
+    // release here: the next selection stage's CTAs would take SMs as they free up and the tail of this
+    // kernel measured 3 % slower at the largest population.
+    grid_dependency_wait();
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
@@ -893,6 +925,8 @@ k_generation(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t
         }
         __syncthreads();
     }
+    grid_dependency_wait();  // scores, elites and rows come from the generation before
+    grid_dependency_release();  // measured: the next generation's CTAs best become resident as early as they can
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
@@ -1080,11 +1114,10 @@ cudaError_t launch_generation(GenerationShape shape, const int32_t* src, int32_t
     kern = always ? k_generation<256, 1, true> : k_generation<256, 1, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shape.smem);
     if (e != cudaSuccess) return e;
-    kern<<<shape.blocks, shape.threads, shape.smem, s>>>(
-        src, dst, ld, n, n_jobs, elitism, pairs, tournament, F_old, F_new, G, parents, elites, elites_next, t, keys,
-        (uint32_t)gen, counter3(STREAM_MUT, gen), counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), thr32,
-        capacity, penalty, reinterpret_cast<Rec*>(scratch), done, shape.queue_cap);
-    return cudaGetLastError();
+    return launch_after_previous(kern, shape.blocks, shape.threads, shape.smem, s, src, dst, ld, n, n_jobs, elitism, pairs,
+                                 tournament, F_old, F_new, G, parents, elites, elites_next, t, keys, (uint32_t)gen,
+                                 counter3(STREAM_MUT, gen), counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), thr32,
+                                 capacity, penalty, reinterpret_cast<Rec*>(scratch), done, shape.queue_cap);
 }
 
 size_t evolve_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (size_t)t.jpad * 8; }
@@ -1104,9 +1137,8 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
     auto kern = thr16 >= 65536u ? k_evolve_score<kThreads, 1, true> : k_evolve_score<kThreads, 1, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
-    kern<<<(int)blocks, kThreads, smem, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
-                                             (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G);
-    return cudaGetLastError();
+    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, src, dst, ld, n, n_jobs, elitism, pairs, parents,
+                                 elites, t, keys, (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1716,9 +1748,20 @@ __device__ __forceinline__ int32_t exponent_that_fits(int32_t b0, int32_t m, int
     return k >= kmin ? k : -1;
 }
 
+// The same in 32-bit arithmetic, for clusters with count * max_per_gpu < 2^31 for every job.
+__device__ __forceinline__ int32_t exponent_that_fits32(int32_t b0, int32_t m, int32_t kmin, int32_t kmax, int32_t count) {
+    const uint32_t room = (uint32_t)count * (uint32_t)m;
+    if (room < (uint32_t)b0) return -1;
+    int32_t k = __clz(b0) - __clz((int32_t)room);
+    if (((uint32_t)b0 << k) > room) --k;
+    k = min(k, kmax);
+    return k >= kmin ? k : -1;
+}
+
 // Per-job terms of one per-GPU candidate from its job counts (shared memory), 256 threads.  A thread
 // takes jobs 4v..4v+3: their counts are one int4, and for each of the four the lanes of a warp read
 // neighbouring entries of the limits and of the model tables (the tables' job order).  Returns the GPUs used.
+template <bool NARROW = false>
 __device__ __forceinline__ int32_t per_gpu_terms(const int32_t* __restrict__ count, double* __restrict__ term,
                                                  int32_t jpad4, const Tables& t, const int4* __restrict__ fit) {
     int32_t used = 0;
@@ -1739,7 +1782,8 @@ __device__ __forceinline__ int32_t per_gpu_terms(const int32_t* __restrict__ cou
             at[e] = -1;
             if (c[e] > 0) {
                 const int4 q = __ldg(fit + entry);  // b0, max_per_gpu, kmin, kmax
-                const int32_t k = exponent_that_fits(q.x, q.y, q.z, q.w, c[e]);
+                const int32_t k = NARROW ? exponent_that_fits32(q.x, q.y, q.z, q.w, c[e])
+                                         : exponent_that_fits(q.x, q.y, q.z, q.w, c[e]);
                 if (k >= 0) at[e] = k * t.jpad + entry;
             }
         }
@@ -1889,8 +1933,15 @@ k_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, in
 
 // The same for rows of at most 256 * PIECE slots: every thread keeps its PIECE neighbouring slots in
 // registers, so the row is read once from global memory and walked without loops over shared memory.
+// RUNS: a thread adds a whole run of equal ids at once (few jobs on many GPUs: long runs, where one atomic
+// per slot would hit the same counter from every lane); otherwise one atomic per slot (after crossover the
+// runs are one or two slots long and the run bookkeeping costs more instructions than it saves).
+// Reorder: the first slot of every job learns where the job's run starts (exclusive scan, over the slots, of
+// the GPU counts of the jobs that start there) and leaves it in first[]; then every slot (or run) takes its
+// place in the job's run with one atomic add on that cursor, so no thread loops over a job's whole run.
+// NARROW: the exponent search in 32-bit arithmetic.
 // Shared memory: count[J] | first[J] | the reordered row, later the per-job terms (fp64).
-template <int PIECE, bool REORDER, bool SCORE>
+template <int PIECE, bool REORDER, bool SCORE, bool RUNS, bool NARROW>
 __global__ void __launch_bounds__(256, 4)
 k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
                const int4* __restrict__ fit, double* __restrict__ F, int32_t* __restrict__ G) {
@@ -1929,7 +1980,7 @@ k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpu
         }
         if (tid == 0) s_used = 0;
         __syncthreads();
-        {   // one atomic per run of equal ids
+        if (RUNS) {  // one atomic per run of equal ids
             int32_t run_id = -1, run_len = 0, run_at = 0;
 #pragma unroll
             for (int u = 0; u <= PIECE; ++u) {
@@ -1945,6 +1996,13 @@ k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpu
                 }
                 ++run_len;
             }
+        } else {
+#pragma unroll
+            for (int u = 0; u < PIECE; ++u)
+                if (id[u] >= 0) {
+                    atomicAdd(&count[id[u]], 1);
+                    if (REORDER) atomicMin(&first[id[u]], from + u);
+                }
         }
         __syncthreads();
         if (REORDER) {
@@ -1964,7 +2022,7 @@ k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpu
                 if (lane >= off) incl += up;
             }
             if (lane == 31) s_warp[warp] = incl;
-            __syncthreads();
+            __syncthreads();  // every thread has read first[] by now: it becomes the jobs' write cursors
             int32_t offset = incl - mine, total = 0;
 #pragma unroll
             for (int w = 0; w < 8; ++w) {
@@ -1973,11 +2031,33 @@ k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpu
                 total += v;
             }
 #pragma unroll
-            for (int u = 0; u < PIECE; ++u) {
-                for (int32_t r = 0; r < c[u]; ++r) out[offset + r] = id[u];
-                offset += c[u];
-            }
+            for (int u = 0; u < PIECE; ++u)
+                if (c[u] > 0) {
+                    first[id[u]] = offset;
+                    offset += c[u];
+                }
             for (int32_t i = total + tid; i < n_gpus; i += 256) out[i] = -1;  // idle GPUs last
+            __syncthreads();
+            if (RUNS) {
+                int32_t run_id = -1, run_len = 0;
+#pragma unroll
+                for (int u = 0; u <= PIECE; ++u) {
+                    const int32_t v = u < PIECE ? id[u] : -2;
+                    if (v != run_id) {
+                        if (run_id >= 0) {
+                            const int32_t dest = atomicAdd(&first[run_id], run_len);
+                            for (int32_t r = 0; r < run_len; ++r) out[dest + r] = run_id;
+                        }
+                        run_id = v;
+                        run_len = 0;
+                    }
+                    ++run_len;
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < PIECE; ++u)
+                    if (id[u] >= 0) out[atomicAdd(&first[id[u]], 1)] = id[u];
+            }
             if (cand + gridDim.x < n) fetch(cand + gridDim.x);
             __syncthreads();
             for (int32_t i = 4 * tid; i < n_gpus; i += 4 * 256) {
@@ -1991,7 +2071,7 @@ k_per_gpu_regs(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_gpu
         }
         if (!REORDER && cand + gridDim.x < n) fetch(cand + gridDim.x);
         if (SCORE) {
-            int32_t used = per_gpu_terms(count, term, jpad4, t, fit);
+            int32_t used = per_gpu_terms<NARROW>(count, term, jpad4, t, fit);
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) used += __shfl_xor_sync(0xFFFFFFFFu, used, off);
             if (lane == 0 && used) atomicAdd(&s_used, used);
@@ -2022,17 +2102,31 @@ static size_t per_gpu_regs_smem(int32_t n_gpus, int32_t n_jobs) {
     return 2 * jpad4 * 4 + tail;
 }
 
-template <int PIECE, bool REORDER, bool SCORE>
-static cudaError_t launch_per_gpu_regs(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                       const int4* fit, double* F, int32_t* G, cudaStream_t s) {
+template <int PIECE, bool REORDER, bool SCORE, bool RUNS, bool NARROW>
+static cudaError_t launch_per_gpu_regs_t(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+                                         const int4* fit, double* F, int32_t* G, cudaStream_t s) {
     const size_t smem = per_gpu_regs_smem(n_gpus, n_jobs);
-    cudaError_t e = cudaFuncSetAttribute(k_per_gpu_regs<PIECE, REORDER, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_per_gpu_regs<PIECE, REORDER, SCORE, RUNS, NARROW>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int64_t blocks = n;
     if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
-    k_per_gpu_regs<PIECE, REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G);
+    k_per_gpu_regs<PIECE, REORDER, SCORE, RUNS, NARROW><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit,
+                                                                                        F, G);
     return cudaGetLastError();
+}
+
+template <int PIECE, bool REORDER, bool SCORE>
+static cudaError_t launch_per_gpu_regs(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
+                                       const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s) {
+    // long runs of equal ids when a job holds many GPUs on average
+    const bool runs = (int64_t)n_gpus >= 8 * (int64_t)n_jobs;
+    narrow = narrow && SCORE;
+    if (runs)
+        return narrow ? launch_per_gpu_regs_t<PIECE, REORDER, SCORE, true, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s)
+                      : launch_per_gpu_regs_t<PIECE, REORDER, SCORE, true, false>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+    return narrow ? launch_per_gpu_regs_t<PIECE, REORDER, SCORE, false, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s)
+                  : launch_per_gpu_regs_t<PIECE, REORDER, SCORE, false, false>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
 }
 
 static size_t per_gpu_smem(int32_t n_gpus, int32_t n_jobs) {
@@ -2041,11 +2135,11 @@ static size_t per_gpu_smem(int32_t n_gpus, int32_t n_jobs) {
 
 template <bool REORDER, bool SCORE>
 static cudaError_t launch_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                  const int4* fit, double* F, int32_t* G, cudaStream_t s) {
+                                  const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     if (per_gpu_regs_smem(n_gpus, n_jobs) <= (size_t)kMaxSmemPerBlock - 2048) {
-        if (n_gpus <= 256 * 4) return launch_per_gpu_regs<4, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
-        if (n_gpus <= 256 * 16) return launch_per_gpu_regs<16, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+        if (n_gpus <= 256 * 4) return launch_per_gpu_regs<4, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, narrow, F, G, s);
+        if (n_gpus <= 256 * 16) return launch_per_gpu_regs<16, REORDER, SCORE>(slots, ld, n, n_gpus, n_jobs, t, fit, narrow, F, G, s);
     }
     const size_t smem = per_gpu_smem(n_gpus, n_jobs);
     if (smem > (size_t)kMaxSmemPerBlock - 2048) return cudaErrorInvalidConfiguration;
@@ -2058,18 +2152,18 @@ static cudaError_t launch_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t
 }
 
 cudaError_t launch_fitness_per_gpu(const int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs,
-                                   Tables t, const int4* fit, double* F, int32_t* G, cudaStream_t s) {
-    return launch_per_gpu<false, true>(const_cast<int32_t*>(slots), ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+                                   Tables t, const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<false, true>(const_cast<int32_t*>(slots), ld, n, n_gpus, n_jobs, t, fit, narrow, F, G, s);
 }
 
 cudaError_t launch_reorder(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, cudaStream_t s) {
     Tables none{};
-    return launch_per_gpu<true, false>(slots, ld, n, n_gpus, n_jobs, none, nullptr, nullptr, nullptr, s);
+    return launch_per_gpu<true, false>(slots, ld, n, n_gpus, n_jobs, none, nullptr, false, nullptr, nullptr, s);
 }
 
 cudaError_t launch_reorder_score(int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs, Tables t,
-                                 const int4* fit, double* F, int32_t* G, cudaStream_t s) {
-    return launch_per_gpu<true, true>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G, s);
+                                 const int4* fit, bool narrow, double* F, int32_t* G, cudaStream_t s) {
+    return launch_per_gpu<true, true>(slots, ld, n, n_gpus, n_jobs, t, fit, narrow, F, G, s);
 }
 
 // admissible values of a slot: any job id (kmin 0, range n_jobs), for the shared operators; and the

@@ -338,6 +338,23 @@ def test_per_gpu_genome_parity(ones, J, gpus, N, kw):
         g.update_jobs(w.jobs, np.arange(J, dtype=np.int32), gpus + 1)  # the cluster keeps its size
 
 
+def test_per_gpu_genome_wide_batches(ones):
+    """Batch sizes and per-GPU limits so large that GPUs x max_per_gpu passes 2^31: the 64-bit exponent search."""
+    w = inputs.custom(50, 600, 80, 2, seed=8, kmax=4, kmin_max=1)
+    w.jobs["b0"] = (w.jobs["b0"].astype(np.int64) << 14).astype(np.int32)          # up to 2^21, << kmax 4 stays below 2^31
+    w.jobs["max_per_gpu"] = (w.jobs["max_per_gpu"].astype(np.int64) << 15).astype(np.int32)   # 2^21 .. 2^23
+    assert 600 * int(w.jobs["max_per_gpu"].max()) >= 2 ** 31
+    g, o = _pair(ones, w, flags=16)
+    g.randomize(1)
+    o.randomize(1)
+    _same_state(g, o)
+    g.evolve(3, 5)
+    o.evolve(3, 5)
+    _same_state(g, o)
+    bg, bo = g.best(), o.best()
+    assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
+
+
 def _changed_job_set(rng, jobs, n_leave, n_new, seed, kmax_new=0, shuffle=False):
     """Some jobs finish, limits move by -1..+1 exponents, new jobs join; returns (jobs, remap)."""
     J = jobs.shape[0]
