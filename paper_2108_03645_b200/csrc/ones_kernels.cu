@@ -445,6 +445,150 @@ __device__ Rec block_next_best(const void* items, int32_t count, int32_t lo, boo
     return r;
 }
 
+// Small e (at most E, E <= 4): every thread keeps the E best of its own items as a sorted list in registers
+// and a warp pops its best e times (butterfly over the heads of the lists; the lane that owned the winner
+// moves its list up), so a slice is read once and the block needs one barrier instead of two per rank.
+template <int E>
+struct TopList {
+    unsigned long long key[E];
+    int32_t idx[E];
+};
+
+// true when record a ranks before record b; a record with idx < 0 is empty and ranks last
+__device__ __forceinline__ bool rec_before(unsigned long long ka, int32_t ia, unsigned long long kb, int32_t ib) {
+    return ia >= 0 && (ib < 0 || before(ka, ia, kb, ib));
+}
+
+template <int E>
+__device__ __forceinline__ void top_list_clear(TopList<E>& l) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        l.key[r] = 0ull;
+        l.idx[r] = -1;
+    }
+}
+
+template <int E>
+__device__ __forceinline__ void top_list_insert(TopList<E>& l, unsigned long long k, int32_t id) {
+    if (!rec_before(k, id, l.key[E - 1], l.idx[E - 1])) return;
+    l.key[E - 1] = k;
+    l.idx[E - 1] = id;
+#pragma unroll
+    for (int r = E - 1; r > 0; --r) {
+        if (rec_before(l.key[r], l.idx[r], l.key[r - 1], l.idx[r - 1])) {
+            const unsigned long long tk = l.key[r];
+            const int32_t ti = l.idx[r];
+            l.key[r] = l.key[r - 1];
+            l.idx[r] = l.idx[r - 1];
+            l.key[r - 1] = tk;
+            l.idx[r - 1] = ti;
+        }
+    }
+}
+
+// The warp's best remaining record (to every lane); its owner drops it from its list.
+template <int E>
+__device__ __forceinline__ Rec warp_pop_best(TopList<E>& l) {
+    Rec best;
+    best.key = l.key[0];
+    best.idx = l.idx[0];
+    best.pad = 0;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xFFFFFFFFu, best.key, off);
+        const int32_t oi = __shfl_xor_sync(0xFFFFFFFFu, best.idx, off);
+        if (rec_before(ok, oi, best.key, best.idx)) {
+            best.key = ok;
+            best.idx = oi;
+        }
+    }
+    if (best.idx >= 0 && l.idx[0] == best.idx) {
+#pragma unroll
+        for (int r = 0; r + 1 < E; ++r) {
+            l.key[r] = l.key[r + 1];
+            l.idx[r] = l.idx[r + 1];
+        }
+        l.key[E - 1] = 0ull;
+        l.idx[E - 1] = -1;
+    }
+    return best;
+}
+
+// The e best (e <= E) of `count` items of one 256-thread block, in rank order, written by thread 0 to out[0..e)
+// (empty records when there are fewer than e items).  SRC 0: the items are scores F[i] with index lo + i;
+// 1: records in global memory, possibly written by other CTAs of the same launch (read through L2, four
+// loads in flight per thread); 2: records in shared memory.  IDX_OUT: out is an int32 array that receives
+// the indices only.  s_list: 8 * E records.
+template <int E, int SRC, bool IDX_OUT = false>
+__device__ __forceinline__ void block_top_small(const void* __restrict__ items, int32_t count, int32_t lo, int32_t e,
+                                                void* __restrict__ out, Rec* __restrict__ s_list) {
+    TopList<E> l;
+    top_list_clear(l);
+    if (SRC == 1) {
+        for (int32_t i0 = threadIdx.x; i0 < count; i0 += 4 * 256) {
+            int4 raw[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * 256 < count) raw[u] = __ldcg(reinterpret_cast<const int4*>(items) + i0 + u * 256);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * 256 < count)
+                    top_list_insert(l, ((unsigned long long)(uint32_t)raw[u].y << 32) | (uint32_t)raw[u].x, raw[u].z);
+        }
+    } else {
+        for (int32_t i = threadIdx.x; i < count; i += 256) {
+            if (SRC == 2) {
+                const Rec q = reinterpret_cast<const Rec*>(items)[i];
+                top_list_insert(l, q.key, q.idx);
+            } else {
+                top_list_insert(l, score_key(reinterpret_cast<const double*>(items)[i]), lo + i);
+            }
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int32_t r = 0; r < e; ++r) {
+        const Rec best = warp_pop_best(l);
+        if (lane == 0) s_list[warp * E + r] = best;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        TopList<E> m;
+        top_list_clear(m);
+        for (int32_t i = lane; i < 8 * E; i += 32) {
+            const int32_t w = i / E, r = i % E;
+            if (r < e) top_list_insert(m, s_list[w * E + r].key, s_list[w * E + r].idx);
+        }
+        for (int32_t r = 0; r < e; ++r) {
+            const Rec best = warp_pop_best(m);
+            if (lane == 0) {
+                if (IDX_OUT) reinterpret_cast<int32_t*>(out)[r] = best.idx;
+                else reinterpret_cast<Rec*>(out)[r] = best;
+            }
+        }
+    }
+}
+
+// The same merge of at most 64 records in global memory by one warp alone (no barrier): idx_out[0..e).
+template <int E>
+__device__ __forceinline__ void warp_merge_small(const Rec* partial, int32_t count, int32_t e,
+                                                 int32_t* __restrict__ idx_out) {
+    const int lane = threadIdx.x & 31;
+    TopList<E> m;
+    top_list_clear(m);
+    int4 raw[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+        if (lane + 32 * u < count) raw[u] = __ldcg(reinterpret_cast<const int4*>(partial) + lane + 32 * u);
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+        if (lane + 32 * u < count)
+            top_list_insert(m, ((unsigned long long)(uint32_t)raw[u].y << 32) | (uint32_t)raw[u].x, raw[u].z);
+    for (int32_t r = 0; r < e; ++r) {
+        const Rec best = warp_pop_best(m);
+        if (lane == 0) idx_out[r] = best.idx;
+    }
+}
+
 __global__ void __launch_bounds__(256) k_top_partial(const double* __restrict__ F, int32_t n, int32_t e,
                                                      int32_t per_block, Rec* __restrict__ partial) {
     __shared__ Rec s_warp[32];
@@ -551,18 +695,24 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
     __shared__ bool s_last;
     const int32_t lo = blockIdx.x * per_block;
     const int32_t count = max(0, min(per_block, n - lo));
+    const bool small = e <= 4;  // lists in registers, one barrier
     Rec prev;
     prev.key = 0;
     prev.idx = -1;
     prev.pad = 0;
-    for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<0>(F + lo, count, lo, r > 0, prev, s_warp);
-        if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
-        prev = best;
-        if (best.idx < 0) {  // fewer than e items in this slice: mark the rest empty
-            for (int32_t r2 = r + 1 + threadIdx.x; r2 < e; r2 += blockDim.x)
-                partial[(int64_t)blockIdx.x * e + r2] = best;
-            break;
+    if (small) {
+        if (e <= 2) block_top_small<2, 0>(F + lo, count, lo, e, partial + (int64_t)blockIdx.x * e, s_warp);
+        else block_top_small<4, 0>(F + lo, count, lo, e, partial + (int64_t)blockIdx.x * e, s_warp);
+    } else {
+        for (int32_t r = 0; r < e; ++r) {
+            Rec best = block_next_best<0>(F + lo, count, lo, r > 0, prev, s_warp);
+            if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * e + r] = best;
+            prev = best;
+            if (best.idx < 0) {  // fewer than e items in this slice: mark the rest empty
+                for (int32_t r2 = r + 1 + threadIdx.x; r2 < e; r2 += blockDim.x)
+                    partial[(int64_t)blockIdx.x * e + r2] = best;
+                break;
+            }
         }
     }
     // from here on only the merging CTA still works: the next kernel's CTAs may take the other SMs (they
@@ -574,12 +724,22 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    prev.key = 0;
-    prev.idx = -1;
-    for (int32_t r = 0; r < e; ++r) {
-        Rec best = block_next_best<1>(partial, top_blocks * e, 0, r > 0, prev, s_warp);
-        if (threadIdx.x == 0) elites[r] = best.idx;
-        prev = best;
+    if (small && top_blocks * e <= 64) {  // a handful of records: one warp, no barrier
+        if (threadIdx.x < 32) {
+            if (e <= 2) warp_merge_small<2>(partial, top_blocks * e, e, elites);
+            else warp_merge_small<4>(partial, top_blocks * e, e, elites);
+        }
+    } else if (small) {
+        if (e <= 2) block_top_small<2, 1, true>(partial, top_blocks * e, 0, e, elites, s_warp);
+        else block_top_small<4, 1, true>(partial, top_blocks * e, 0, e, elites, s_warp);
+    } else {
+        prev.key = 0;
+        prev.idx = -1;
+        for (int32_t r = 0; r < e; ++r) {
+            Rec best = block_next_best<1>(partial, top_blocks * e, 0, r > 0, prev, s_warp);
+            if (threadIdx.x == 0) elites[r] = best.idx;
+            prev = best;
+        }
     }
     if (threadIdx.x == 0) *done = 0u;
 }

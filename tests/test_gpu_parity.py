@@ -196,6 +196,26 @@ def test_evolve_parity_parameter_corners(ones, kw):
         _same_state(g, o)
 
 
+@pytest.mark.parametrize("elitism", [1, 2, 3, 4, 5, 9])
+@pytest.mark.parametrize("N,flags", [(300, 2), (5000, 0), (1031, 2), (1031, 8), (2500, 8)])
+def test_selection_stage_elites_with_ties(ones, elitism, N, flags):
+    """Elites of the selection stage (register lists up to 4, block rounds above) on populations full of equal
+    scores: slices with fewer distinct candidates than elites, ties decided by the row index."""
+    w = inputs.custom(24, 40, N, 3, seed=N + elitism, kmax=5)
+    g, o = _pair(ones, w, elitism=elitism, flags=flags)
+    rows = inputs.random_genomes(w.jobs, 7, seed=3)[:, :24]
+    pop = rows[np.random.default_rng(elitism).integers(0, 7, size=N)]   # only 7 distinct candidates
+    g.set_population(pop)
+    o.set_population(pop)
+    for _ in range(3):
+        g.evolve(1, 21)
+        o.evolve(1, 21)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (eg == eo).all() and (pg == po).all()
+        _same_state(g, o)
+
+
 @pytest.mark.parametrize("flags", [0, 8])
 @pytest.mark.parametrize("J,N", [(1, 2), (2, 3), (5, 4), (6, 4096), (127, 33), (129, 64), (260, 1025), (700, 2000)])
 def test_evolve_parity_ragged_shapes(ones, J, N, flags):
