@@ -311,7 +311,7 @@ def main():
 
     # ---- end to end: every step uploads the job table and reads the best schedule back ----
     J, N, E = w.n_jobs, w.pop, w.params.elitism
-    e2e_steps = 0 if (args.no_e2e or args.scheme == "per_gpu") else min(steps, 100)
+    e2e_steps = 0 if args.no_e2e else min(steps, 100)
     identity = np.arange(J, dtype=np.int32)
     jobs_pinned = torch.from_numpy(w.jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
     jobs_host = jobs_pinned.numpy().view(inputs.JOB_DTYPE)

@@ -514,29 +514,29 @@ __device__ __forceinline__ Rec warp_pop_best(TopList<E>& l) {
     return best;
 }
 
-// The e best (e <= E) of `count` items of one 256-thread block, in rank order, written by thread 0 to out[0..e)
+// The e best (e <= E) of `count` items of one block of THREADS threads, in rank order, written by thread 0 to out[0..e)
 // (empty records when there are fewer than e items).  SRC 0: the items are scores F[i] with index lo + i;
 // 1: records in global memory, possibly written by other CTAs of the same launch (read through L2, four
 // loads in flight per thread); 2: records in shared memory.  IDX_OUT: out is an int32 array that receives
-// the indices only.  s_list: 8 * E records.
-template <int E, int SRC, bool IDX_OUT = false>
+// the indices only.  s_list: (THREADS / 32) * E records.
+template <int E, int SRC, bool IDX_OUT = false, int THREADS = 256>
 __device__ __forceinline__ void block_top_small(const void* __restrict__ items, int32_t count, int32_t lo, int32_t e,
                                                 void* __restrict__ out, Rec* __restrict__ s_list) {
     TopList<E> l;
     top_list_clear(l);
     if (SRC == 1) {
-        for (int32_t i0 = threadIdx.x; i0 < count; i0 += 4 * 256) {
+        for (int32_t i0 = threadIdx.x; i0 < count; i0 += 4 * THREADS) {
             int4 raw[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (i0 + u * 256 < count) raw[u] = __ldcg(reinterpret_cast<const int4*>(items) + i0 + u * 256);
+                if (i0 + u * THREADS < count) raw[u] = __ldcg(reinterpret_cast<const int4*>(items) + i0 + u * THREADS);
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (i0 + u * 256 < count)
+                if (i0 + u * THREADS < count)
                     top_list_insert(l, ((unsigned long long)(uint32_t)raw[u].y << 32) | (uint32_t)raw[u].x, raw[u].z);
         }
     } else {
-        for (int32_t i = threadIdx.x; i < count; i += 256) {
+        for (int32_t i = threadIdx.x; i < count; i += THREADS) {
             if (SRC == 2) {
                 const Rec q = reinterpret_cast<const Rec*>(items)[i];
                 top_list_insert(l, q.key, q.idx);
@@ -554,7 +554,7 @@ __device__ __forceinline__ void block_top_small(const void* __restrict__ items, 
     if (warp == 0) {
         TopList<E> m;
         top_list_clear(m);
-        for (int32_t i = lane; i < 8 * E; i += 32) {
+        for (int32_t i = lane; i < (THREADS / 32) * E; i += 32) {
             const int32_t w = i / E, r = i % E;
             if (r < e) top_list_insert(m, s_list[w * E + r].key, s_list[w * E + r].idx);
         }
@@ -1347,7 +1347,8 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                  uint64_t gen0, int32_t generations, uint32_t thr32, int32_t capacity, double penalty,
                  int32_t rows_shift /* rows per CTA = 1 << rows_shift */, int32_t gs) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ Rec s_warp[32];
+    __shared__ Rec s_warp[64];
+    __shared__ Rec s_top[4];
     cg::cluster_group cluster = cg::this_cluster();
     const int32_t C = (int32_t)cluster.num_blocks(), me = (int32_t)cluster.block_rank();
     const int32_t planes = t.k1 + 1, jpad = t.jpad;
@@ -1403,7 +1404,15 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             sFall[i] = *cluster.map_shared_rank(sF[cur] + (i & rows_mask), (unsigned int)(i >> rows_shift));
         }
         __syncthreads();
-        if (elitism > 0) {
+        if (elitism > 0 && elitism <= 4) {  // sorted lists in registers, one barrier
+            if (elitism <= 2) block_top_small<2, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
+            else block_top_small<4, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
+            __syncthreads();
+            if ((int32_t)threadIdx.x < elitism) {
+                sElit[threadIdx.x] = s_top[threadIdx.x].idx;
+                if (me == 0) elites_out[threadIdx.x] = s_top[threadIdx.x].idx;
+            }
+        } else if (elitism > 0) {
             Rec prev;
             prev.key = 0;
             prev.idx = -1;
@@ -1428,7 +1437,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             uint32_t thr = 0u;
             if (is_elite) {
                 slot0 = elite_lo + item;
-                pa = pb = sElit[slot0];
+                pa = pb = elitism <= 4 ? s_top[slot0].idx : sElit[slot0];
             } else if (live) {
                 const int32_t q = q_lo + (item - (elite_hi - elite_lo));
                 // both tournaments, every lane of the group for itself (same draws, same winner)
