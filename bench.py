@@ -397,9 +397,12 @@ def main():
         line["new_candidates_per_s"] = 3 * line["value"]
         if stage_n.get("evolve"):
             peak, peak_kind = measured_peak()
-            rows = {"children (k_trunc_draws + k_trunc_children)": ("evolve", 6 * N * J * 4),
-                    "k_fitness over the 3N new rows": ("fitness", 3 * N * (4 * J + 12)),
-                    "selection (radix threshold, compaction, k_trunc_gather)": ("select", 2 * N * J * 4 + 4 * N * 8 * 10)}
+            if stage_n.get("fitness"):  # children written first, scored by a separate pass
+                rows = {"children (k_trunc_draws + k_trunc_children)": ("evolve", 6 * N * J * 4),
+                        "k_fitness over the 3N new rows": ("fitness", 3 * N * (4 * J + 12))}
+            else:  # 3N children written and scored in one pass: 3N row reads, 3N row writes, (F, G) of each
+                rows = {"children + scores (k_trunc_draws + k_trunc_children_score)": ("evolve", 6 * N * J * 4 + 3 * N * 12)}
+            rows["selection (radix threshold, compaction, k_trunc_gather)"] = ("select", 2 * N * J * 4 + 4 * N * 8 * 10)
             line["kernels"] = {}
             for name, (stage, nbytes) in rows.items():
                 t_ms = stage_ms[stage] / stage_n[stage]

@@ -503,19 +503,27 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
             c->prof.sample = it % c->prof.every == 0;
             const int64_t K = c->N;
             if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
-            CU(c, launch_trunc_children(c->pop(c->cur), c->ld, c->N, c->parents(), c->tab, keys, c->gen, c->thr16,
-                                        c->stream));
-            if ((rc = prof_end(c)) != ONES_OK) return rc;
-            if ((rc = prof_begin(c, 0)) != ONES_OK) return rc;
-            CU(c, launch_fitness(c->pop(c->cur) + K * c->ld, c->ld, 3 * c->N, c->J, c->tab, c->cap, c->prm.penalty,
-                                 c->Fbuf(c->fcur) + K, c->Gbuf(c->gcur) + K, c->stream));
-            if ((rc = prof_end(c)) != ONES_OK) return rc;
+            if (c->fused) {  // the 3K new rows are scored while they are written
+                CU(c, launch_trunc_children_score(c->pop(c->cur), c->ld, c->N, c->parents(), c->tab, keys, c->gen,
+                                                  c->thr16, c->cap, c->prm.penalty, c->Fbuf(c->fcur), c->Gbuf(c->gcur),
+                                                  c->stream));
+                if ((rc = prof_end(c)) != ONES_OK) return rc;
+            } else {
+                CU(c, launch_trunc_children(c->pop(c->cur), c->ld, c->N, c->parents(), c->tab, keys, c->gen, c->thr16,
+                                            c->stream));
+                if ((rc = prof_end(c)) != ONES_OK) return rc;
+                if ((rc = prof_begin(c, 0)) != ONES_OK) return rc;
+                CU(c, launch_fitness(c->pop(c->cur) + K * c->ld, c->ld, 3 * c->N, c->J, c->tab, c->cap, c->prm.penalty,
+                                     c->Fbuf(c->fcur) + K, c->Gbuf(c->gcur) + K, c->stream));
+                if ((rc = prof_end(c)) != ONES_OK) return rc;
+                c->launches += 1;
+            }
             if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
             CU(c, launch_trunc_select(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->Fbuf(c->fcur),
                                       c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1), c->Gbuf(c->gcur ^ 1),
                                       c->ws + c->L.trunc, c->stream));
             if ((rc = prof_end(c)) != ONES_OK) return rc;
-            c->launches += 15;
+            c->launches += 14;
             c->cur ^= 1;
             c->fcur ^= 1;
             c->gcur ^= 1;

@@ -97,6 +97,10 @@ cudaError_t launch_evolve_cluster(ClusterShape shape, int32_t* pop_io, int64_t l
 size_t trunc_scratch_bytes(int32_t k);
 cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
                                   uint64_t gen, uint32_t thr16, cudaStream_t s);  // 2 launches
+// the same, scoring the 3K new rows in the same pass (needs evolve_score_smem(t) <= kMaxSmemPerBlock); 2 launches
+cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
+                                        uint64_t gen, uint32_t thr16, int32_t capacity, double penalty, double* F,
+                                        int32_t* G, cudaStream_t s);
 cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
                                 const int32_t* G, double* F_next, int32_t* G_next, void* scratch,
                                 cudaStream_t s);  // 12 launches

@@ -1669,6 +1669,101 @@ k_trunc_children(int32_t* __restrict__ pool, int64_t ld, int32_t k, const int32_
     }
 }
 
+// The same children, scored while they are written (as k_evolve_score: one persistent CTA per SM with the
+// model tables in shared memory, one warp per work item, the fixed summation order), so the 3K new rows are
+// not read back for their fitness.  F, G: the pool's score arrays (4K entries; rows K..4K-1 are written).
+template <bool ALWAYS>
+__global__ void __launch_bounds__(1024, 1)
+k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const int32_t* __restrict__ draws, Tables t,
+                       RoundKeys keys, uint32_t gen_lo, uint32_t c3cross, uint32_t c3mutant, uint32_t thr32,
+                       int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const int32_t jpad = t.jpad;
+    double* sX = reinterpret_cast<double*>(smem_raw);
+    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
+    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
+    int4* sRange = sKmin + jpad / 4;
+    {
+        const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
+            const int4 g = gG[i];
+            reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
+                                                         (uint32_t)g.z | ((uint32_t)g.w << 16));
+        }
+        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
+            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
+            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
+        }
+        __syncthreads();
+    }
+    grid_dependency_wait();  // the draws come from the kernel before
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const uint32_t kcap = (uint32_t)t.k1;
+    for (int64_t item = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); item < 2 * (int64_t)k;
+         item += total_warps) {
+        double sum0 = 0.0, sum1 = 0.0;
+        int32_t gp0 = 0, gp1 = 0;
+        int64_t slot0;
+        const bool pair = item < k;
+        if (pair) {
+            const int32_t q = (int32_t)item;
+            const int4* A = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q] * ld);
+            const int4* B = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q + 1] * ld);
+            slot0 = (int64_t)k + 2 * q;
+            int4* C0 = reinterpret_cast<int4*>(pool + slot0 * ld);
+            int4* C1 = reinterpret_cast<int4*>(pool + (slot0 + 1) * ld);
+            for (int32_t v = lane; v < nvec; v += 32) {
+                const int4 a = A[v], b = B[v];
+                const uint4 W = philox((uint32_t)v, (uint32_t)(2 * q), gen_lo, c3cross, keys);
+                int4 c0, c1;
+                sibling_int4<false>(W, a, b, sKmin[v], sRange[v], 0u, true, c0, c1);  // threshold 0: no mutation
+                C0[v] = c0;
+                C1[v] = c1;
+                const int32_t base = (v >> 5) * 128 + lane;
+                score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
+                score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+            }
+        } else {
+            const int32_t m = (int32_t)(item - k);
+            const int4* S = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * k + m] * ld);
+            slot0 = (int64_t)3 * k + m;
+            int4* C = reinterpret_cast<int4*>(pool + slot0 * ld);
+            for (int32_t v = lane; v < nvec; v += 32) {
+                const int4 g = S[v];
+                const uint4 W = philox((uint32_t)v, (uint32_t)m, gen_lo, c3mutant, keys);
+                int4 c0, c1;
+                sibling_int4<ALWAYS>(W, g, g, sKmin[v], sRange[v], thr32, false, c0, c1);  // the even child's draws
+                C[v] = c0;
+                score4(c0, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
+            gp0 += __shfl_xor_sync(0xFFFFFFFFu, gp0, off);
+            sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
+            gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
+        }
+        if (lane == 0) {
+            const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
+            F[slot0] = __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+            G[slot0] = gp0;
+            if (pair) {
+                const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                F[slot0 + 1] = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                G[slot0 + 1] = gp1;
+            }
+        }
+    }
+}
+
 struct TruncPick {  // result of the selection threshold search
     unsigned long long key;  // key of the K-th best candidate
     int32_t quota;           // how many candidates with exactly that key survive (lowest rows first)
@@ -1687,6 +1782,7 @@ struct TruncState {
 
 __global__ void __launch_bounds__(256) k_trunc_radix_pass(const double* __restrict__ F, int32_t n, int32_t k, int pass,
                                                           TruncState* __restrict__ st, TruncPick* __restrict__ out) {
+    grid_dependency_wait();  // launched as a programmatic dependent: only the launch latency overlaps
     __shared__ unsigned int hist[256];
     __shared__ bool s_last;
     hist[threadIdx.x] = 0u;
@@ -1737,6 +1833,7 @@ __global__ void __launch_bounds__(256) k_trunc_radix_pass(const double* __restri
 // per block of `per_block` consecutive rows: how many rank above the threshold, how many tie with it
 __global__ void __launch_bounds__(256) k_trunc_count(const double* __restrict__ F, int32_t n, int32_t per_block,
                                                      const TruncPick* __restrict__ pick, int32_t* __restrict__ bsum) {
+    grid_dependency_wait();  // launched as a programmatic dependent: only the launch latency overlaps
     __shared__ int32_t s_gt, s_eq;
     if (threadIdx.x == 0) s_gt = s_eq = 0;
     __syncthreads();
@@ -1759,6 +1856,7 @@ __global__ void __launch_bounds__(256) k_trunc_count(const double* __restrict__ 
 
 // exclusive scan of the per-block counts (one CTA, blocks <= 1024)
 __global__ void __launch_bounds__(1024) k_trunc_scan(int32_t* __restrict__ bsum, int32_t blocks) {
+    grid_dependency_wait();  // launched as a programmatic dependent: only the launch latency overlaps
     __shared__ int32_t sg[1024], se[1024];
     const int t = threadIdx.x;
     sg[t] = t < blocks ? bsum[2 * t] : 0;
@@ -1781,6 +1879,7 @@ __global__ void __launch_bounds__(1024) k_trunc_scan(int32_t* __restrict__ bsum,
 __global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ F, int32_t n, int32_t per_block,
                                                      const TruncPick* __restrict__ pick,
                                                      const int32_t* __restrict__ bsum, int32_t* __restrict__ kept) {
+    grid_dependency_wait();  // launched as a programmatic dependent: only the launch latency overlaps
     __shared__ int32_t tg[256], te[256];
     const unsigned long long T = pick->key;
     const int32_t quota = pick->quota;
@@ -1823,6 +1922,7 @@ __global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict_
                                                       int64_t ld, int32_t k, const int32_t* __restrict__ kept,
                                                       const double* __restrict__ F, const int32_t* __restrict__ G,
                                                       double* __restrict__ F_new, int32_t* __restrict__ G_new) {
+    grid_dependency_wait();  // launched as a programmatic dependent: only the launch latency overlaps
     const int lane = threadIdx.x & 31;
     const int64_t p = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (p >= k) return;
@@ -1859,6 +1959,27 @@ cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t*
     return cudaGetLastError();
 }
 
+cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
+                                        uint64_t gen, uint32_t thr16, int32_t capacity, double penalty, double* F,
+                                        int32_t* G, cudaStream_t s) {
+    const size_t smem = evolve_score_smem(t);
+    if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    k_trunc_draws<<<(3 * k + 255) / 256, 256, 0, s>>>(k, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
+                                                      counter3(STREAM_SEL_B, gen), counter3(STREAM_PICK, gen), draws);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    constexpr int kThreads = 1024;
+    int64_t blocks = (2 * (int64_t)k + kThreads / 32 - 1) / (kThreads / 32);
+    if (blocks > kSMs) blocks = kSMs;
+    auto kern = thr16 >= 65536u ? k_trunc_children_score<true> : k_trunc_children_score<false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
+    if (e != cudaSuccess) return e;
+    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, pool, ld, k, (const int32_t*)draws, t, keys,
+                                 (uint32_t)gen, counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32, capacity,
+                                 penalty, F, G);
+}
+
 // Keep the best K of the 4K scored rows: F, G hold 4K entries; the survivors become rows 0..K-1 of
 // pool_next with F_next, G_next.  12 launches.
 cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
@@ -1874,17 +1995,18 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
     int rb = (n + 2047) / 2048;
     if (rb > kSMs) rb = kSMs;
     for (int pass = 0; pass < 8; ++pass) {
-        k_trunc_radix_pass<<<rb, 256, 0, s>>>(F, n, k, pass, state, pick);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        e = launch_after_previous(k_trunc_radix_pass, rb, 256, 0, s, F, n, k, pass, state, pick);
+        if (e != cudaSuccess) return e;
     }
-    k_trunc_count<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_trunc_scan<<<1, 1024, 0, s>>>(bsum, blocks);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_trunc_place<<<blocks, 256, 0, s>>>(F, n, per_block, pick, bsum, kept);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_trunc_gather<<<(k + 7) / 8, 256, 0, s>>>(pool, pool_next, ld, k, kept, F, G, F_next, G_next);
-    return cudaGetLastError();
+    e = launch_after_previous(k_trunc_count, blocks, 256, 0, s, F, n, per_block, (const TruncPick*)pick, bsum);
+    if (e != cudaSuccess) return e;
+    e = launch_after_previous(k_trunc_scan, 1, 1024, 0, s, bsum, blocks);
+    if (e != cudaSuccess) return e;
+    e = launch_after_previous(k_trunc_place, blocks, 256, 0, s, F, n, per_block, (const TruncPick*)pick,
+                              (const int32_t*)bsum, kept);
+    if (e != cudaSuccess) return e;
+    return launch_after_previous(k_trunc_gather, (k + 7) / 8, 256, 0, s, pool, pool_next, ld, k, (const int32_t*)kept, F,
+                                 G, F_next, G_next);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -292,10 +292,13 @@ def test_set_get_population_roundtrip(ones):
 
 # ---- the paper's truncation selection (originals + crossover children + mutants, best K survive) -------
 @pytest.mark.parametrize("J,N,kw", [(16, 32, {}), (100, 1024, {}), (37, 101, dict(p_mut=1.0)), (5, 3, dict(p_mut=0.0)),
-                                    (130, 257, dict(p_mut=0.02)), (1, 3, {}), (512, 4096, {})])
+                                    (130, 257, dict(p_mut=0.02)), (1, 3, {}), (512, 4096, {}),
+                                    (130, 257, dict(flags=6)), (37, 101, dict(p_mut=1.0, flags=6)),   # separate scoring pass
+                                    (2048, 700, dict(p_mut=0.02))])
 def test_truncation_selection_parity(ones, J, N, kw):
     w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, pinned=J // 5, kmin_max=2)
-    g, o = _pair(ones, w, flags=4, **kw)
+    kw = dict(kw)
+    g, o = _pair(ones, w, flags=kw.pop("flags", 4), **kw)
     g.randomize(2)
     o.randomize(2)
     for step in (1, 1, 3):
@@ -433,6 +436,24 @@ def test_per_gpu_refresh_parity(ones, J, gpus, N, leave, arrive, kw):
         jobs = jobs2
     bg, bo = g.best(), o.best()
     assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
+
+
+def test_per_gpu_refresh_rejected_update_leaves_the_search_untouched(ones):
+    w = inputs.custom(9, 20, 40, 2, seed=6, kmax=3)
+    g, o = _pair(ones, w, flags=16)
+    g.randomize(4)
+    o.randomize(4)
+    g.evolve(2, 4)
+    o.evolve(2, 4)
+    bad = w.jobs.copy()
+    bad["a"][2] = bad["c"][2] = bad["d"][2] = 0.0          # zero seconds per iteration: no throughput
+    with pytest.raises(ones.OnesError) as err:
+        g.update_jobs(bad, np.arange(9, dtype=np.int32), 20)
+    assert err.value.code == -2
+    _same_state(g, o)                                      # population, scores and tables as before
+    g.evolve(2, 5)
+    o.evolve(2, 5)
+    _same_state(g, o)
 
 
 def test_per_gpu_refresh_limits(ones):
