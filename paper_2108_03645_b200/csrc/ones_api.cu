@@ -689,15 +689,22 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
         return ONES_OK;
     }
     const int64_t new_ld = ld_of(n_jobs);
-    CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(n_jobs), c->tab.kmin,
-                       c->tab.range, c->stream));
+    // c->fused: the new job set's GPU counts fit the 16-bit table and the tables fit shared memory
+    const bool scored = c->fused && remap_score_smem(c->tab) <= (size_t)kMaxSmemPerBlock;
+    if (scored) {  // the new rows are scored while they are written
+        CU(c, launch_remap_score(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(n_jobs),
+                                 c->tab, capacity, c->prm.penalty, c->F(), c->G(), c->stream));
+    } else {
+        CU(c, launch_remap(c->pop(c->cur), old_ld, c->pop(c->cur ^ 1), new_ld, c->N, n_jobs, c->remap(n_jobs),
+                           c->tab.kmin, c->tab.range, c->stream));
+    }
     c->launches += 1;
     c->cur ^= 1;
     c->J = n_jobs;
     c->W = n_jobs;
     c->ld = new_ld;
     c->cap = capacity;
-    c->f_valid = false;
+    c->f_valid = scored;
     c->elites_valid = false;
     return ONES_OK;
 }

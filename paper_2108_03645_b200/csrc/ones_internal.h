@@ -131,6 +131,12 @@ cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const in
 cudaError_t launch_remap(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
                          int32_t n_jobs_new, const int32_t* remap, const int32_t* kmin_new,
                          const int32_t* range_new, cudaStream_t s);
+// remap and score in one pass (tables of the new job set; needs remap_score_smem(t) <= kMaxSmemPerBlock and
+// GPU counts that fit 16 bits)
+size_t remap_score_smem(Tables t);
+cudaError_t launch_remap_score(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                               int32_t n_jobs_new, const int32_t* remap, Tables t, int32_t capacity, double penalty,
+                               double* F, int32_t* G, cudaStream_t s);
 cudaError_t launch_copy_rows(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
                              int32_t n_jobs, int zero_pad, cudaStream_t s);
 cudaError_t launch_export_tables(Tables t, int32_t n_jobs, double* X_out, int32_t* G_out, cudaStream_t s);

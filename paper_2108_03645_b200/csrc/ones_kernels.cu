@@ -1002,6 +1002,101 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
 }
 
 // ---------------------------------------------------------------------------------------------
+// Warm start across a changed job set, scored in the same pass: as k_remap (column j of the new row is
+// column remap[j] of the old one clamped into the new limits, or the lower limit for a new job), one warp
+// per candidate, the new row scored from registers in the fixed order while it is written.  One persistent
+// CTA per SM with the new model tables, limits and the column map in shared memory.  A lane whose four
+// columns come from four neighbouring old columns at the same place takes them as one int4.
+// ---------------------------------------------------------------------------------------------
+size_t remap_score_smem(Tables t) { return evolve_score_smem(t) + (size_t)t.jpad * 4; }
+
+__global__ void __launch_bounds__(1024, 1)
+k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restrict__ dst, int64_t ld_dst, int32_t n,
+              int32_t n_jobs_new, const int32_t* __restrict__ remap, Tables t, int32_t capacity, double penalty,
+              double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const int32_t jpad = t.jpad;
+    double* sX = reinterpret_cast<double*>(smem_raw);
+    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
+    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
+    int4* sRange = sKmin + jpad / 4;
+    int4* sFrom = sRange + jpad / 4;
+    {
+        const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
+            const int4 g = gG[i];
+            reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
+                                                         (uint32_t)g.z | ((uint32_t)g.w << 16));
+        }
+        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
+            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
+            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
+        }
+        // padding columns: no source, limits [0, 0] (k_build_tables), so they come out as 0
+        for (int32_t j = threadIdx.x; j < jpad; j += blockDim.x)
+            reinterpret_cast<int32_t*>(sFrom)[j] = j < n_jobs_new ? remap[j] : -1;
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t nvec = (int32_t)(ld_dst >> 2);
+    const uint32_t kcap = (uint32_t)t.k1;
+    for (int64_t row = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); row < n; row += total_warps) {
+        const int32_t* old_row = src + row * ld_src;
+        int4* new_row = reinterpret_cast<int4*>(dst + row * ld_dst);
+        double sum = 0.0;
+        int32_t gpus = 0;
+        for (int32_t v = lane; v < nvec; v += 32) {
+            const int4 from = sFrom[v], lo = sKmin[v], range = sRange[v];
+            int4 k = lo;
+            if (from.x == 4 * v && from.y == 4 * v + 1 && from.z == 4 * v + 2 && from.w == 4 * v + 3) {
+                k = *reinterpret_cast<const int4*>(old_row + 4 * v);
+            } else {
+                if (from.x >= 0) k.x = old_row[from.x];
+                if (from.y >= 0) k.y = old_row[from.y];
+                if (from.z >= 0) k.z = old_row[from.z];
+                if (from.w >= 0) k.w = old_row[from.w];
+            }
+            k.x = min(max(k.x, lo.x), lo.x + range.x - 1);
+            k.y = min(max(k.y, lo.y), lo.y + range.y - 1);
+            k.z = min(max(k.z, lo.z), lo.z + range.z - 1);
+            k.w = min(max(k.w, lo.w), lo.w + range.w - 1);
+            new_row[v] = k;
+            score4(k, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum, gpus);
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            gpus += __shfl_xor_sync(0xFFFFFFFFu, gpus, off);
+        }
+        if (lane == 0) {
+            const int32_t over = gpus > capacity ? gpus - capacity : 0;
+            F[row] = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            G[row] = gpus;
+        }
+    }
+}
+
+cudaError_t launch_remap_score(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
+                               int32_t n_jobs_new, const int32_t* remap, Tables t, int32_t capacity, double penalty,
+                               double* F, int32_t* G, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const size_t smem = remap_score_smem(t);
+    if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaFuncSetAttribute(k_remap_score, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = ((int64_t)n + 31) / 32;
+    if (blocks > kSMs) blocks = kSMs;
+    k_remap_score<<<(int)blocks, 1024, smem, s>>>(src, ld_src, dst, ld_dst, n, n_jobs_new, remap, t, capacity, penalty, F, G);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // A whole generation in one launch: each warp runs the two tournaments of its pair (one draw per
 // lane, butterfly for the winner), then crossover, mutation and scoring as k_evolve_score, and
 // queues the scores it produced in shared memory; at the end every CTA reduces its queue to its e
