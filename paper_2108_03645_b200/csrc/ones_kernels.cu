@@ -1051,23 +1051,39 @@ k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restri
         int4* new_row = reinterpret_cast<int4*>(dst + row * ld_dst);
         double sum = 0.0;
         int32_t gpus = 0;
-        for (int32_t v = lane; v < nvec; v += 32) {
-            const int4 from = sFrom[v], lo = sKmin[v], range = sRange[v];
-            int4 k = lo;
-            if (from.x == 4 * v && from.y == 4 * v + 1 && from.z == 4 * v + 2 && from.w == 4 * v + 3) {
-                k = *reinterpret_cast<const int4*>(old_row + 4 * v);
-            } else {
-                if (from.x >= 0) k.x = old_row[from.x];
-                if (from.y >= 0) k.y = old_row[from.y];
-                if (from.z >= 0) k.z = old_row[from.z];
-                if (from.w >= 0) k.w = old_row[from.w];
+        constexpr int UN = 4;  // int4 of the old row in flight per lane
+        for (int32_t v0 = lane; v0 < nvec; v0 += 32 * UN) {
+            int4 k[UN];
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int32_t v = v0 + 32 * u;
+                if (v < nvec) {
+                    const int4 from = sFrom[v];
+                    if (from.x == 4 * v && from.y == 4 * v + 1 && from.z == 4 * v + 2 && from.w == 4 * v + 3) {
+                        k[u] = *reinterpret_cast<const int4*>(old_row + 4 * v);
+                    } else {
+                        k[u] = sKmin[v];
+                        if (from.x >= 0) k[u].x = old_row[from.x];
+                        if (from.y >= 0) k[u].y = old_row[from.y];
+                        if (from.z >= 0) k[u].z = old_row[from.z];
+                        if (from.w >= 0) k[u].w = old_row[from.w];
+                    }
+                }
             }
-            k.x = min(max(k.x, lo.x), lo.x + range.x - 1);
-            k.y = min(max(k.y, lo.y), lo.y + range.y - 1);
-            k.z = min(max(k.z, lo.z), lo.z + range.z - 1);
-            k.w = min(max(k.w, lo.w), lo.w + range.w - 1);
-            new_row[v] = k;
-            score4(k, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum, gpus);
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int32_t v = v0 + 32 * u;
+                if (v < nvec) {
+                    const int4 lo = sKmin[v], range = sRange[v];
+                    int4 c = k[u];
+                    c.x = min(max(c.x, lo.x), lo.x + range.x - 1);
+                    c.y = min(max(c.y, lo.y), lo.y + range.y - 1);
+                    c.z = min(max(c.z, lo.z), lo.z + range.z - 1);
+                    c.w = min(max(c.w, lo.w), lo.w + range.w - 1);
+                    new_row[v] = c;
+                    score4(c, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum, gpus);
+                }
+            }
         }
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
@@ -2992,16 +3008,33 @@ k_best(const int32_t* __restrict__ pop, int64_t ld, int32_t n_jobs, const int32_
     if (threadIdx.x == 0) { s_total = 0; s_status = 0; }
     __syncthreads();
     long long part = 0;
-    for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) {
-        const int32_t k = row[j];
-        const int32_t p = (int32_t)min((uint32_t)k, kcap);
-        const int32_t g = t.G[(int64_t)p * t.jpad + slot_of(j)];
-        int32_t less = -1;
-        if (g > 0 && k > t.kmin[j]) less = t.G[(int64_t)(p - 1) * t.jpad + slot_of(j)];
-        wk[j] = k;  // genes that already mean "waiting" are returned as stored
-        wg[j] = g;
-        wl[j] = (less >= 0 && less < g) ? less : -1;
-        part += g;
+    for (int32_t j0 = threadIdx.x; j0 < n_jobs; j0 += 4 * blockDim.x) {
+        // four jobs per step, each kind of load issued for all four before the next kind (the row lives in HBM)
+        int32_t k[4], lo[4], g[4], less[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            k[u] = j < n_jobs ? row[j] : -1;
+            lo[u] = j < n_jobs ? t.kmin[j] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            const int32_t p = (int32_t)min((uint32_t)k[u], kcap);
+            g[u] = j < n_jobs ? t.G[(int64_t)p * t.jpad + slot_of(j)] : 0;
+            less[u] = -1;
+            if (j < n_jobs && p > 0 && k[u] > lo[u]) less[u] = t.G[(int64_t)(p - 1) * t.jpad + slot_of(j)];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            if (j < n_jobs) {
+                wk[j] = k[u];  // genes that already mean "waiting" are returned as stored
+                wg[j] = g[u];
+                wl[j] = (g[u] > 0 && less[u] >= 0 && less[u] < g[u]) ? less[u] : -1;
+                part += g[u];
+            }
+        }
     }
     atomicAdd(reinterpret_cast<unsigned long long*>(&s_total), (unsigned long long)part);
     __syncthreads();
@@ -3055,26 +3088,56 @@ k_best(const int32_t* __restrict__ pop, int64_t ld, int32_t n_jobs, const int32_
     }
     __syncthreads();
 
-    // outputs and the score of the (repaired) row, summed in the fixed order by warp 0
+    // outputs, then the score of the (repaired) row summed in the fixed order by warp 0.  Every thread
+    // looks its jobs' terms up and leaves them where the GPU counts were (2 * jpad int32 = jpad doubles),
+    // so that the summing warp reads one contiguous array, sixteen terms in flight per lane.
     for (int32_t j = threadIdx.x; j < n_jobs; j += blockDim.x) {
-        const int32_t k = wk[j];
-        const int32_t p = (int32_t)min((uint32_t)k, kcap);
-        if (genome_out) genome_out[j] = k;
+        if (genome_out) genome_out[j] = wk[j];
         if (gpus_out) gpus_out[j] = wg[j];
-        if (rate_out) rate_out[j] = t.X[(int64_t)p * t.jpad + slot_of(j)];
     }
+    __syncthreads();
+    double* term = reinterpret_cast<double*>(wg);
+    for (int32_t j0 = threadIdx.x; j0 < n_jobs; j0 += 4 * blockDim.x) {
+        int32_t p[4];
+        double x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            p[u] = j < n_jobs ? (int32_t)min((uint32_t)wk[j], kcap) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            x[u] = j < n_jobs ? t.X[(int64_t)p[u] * t.jpad + slot_of(j)] : 0.0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t j = j0 + u * (int32_t)blockDim.x;
+            if (j < n_jobs) {
+                term[j] = x[u];
+                if (rate_out) rate_out[j] = x[u];
+            }
+        }
+    }
+    __syncthreads();
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         double sum = 0.0;
         const int32_t nvec = (n_jobs + 3) >> 2;
-        for (int32_t v = lane; v < nvec; v += 32) {
-            for (int s = 0; s < 4; ++s) {
-                const int32_t j = 4 * v + s;
-                if (j < n_jobs) {
-                    const int32_t p = (int32_t)min((uint32_t)wk[j], kcap);
-                    sum = __dadd_rn(sum, t.X[(int64_t)p * t.jpad + slot_of(j)]);
+        for (int32_t v0 = lane; v0 < nvec; v0 += 32 * 4) {
+            double x[4][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int s = 0; s < 4; ++s) {
+                    const int32_t j = 4 * (v0 + 32 * u) + s;
+                    x[u][s] = j < n_jobs ? term[j] : 0.0;
                 }
-            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    if (4 * (v0 + 32 * u) + s < n_jobs) sum = __dadd_rn(sum, x[u][s]);
         }
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
