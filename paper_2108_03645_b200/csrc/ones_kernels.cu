@@ -2716,6 +2716,91 @@ __device__ __forceinline__ int32_t last_at_most(const int32_t* __restrict__ a, i
     return lo;
 }
 
+// Order of service in step (4): larger gain first, lower job index on equal gains
+__device__ __forceinline__ bool served_first(double ga, int32_t ja, double gb, int32_t jb) {
+    return ga > gb || (ga == gb && ja < jb);
+}
+
+// Bitonic sort of 256 * PER (gain, job) records in shared memory into the order of service, by a block of
+// 256 threads.  Thread t keeps records PER*t .. PER*t + PER-1 in registers: steps at distance < PER are
+// compare-exchanges between its own registers, steps at distance < 32 * PER exchange with another lane of
+// the warp by shuffles, and only the remaining steps (6 of 66 for 2048 records) go through shared memory,
+// stored transposed (record r of thread t at r * 256 + t) so that lanes touch neighbouring words.
+// The job indices are distinct, so of two records exactly one is served first.
+template <int PER>
+__device__ void block_sort_service_order(double* __restrict__ key, int32_t* __restrict__ who) {
+    static_assert(PER >= 2 && (PER & (PER - 1)) == 0, "at least two records per thread, a power of two");
+    const int tid = threadIdx.x;
+    constexpr int32_t n = 256 * PER;
+    double g[PER];
+    int32_t w[PER];
+#pragma unroll
+    for (int r = 0; r < PER; ++r) {
+        g[r] = key[PER * tid + r];
+        w[r] = who[PER * tid + r];
+    }
+    for (int32_t k = 2; k <= n; k <<= 1) {
+        // in the run of k records that holds position s the lower half keeps the records served first
+        // when (s & k) == 0, the upper half otherwise
+        for (int32_t d = k >> 1; d >= PER; d >>= 1) {
+            const int32_t hop = d / PER;  // the partner record sits in thread t ^ hop, same register
+            if (hop >= 32) {
+                __syncthreads();
+#pragma unroll
+                for (int r = 0; r < PER; ++r) {
+                    key[r * 256 + tid] = g[r];
+                    who[r * 256 + tid] = w[r];
+                }
+                __syncthreads();
+            }
+#pragma unroll
+            for (int r = 0; r < PER; ++r) {
+                double og;
+                int32_t ow;
+                if (hop >= 32) {
+                    og = key[r * 256 + (tid ^ hop)];
+                    ow = who[r * 256 + (tid ^ hop)];
+                } else {
+                    og = __shfl_xor_sync(0xFFFFFFFFu, g[r], hop);
+                    ow = __shfl_xor_sync(0xFFFFFFFFu, w[r], hop);
+                }
+                const int32_t s = PER * tid + r;
+                const bool keep_first = ((s & k) == 0) == ((s & d) == 0);
+                if (served_first(g[r], w[r], og, ow) != keep_first) {
+                    g[r] = og;
+                    w[r] = ow;
+                }
+            }
+        }
+#pragma unroll
+        for (int dd = PER / 2; dd >= 1; dd >>= 1) {
+            if (dd < k) {
+#pragma unroll
+                for (int r = 0; r < PER; ++r) {
+                    if ((r & dd) == 0) {
+                        const bool low_keeps_first = ((PER * tid + r) & k) == 0;
+                        if (served_first(g[r | dd], w[r | dd], g[r], w[r]) == low_keeps_first) {
+                            const double tg = g[r];
+                            const int32_t tw = w[r];
+                            g[r] = g[r | dd];
+                            w[r] = w[r | dd];
+                            g[r | dd] = tg;
+                            w[r | dd] = tw;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();  // the last transposed copy may still be read
+#pragma unroll
+    for (int r = 0; r < PER; ++r) {
+        key[PER * tid + r] = g[r];
+        who[PER * tid + r] = w[r];
+    }
+    __syncthreads();
+}
+
 // Once per job-set change: inv[old id] = the new id of a surviving job (the highest, should several claim
 // one old job) or -1, and newcum[j] = the GPUs that the new jobs before j need for their smallest batch
 // (newcum[n_jobs] = all of them), capped at the cluster's size: needs beyond it can never be met.
@@ -2768,7 +2853,7 @@ k_refresh_prepare(const int32_t* __restrict__ remap, int32_t n_old, int32_t n_jo
 static int32_t refresh_sort_len(int32_t n_jobs) {
     int32_t j2 = 2;
     while (j2 < n_jobs) j2 <<= 1;
-    return j2;
+    return j2 == 256 ? 512 : j2;  // from 512 records on the sort keeps at least two records per thread in registers
 }
 
 size_t refresh_smem(int32_t n_gpus, int32_t n_jobs) {
@@ -2906,23 +2991,27 @@ k_refresh_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_
                 sj[s] = who;
             }
             __syncthreads();
-            for (int32_t k = 2; k <= j2; k <<= 1)
-                for (int32_t d = k >> 1; d > 0; d >>= 1) {
-                    for (int32_t s = tid; s < j2; s += 256) {
-                        const int32_t p = s ^ d;
-                        if (p > s) {
-                            const double ka = key[s], kb = key[p];
-                            const int32_t ja = sj[s], jb = sj[p];
-                            const bool b_first = kb > ka || (kb == ka && jb < ja);  // p's job is served before s's
-                            const bool a_first = ka > kb || (ka == kb && ja < jb);
-                            if (((s & k) == 0) ? b_first : a_first) {
-                                key[s] = kb; key[p] = ka;
-                                sj[s] = jb; sj[p] = ja;
+            if (j2 == 512) block_sort_service_order<2>(key, sj);
+            else if (j2 == 1024) block_sort_service_order<4>(key, sj);
+            else if (j2 == 2048) block_sort_service_order<8>(key, sj);
+            else if (j2 == 4096) block_sort_service_order<16>(key, sj);
+            else  // a few records (or more than fit registers): every step through shared memory
+                for (int32_t k = 2; k <= j2; k <<= 1)
+                    for (int32_t d = k >> 1; d > 0; d >>= 1) {
+                        for (int32_t s = tid; s < j2; s += 256) {
+                            const int32_t p = s ^ d;
+                            if (p > s) {
+                                const double ka = key[s], kb = key[p];
+                                const int32_t ja = sj[s], jb = sj[p];
+                                // ascending runs put the record served first at the lower place
+                                if (served_first(kb, jb, ka, ja) == ((s & k) == 0)) {
+                                    key[s] = kb; key[p] = ka;
+                                    sj[s] = jb; sj[p] = ja;
+                                }
                             }
                         }
+                        __syncthreads();
                     }
-                    __syncthreads();
-                }
             for (int32_t s = tid; s < j2; s += 256) {
                 const int32_t j = sj[s];
                 cum[s] = j < n_jobs ? min(lim[j] - count[j], n_gpus) : 0;

@@ -402,6 +402,9 @@ def _changed_job_set(rng, jobs, n_leave, n_new, seed, kmax_new=0, shuffle=False)
     (64, 1027, 40, 60, 1, {}),                               # the cluster empties: one big refill
     (2048, 4096, 150, 200, 150, dict(p_mut=0.02)),           # benchmark shape
     (40, 4100, 33, 7, 9, {}),                                # rows above 4096 slots
+    (200, 300, 50, 20, 10, {}),                              # sort lengths 256, 1024 and 4096 (1, 4, 16 records
+    (700, 900, 40, 100, 30, {}),                             # per thread in registers)
+    (2500, 1500, 24, 300, 100, dict(p_mut=0.02)),
 ])
 def test_per_gpu_refresh_parity(ones, J, gpus, N, leave, arrive, kw):
     """ones_update_jobs on per-GPU candidates = the oracle's Refresh + Reorder, row by row."""
