@@ -1425,7 +1425,7 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
 namespace cg = cooperative_groups;
 
 struct ClusterSmem {  // byte offsets into dynamic shared memory
-    size_t X, F0, Fall0, Fall1, G16, pop0, pop1, Gc, kmin, range, elit, total;
+    size_t X, F0, F1, Fall, G16, pop0, pop1, Gc, kmin, range, elit, total;
 };
 
 __host__ __device__ inline ClusterSmem cluster_smem(int32_t planes, int32_t jpad, int64_t ld, int32_t rows,
@@ -1436,8 +1436,8 @@ __host__ __device__ inline ClusterSmem cluster_smem(int32_t planes, int32_t jpad
 #define ONES_TAKE(field, bytes) m.field = at; at = (at + (size_t)(bytes) + 15) & ~(size_t)15
     ONES_TAKE(X, (size_t)planes * jpad * 8);
     ONES_TAKE(F0, (size_t)rows * 8);
-    ONES_TAKE(Fall0, (size_t)n * 8);
-    ONES_TAKE(Fall1, (size_t)n * 8);
+    ONES_TAKE(F1, (size_t)rows * 8);
+    ONES_TAKE(Fall, (size_t)n * 8);
     ONES_TAKE(pop0, (size_t)rows * ld * 4);
     ONES_TAKE(pop1, (size_t)rows * ld * 4);
     ONES_TAKE(Gc, (size_t)rows * 4);
@@ -1467,14 +1467,12 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
     const ClusterSmem m = cluster_smem(planes, jpad, ld, rows_per_cta, elitism, n);
     double* sX = reinterpret_cast<double*>(smem_raw + m.X);
     uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + m.G16);
-    double* sF0 = reinterpret_cast<double*>(smem_raw + m.F0);  // my rows' scores as staged at the start
-    // every candidate's score, one private copy per CTA and generation parity: the CTA that scores a child
-    // stores the score into every CTA's copy for the next generation, so nobody fetches scores after the barrier
-    double* sFall[2] = {reinterpret_cast<double*>(smem_raw + m.Fall0), reinterpret_cast<double*>(smem_raw + m.Fall1)};
+    double* sF[2] = {reinterpret_cast<double*>(smem_raw + m.F0), reinterpret_cast<double*>(smem_raw + m.F1)};
     int32_t* sPop[2] = {reinterpret_cast<int32_t*>(smem_raw + m.pop0), reinterpret_cast<int32_t*>(smem_raw + m.pop1)};
     int32_t* sGc = reinterpret_cast<int32_t*>(smem_raw + m.Gc);
     int4* sKmin = reinterpret_cast<int4*>(smem_raw + m.kmin);
     int4* sRange = reinterpret_cast<int4*>(smem_raw + m.range);
+    double* sFall = reinterpret_cast<double*>(smem_raw + m.Fall);  // every candidate's score, copied each generation
     int32_t* sElit = reinterpret_cast<int32_t*>(smem_raw + m.elit);
 
     const int32_t lo = me * rows_per_cta, hi = min(n, lo + rows_per_cta), mine = max(0, hi - lo);
@@ -1491,13 +1489,10 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         }
         const int4* src = reinterpret_cast<const int4*>(pop_io + (int64_t)lo * ld);
         for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) reinterpret_cast<int4*>(sPop[0])[i] = src[i];
-        for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) sF0[i] = F_io[lo + i];
+        for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) sF[0][i] = F_io[lo + i];
     }
     __syncthreads();
     cluster.sync();  // everybody's rows and scores are staged
-    for (int32_t i = threadIdx.x; i < n; i += blockDim.x)
-        sFall[0][i] = *cluster.map_shared_rank(sF0 + (i & rows_mask), (unsigned int)(i >> rows_shift));
-    __syncthreads();
 
     const uint32_t kcap = (uint32_t)t.k1;
     const int32_t groups = (int32_t)blockDim.x / gs;
@@ -1515,11 +1510,14 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         const uint64_t gen = gen0 + (uint64_t)g;
         const uint32_t gen_lo = (uint32_t)gen;
         const uint32_t c3 = counter3(STREAM_MUT, gen), c3a = counter3(STREAM_SEL_A, gen), c3b = counter3(STREAM_SEL_B, gen);
-        // ---- every CTA finds the elites for itself in its copy of the scores ----
-        const double* Fcur = sFall[cur];
+        // ---- every CTA takes a private copy of all scores, then finds the elites for itself ----
+        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
+            sFall[i] = *cluster.map_shared_rank(sF[cur] + (i & rows_mask), (unsigned int)(i >> rows_shift));
+        }
+        __syncthreads();
         if (elitism > 0 && elitism <= 4) {  // sorted lists in registers, one barrier
-            if (elitism <= 2) block_top_small<2, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
-            else block_top_small<4, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
+            if (elitism <= 2) block_top_small<2, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
+            else block_top_small<4, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
             __syncthreads();
             if ((int32_t)threadIdx.x < elitism) {
                 sElit[threadIdx.x] = s_top[threadIdx.x].idx;
@@ -1531,7 +1529,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             prev.idx = -1;
             prev.pad = 0;
             for (int32_t r = 0; r < elitism; ++r) {
-                Rec best = block_next_best<0>(Fcur, n, 0, r > 0, prev, s_warp);
+                Rec best = block_next_best<0>(sFall, n, 0, r > 0, prev, s_warp);
                 if (threadIdx.x == 0) {
                     sElit[r] = best.idx;
                     if (me == 0) elites_out[r] = best.idx;
@@ -1564,7 +1562,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                         for (int u = 0; u < 4; ++u) {
                             if (t0 + u < tournament) {
                                 const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
-                                const double f = Fcur[idx];
+                                const double f = sFall[idx];
                                 if (win < 0 || f > fwin || (f == fwin && idx < win)) {
                                     win = idx;
                                     fwin = f;
@@ -1616,21 +1614,18 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                 sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
                 gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
             }
-            if (live) {
-                // after the butterfly every lane of the group holds the sums: lane r of the group stores the
-                // scores into CTA r's copy for the next generation (CTA r, r + gs, ... when the group is small)
+            if (live && gl == 0) {
+                const int32_t o0 = slot0 >> rows_shift;
                 const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
-                const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
-                const double f0 = __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
-                const double f1 = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
-                for (int32_t r = gl; r < C; r += gs) {
-                    double* theirs = cluster.map_shared_rank(sFall[nxt], (unsigned int)r);
-                    theirs[slot0] = f0;
-                    if (has1) theirs[slot1] = f1;
-                }
-                if (gl == 0) {
-                    *cluster.map_shared_rank(sGc + (slot0 & rows_mask), (unsigned int)(slot0 >> rows_shift)) = gp0;
-                    if (has1) *cluster.map_shared_rank(sGc + (slot1 & rows_mask), (unsigned int)(slot1 >> rows_shift)) = gp1;
+                *cluster.map_shared_rank(sF[nxt] + (slot0 & rows_mask), (unsigned int)o0) =
+                    __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+                *cluster.map_shared_rank(sGc + (slot0 & rows_mask), (unsigned int)o0) = gp0;
+                if (has1) {
+                    const int32_t o1 = slot1 >> rows_shift;
+                    const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                    *cluster.map_shared_rank(sF[nxt] + (slot1 & rows_mask), (unsigned int)o1) =
+                        __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                    *cluster.map_shared_rank(sGc + (slot1 & rows_mask), (unsigned int)o1) = gp1;
                 }
             }
         }
@@ -1641,7 +1636,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
     int4* dst = reinterpret_cast<int4*>(pop_io + (int64_t)lo * ld);
     for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) dst[i] = reinterpret_cast<const int4*>(sPop[fin])[i];
     for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) {
-        F_io[lo + i] = sFall[fin][lo + i];
+        F_io[lo + i] = sF[fin][i];
         G_out[lo + i] = sGc[i];
     }
 }
