@@ -1812,6 +1812,7 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
         __syncthreads();
     }
     grid_dependency_wait();  // the draws come from the kernel before
+    constexpr int UN = 1;  // int4 per source row in flight per lane (2 measured 2 % slower)
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
@@ -1830,29 +1831,52 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
             slot0 = (int64_t)k + 2 * q;
             int4* C0 = reinterpret_cast<int4*>(pool + slot0 * ld);
             int4* C1 = reinterpret_cast<int4*>(pool + (slot0 + 1) * ld);
-            for (int32_t v = lane; v < nvec; v += 32) {
-                const int4 a = A[v], b = B[v];
-                const uint4 W = philox((uint32_t)v, (uint32_t)(2 * q), gen_lo, c3cross, keys);
-                int4 c0, c1;
-                sibling_int4<false>(W, a, b, sKmin[v], sRange[v], 0u, true, c0, c1);  // threshold 0: no mutation
-                C0[v] = c0;
-                C1[v] = c1;
-                const int32_t base = (v >> 5) * 128 + lane;
-                score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
-                score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+            for (int32_t v0 = lane; v0 < nvec; v0 += 32 * UN) {
+                int4 a[UN], b[UN];
+#pragma unroll
+                for (int u = 0; u < UN; ++u) {
+                    const int32_t v = v0 + 32 * u;
+                    if (v < nvec) {
+                        a[u] = A[v];
+                        b[u] = B[v];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < UN; ++u) {
+                    const int32_t v = v0 + 32 * u;
+                    if (v < nvec) {
+                        const uint4 W = philox((uint32_t)v, (uint32_t)(2 * q), gen_lo, c3cross, keys);
+                        int4 c0, c1;
+                        sibling_int4<false>(W, a[u], b[u], sKmin[v], sRange[v], 0u, true, c0, c1);  // threshold 0: no mutation
+                        C0[v] = c0;
+                        C1[v] = c1;
+                        const int32_t base = (v >> 5) * 128 + lane;
+                        score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
+                        score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+                    }
+                }
             }
         } else {
             const int32_t m = (int32_t)(item - k);
             const int4* S = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * k + m] * ld);
             slot0 = (int64_t)3 * k + m;
             int4* C = reinterpret_cast<int4*>(pool + slot0 * ld);
-            for (int32_t v = lane; v < nvec; v += 32) {
-                const int4 g = S[v];
-                const uint4 W = philox((uint32_t)v, (uint32_t)m, gen_lo, c3mutant, keys);
-                int4 c0, c1;
-                sibling_int4<ALWAYS>(W, g, g, sKmin[v], sRange[v], thr32, false, c0, c1);  // the even child's draws
-                C[v] = c0;
-                score4(c0, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
+            for (int32_t v0 = lane; v0 < nvec; v0 += 32 * UN) {
+                int4 g[UN];
+#pragma unroll
+                for (int u = 0; u < UN; ++u)
+                    if (v0 + 32 * u < nvec) g[u] = S[v0 + 32 * u];
+#pragma unroll
+                for (int u = 0; u < UN; ++u) {
+                    const int32_t v = v0 + 32 * u;
+                    if (v < nvec) {
+                        const uint4 W = philox((uint32_t)v, (uint32_t)m, gen_lo, c3mutant, keys);
+                        int4 c0, c1;
+                        sibling_int4<ALWAYS>(W, g[u], g[u], sKmin[v], sRange[v], thr32, false, c0, c1);  // the even child's draws
+                        C[v] = c0;
+                        score4(c0, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
+                    }
+                }
             }
         }
 #pragma unroll
