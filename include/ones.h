@@ -203,8 +203,9 @@ int ones_best(ones_ctx* ctx, int repair, int32_t* h_genome, int32_t* h_gpus_per_
  *   (4) while a GPU is idle, the job below its limit whose score term gains most from growing to the limit
  *       (ties: lower index) takes the GPUs it needs for that, or what is left, lowest idle GPUs first.
  * capacity must equal the cluster size of ones_create (ONES_ERR_BAD_PARAM otherwise).  The step keeps one
- * candidate and its per-job lists in the shared memory of a thread block: 8 * capacity + 40 * n_jobs bytes
- * (n_jobs rounded up to a power of two) must stay below 226 KiB, else ONES_ERR_WORKSPACE. */
+ * candidate and its per-job lists in the shared memory of a thread block: 8 * capacity + 16 * n_jobs + 16 * P
+ * bytes, P = n_jobs rounded up to a power of two (512 for 129..256 jobs), must stay below 226 KiB, else
+ * ONES_ERR_WORKSPACE (e.g. 4096 GPUs with up to 4220 jobs, 64 GPUs with up to 6236). */
 int ones_update_jobs(ones_ctx* ctx, const ones_job* jobs, int32_t n_jobs, const int32_t* remap,
                      int32_t capacity);
 
