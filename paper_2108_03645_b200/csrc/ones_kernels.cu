@@ -1008,7 +1008,9 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
 // CTA per SM with the new model tables, limits and the column map in shared memory.  A lane whose four
 // columns come from four neighbouring old columns at the same place takes them as one int4.
 // ---------------------------------------------------------------------------------------------
-size_t remap_score_smem(Tables t) { return evolve_score_smem(t) + (size_t)t.jpad * 4; }
+// shared memory: X planes (fp64), g planes (16 bits), column map (int32), limits as two bytes per job, one
+// "same four columns" flag per int4
+size_t remap_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (size_t)t.jpad * 4 + (size_t)t.jpad * 2 + (size_t)t.jpad / 4; }
 
 __global__ void __launch_bounds__(1024, 1)
 k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restrict__ dst, int64_t ld_dst, int32_t n,
@@ -1019,9 +1021,9 @@ k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restri
     const int32_t jpad = t.jpad;
     double* sX = reinterpret_cast<double*>(smem_raw);
     uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
-    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
-    int4* sRange = sKmin + jpad / 4;
-    int4* sFrom = sRange + jpad / 4;
+    int4* sFrom = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
+    uint2* sLim = reinterpret_cast<uint2*>(sFrom + jpad / 4);  // per job: lower limit | upper limit << 8 (both <= 15)
+    uint8_t* sSame = reinterpret_cast<uint8_t*>(sLim + jpad / 4);  // per int4: its columns are the same four old columns
     {
         const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
         const int4* gX = reinterpret_cast<const int4*>(t.X);
@@ -1032,13 +1034,23 @@ k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restri
             reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
                                                          (uint32_t)g.z | ((uint32_t)g.w << 16));
         }
-        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
-            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
-            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
-        }
         // padding columns: no source, limits [0, 0] (k_build_tables), so they come out as 0
-        for (int32_t j = threadIdx.x; j < jpad; j += blockDim.x)
-            reinterpret_cast<int32_t*>(sFrom)[j] = j < n_jobs_new ? remap[j] : -1;
+        for (int32_t v = threadIdx.x; v < jpad / 4; v += blockDim.x) {
+            int32_t from[4];
+            uint32_t lim[4];
+            bool same = true;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int32_t j = 4 * v + c;
+                from[c] = j < n_jobs_new ? remap[j] : -1;
+                const int32_t lo = t.kmin[j];
+                lim[c] = (uint32_t)lo | ((uint32_t)(lo + t.range[j] - 1) << 8);
+                same = same && from[c] == j;
+            }
+            sFrom[v] = make_int4(from[0], from[1], from[2], from[3]);
+            sLim[v] = make_uint2(lim[0] | (lim[1] << 16), lim[2] | (lim[3] << 16));
+            sSame[v] = same ? 1 : 0;
+        }
         __syncthreads();
     }
     const int lane = threadIdx.x & 31;
@@ -1058,11 +1070,12 @@ k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restri
             for (int u = 0; u < UN; ++u) {
                 const int32_t v = v0 + 32 * u;
                 if (v < nvec) {
-                    const int4 from = sFrom[v];
-                    if (from.x == 4 * v && from.y == 4 * v + 1 && from.z == 4 * v + 2 && from.w == 4 * v + 3) {
+                    if (sSame[v]) {
                         k[u] = *reinterpret_cast<const int4*>(old_row + 4 * v);
                     } else {
-                        k[u] = sKmin[v];
+                        const int4 from = sFrom[v];
+                        const int32_t none = -0x7FFFFFFF;  // a new job: the clamp below puts it at its lower limit
+                        k[u] = make_int4(none, none, none, none);
                         if (from.x >= 0) k[u].x = old_row[from.x];
                         if (from.y >= 0) k[u].y = old_row[from.y];
                         if (from.z >= 0) k[u].z = old_row[from.z];
@@ -1074,12 +1087,12 @@ k_remap_score(const int32_t* __restrict__ src, int64_t ld_src, int32_t* __restri
             for (int u = 0; u < UN; ++u) {
                 const int32_t v = v0 + 32 * u;
                 if (v < nvec) {
-                    const int4 lo = sKmin[v], range = sRange[v];
+                    const uint2 lim = sLim[v];
                     int4 c = k[u];
-                    c.x = min(max(c.x, lo.x), lo.x + range.x - 1);
-                    c.y = min(max(c.y, lo.y), lo.y + range.y - 1);
-                    c.z = min(max(c.z, lo.z), lo.z + range.z - 1);
-                    c.w = min(max(c.w, lo.w), lo.w + range.w - 1);
+                    c.x = min(max(c.x, (int32_t)(lim.x & 0xFFu)), (int32_t)((lim.x >> 8) & 0xFFu));
+                    c.y = min(max(c.y, (int32_t)((lim.x >> 16) & 0xFFu)), (int32_t)(lim.x >> 24));
+                    c.z = min(max(c.z, (int32_t)(lim.y & 0xFFu)), (int32_t)((lim.y >> 8) & 0xFFu));
+                    c.w = min(max(c.w, (int32_t)((lim.y >> 16) & 0xFFu)), (int32_t)(lim.y >> 24));
                     new_row[v] = c;
                     score4(c, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum, gpus);
                 }
