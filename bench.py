@@ -352,6 +352,21 @@ def main():
         s2.evolve(min(steps, 200), seed)
         sep = s2.stage_times()
         s2.set_profiling(False)
+        # the score step on packed rows (one byte per gene); two copies read in turn so that a launch never
+        # finds its rows in L2 from the launch before (2 x N x ld8 bytes against 126 MB of L2)
+        packs = [s2.pack(), s2.pack()]
+        outF, outG = s2.evaluate_packed(packs[0])
+        reps = 20
+        torch.cuda.synchronize()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record()
+        for i in range(reps):
+            s2.evaluate_packed(packs[i & 1], out=(outF, outG))
+        p1.record()
+        torch.cuda.synchronize()
+        packed_ms = p0.elapsed_time(p1) / reps
+        packed_bytes = packs[0].shape[0] * (packs[0].shape[1] + 12)
+        del packs
         s2.close()
 
     if rank != 0:
@@ -445,6 +460,13 @@ def main():
                                          "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, N, name)),
                                          "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
                                          "how": "same workload with ONES_FLAG_UNFUSED (separate scoring pass)"}
+            a = packed_bytes / (packed_ms * 1e-3) / 1e9
+            line["kernels"]["k_fitness_packed"] = {
+                "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
+                "bytes_per_launch": packed_bytes, "ms_per_launch": packed_ms, "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
+                "candidate_evals_per_s": N / (packed_ms * 1e-3),
+                "how": "ones_evaluate_packed on the same population stored as one byte per gene (a variant beside the "
+                       "int32 contract); 20 launches back to back, two packed copies read in turn"}
     if base is not None:
         line["cpu_baseline"] = base
     print(json.dumps(line))

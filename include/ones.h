@@ -162,6 +162,23 @@ int ones_get_population(ones_ctx* ctx, int32_t* genomes, int64_t ld, int on_devi
 int ones_evaluate(ones_ctx* ctx, const int32_t* d_genomes, int64_t ld, int32_t n, double* d_fitness,
                   int32_t* d_gpus);
 
+/* Packed candidates: the same score step (Alg. 1, Eq. 8; Eq. 4) on rows of one byte per gene, a quarter of
+ * the bytes of the int32 rows.  A byte holds the exponent (at most 15; any gene outside [0, 254] is stored as
+ * 0xFF = the job waits).  A packed row is a sequence of tiles of 512 genes; the row stride ld8 is a multiple of
+ * 512 bytes, at least ones_packed_row_bytes(n_jobs).  Inside a tile, byte 16*l + 4*b + s holds gene
+ * 128*b + 4*l + s of the tile (l = 0..31, b = 0..3, s = 0..3; genes past n_jobs are 0xFF): one 16-byte load gives
+ * a lane the genes it adds, in the order of the fixed summation, so fitness and gpus are bit-identical to
+ * ones_evaluate on the int32 rows.
+ *   ones_pack_population   d_genomes device int32[n][ld] (NULL: the handle's population, ld and n ignored)
+ *                          -> d_packed device uint8[n][ld8], 16-byte aligned.
+ *   ones_evaluate_packed   d_packed -> d_fitness device double[n], d_gpus device int32[n] or NULL.
+ * Not available with ONES_FLAG_PER_GPU (job ids do not fit a byte).  Asynchronous. */
+size_t ones_packed_row_bytes(int32_t n_jobs);
+int ones_pack_population(ones_ctx* ctx, const int32_t* d_genomes, int64_t ld, int32_t n, uint8_t* d_packed,
+                         int64_t ld8);
+int ones_evaluate_packed(ones_ctx* ctx, const uint8_t* d_packed, int64_t ld8, int32_t n, double* d_fitness,
+                         int32_t* d_gpus);
+
 /* Run `generations` generations (Fig. 4: G_i -> G'_i -> G_{i+1}).  Each one: the
  * `elitism` best candidates (score descending, index ascending) move unchanged to
  * rows 0..E-1; for every pair of remaining rows two parents are chosen by

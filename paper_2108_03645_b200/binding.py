@@ -53,6 +53,9 @@ _SIGNATURES = {
     "ones_set_population": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int]),
     "ones_get_population": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int]),
     "ones_evaluate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
+    "ones_packed_row_bytes": (C.c_size_t, [C.c_int32]),
+    "ones_pack_population": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64]),
+    "ones_evaluate_packed": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
     "ones_evolve": (C.c_int, [C.c_void_p, C.c_int32, C.c_uint64]),
     "ones_best": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                             C.c_void_p]),
@@ -228,6 +231,33 @@ class Search:
         if genomes is not None and n == 0:
             return F, G  # an empty tensor has no address to pass
         self._check(lib().ones_evaluate(self._h, ptr, ld, n, _t_ptr(F), _t_ptr(G)), "ones_evaluate")
+        return F, G
+
+    def pack(self, genomes: torch.Tensor | None = None) -> torch.Tensor:
+        """`genomes` (device int32[n, ld]), or the current population, as packed rows: uint8[n, ld8]."""
+        ld8 = int(lib().ones_packed_row_bytes(self.J))
+        if genomes is None:
+            n, ld, ptr = self.N, 0, None
+        else:
+            assert genomes.is_cuda and genomes.dtype == torch.int32 and genomes.is_contiguous()
+            n, ld, ptr = genomes.shape[0], genomes.shape[1], _t_ptr(genomes)
+        packed = torch.empty((n, ld8), dtype=torch.uint8, device=self.device)
+        if n:
+            self._check(lib().ones_pack_population(self._h, ptr, ld, n, _t_ptr(packed), ld8), "ones_pack_population")
+        return packed
+
+    def evaluate_packed(self, packed: torch.Tensor, out=None):
+        """Scores and GPU demand of packed rows (see `pack`)."""
+        assert packed.is_cuda and packed.dtype == torch.uint8 and packed.is_contiguous()
+        n, ld8 = packed.shape
+        if out is None:
+            F = torch.empty(n, dtype=torch.float64, device=self.device)
+            G = torch.empty(n, dtype=torch.int32, device=self.device)
+        else:
+            F, G = out
+        if n:
+            self._check(lib().ones_evaluate_packed(self._h, _t_ptr(packed), ld8, n, _t_ptr(F), _t_ptr(G)),
+                        "ones_evaluate_packed")
         return F, G
 
     def evolve(self, generations: int, seed: int):

@@ -488,6 +488,43 @@ int ones_evaluate(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, 
     return prof_end(c);
 }
 
+size_t ones_packed_row_bytes(int32_t n_jobs) {
+    if (n_jobs <= 0 || n_jobs > kJobsLimit) return 0;
+    return ((size_t)n_jobs + 511) / 512 * 512;
+}
+
+int ones_pack_population(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int32_t n, uint8_t* d_packed, int64_t ld8) {
+    DeviceScope scope(c);
+    if (!c || !d_packed) return ONES_ERR_NULL;
+    if (c->per_gpu) return ONES_ERR_BAD_PARAM;  // job ids do not fit a byte
+    if (!d_genomes) {
+        d_genomes = c->pop(c->cur);
+        ld = c->ld;
+        n = c->N;
+    }
+    if (n < 0 || ld < c->J || ld8 < (int64_t)ones_packed_row_bytes(c->J)) return ONES_ERR_BAD_PARAM;
+    if ((ld & 3) != 0 || (ld8 & 511) != 0 || !aligned16(d_genomes) || !aligned16(d_packed)) return ONES_ERR_ALIGN;
+    if (n == 0) return ONES_OK;
+    CU(c, launch_pack_rows(d_genomes, ld, n, c->J, d_packed, ld8, c->stream));
+    c->launches += 1;
+    return ONES_OK;
+}
+
+int ones_evaluate_packed(ones_ctx* c, const uint8_t* d_packed, int64_t ld8, int32_t n, double* d_fitness,
+                         int32_t* d_gpus) {
+    DeviceScope scope(c);
+    if (!c || !d_packed || !d_fitness) return ONES_ERR_NULL;
+    if (c->per_gpu) return ONES_ERR_BAD_PARAM;
+    if (n < 0 || ld8 < (int64_t)ones_packed_row_bytes(c->J)) return ONES_ERR_BAD_PARAM;
+    if ((ld8 & 511) != 0 || !aligned16(d_packed)) return ONES_ERR_ALIGN;
+    if (n == 0) return ONES_OK;
+    int rc = prof_begin(c, 0);
+    if (rc) return rc;
+    CU(c, launch_fitness_packed(d_packed, ld8, n, c->tab, c->cap, c->prm.penalty, d_fitness, d_gpus, c->stream));
+    c->launches += 1;
+    return prof_end(c);
+}
+
 int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;

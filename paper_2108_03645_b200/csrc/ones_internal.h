@@ -52,6 +52,11 @@ cudaError_t launch_randomize(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs
                              RoundKeys keys, cudaStream_t s);
 cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_t n_jobs, Tables t,
                            int32_t capacity, double penalty, double* F, int32_t* G, cudaStream_t s);
+// packed candidates (one byte per gene, tiles of 512 genes ordered for one 16-byte load per lane; ld8 % 512 == 0)
+cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t n_jobs, uint8_t* dst, int64_t ld8,
+                             cudaStream_t s);
+cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, Tables t, int32_t capacity,
+                                  double penalty, double* F, int32_t* G, cudaStream_t s);
 // tournaments + top-e in one launch; *done must be 0 at launch (the kernel leaves it 0)
 cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
                                 uint64_t gen, int32_t* parents, int32_t e, int32_t* elites, void* scratch,

@@ -364,6 +364,148 @@ cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_
 }
 
 // ---------------------------------------------------------------------------------------------
+// Packed candidates: one byte per gene (exponents are at most 15; 0xFF = the job waits), a quarter of the
+// bytes of the int32 rows.  A packed row is a sequence of tiles of 512 genes (row stride = jobs rounded up
+// to 512 bytes).  Inside a tile the bytes are ordered so that ONE 16-byte load gives lane l exactly the
+// genes it sums in the fixed order: byte 16*l + 4*b + s holds gene 128*b + 4*l + s of the tile (b = 0..3
+// the 128-gene block, s = 0..3), i.e. the genes 4l..4l+3 of four consecutive blocks.  The lane adds them
+// block after block, so partial sum l receives its jobs in increasing order and scores are bit-identical
+// to those of the int32 rows.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_pack_rows(const int32_t* __restrict__ src, int64_t ld, int32_t n, int32_t n_jobs, uint8_t* __restrict__ dst, int64_t ld8) {
+    const int32_t groups = (int32_t)(ld8 >> 4);  // 16-byte groups per packed row
+    const int64_t total = (int64_t)n * groups;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / groups;
+        const int32_t grp = (int32_t)(i % groups);
+        const int32_t tile = grp >> 5, l = grp & 31;
+        uint32_t w[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int32_t j0 = tile * 512 + b * 128 + 4 * l;
+            int4 g = make_int4(-1, -1, -1, -1);
+            if (j0 + 3 < n_jobs) {
+                g = *reinterpret_cast<const int4*>(src + row * ld + j0);
+            } else {
+                if (j0 < n_jobs) g.x = src[row * ld + j0];
+                if (j0 + 1 < n_jobs) g.y = src[row * ld + j0 + 1];
+                if (j0 + 2 < n_jobs) g.z = src[row * ld + j0 + 2];
+            }
+            w[b] = min((uint32_t)g.x, 255u) | (min((uint32_t)g.y, 255u) << 8) | (min((uint32_t)g.z, 255u) << 16) |
+                   (min((uint32_t)g.w, 255u) << 24);
+        }
+        *reinterpret_cast<uint4*>(dst + row * ld8 + 16 * (int64_t)grp) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t n_jobs, uint8_t* dst, int64_t ld8,
+                             cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const int64_t total = (int64_t)n * (ld8 >> 4);
+    const int64_t grid = (total + 255) / 256;
+    k_pack_rows<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld, n, n_jobs, dst, ld8);
+    return cudaGetLastError();
+}
+
+// Fitness of packed candidates: one candidate per warp, one 16-byte load per lane and tile (UNROLL tiles in
+// flight), tables in shared memory as for k_fitness.
+template <bool SMEM, int UNROLL>
+__global__ void __launch_bounds__(1024, 1)
+k_fitness_packed(const uint8_t* __restrict__ rows, int64_t ld8, int32_t n, Tables t, int32_t capacity, double penalty,
+                 double* __restrict__ F, int32_t* __restrict__ G) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const double* __restrict__ lutX = t.X;
+    const int32_t* __restrict__ lutG = t.G;
+    if (SMEM) {
+        double* sX = reinterpret_cast<double*>(smem_raw);
+        int32_t* sG = reinterpret_cast<int32_t*>(smem_raw + (size_t)planes * t.jpad * sizeof(double));
+        const int32_t nX = planes * t.jpad / 2;
+        const int32_t nG = planes * t.jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) reinterpret_cast<int4*>(sG)[i] = gG[i];
+        __syncthreads();
+        lutX = sX;
+        lutG = sG;
+    }
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = blockDim.x >> 5;
+    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const uint32_t kcap = (uint32_t)t.k1;
+    const int32_t jpad = t.jpad;
+    const int32_t tiles = (jpad + 511) >> 9;  // tiles that hold jobs (the tables end at jpad)
+
+    for (int64_t cand = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); cand < n; cand += total_warps) {
+        const uint4* row = reinterpret_cast<const uint4*>(rows + cand * ld8);
+        double sum = 0.0;
+        int32_t gpus = 0;
+        for (int32_t t0 = 0; t0 < tiles; t0 += UNROLL) {
+            uint4 q[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u)
+                if (t0 + u < tiles) q[u] = __ldcs(row + (t0 + u) * 32 + lane);
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (t0 + u < tiles) {
+                    const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const int32_t base = ((t0 + u) * 4 + b) * 128 + lane;  // slot of gene 4l of this block
+                        if (base < jpad) {  // whole blocks past the tables hold no jobs (warp-uniform)
+#pragma unroll
+                            for (int s4 = 0; s4 < 4; ++s4) {
+                                const uint32_t k = (w[b] >> (8 * s4)) & 0xFFu;
+                                const int32_t at = (int32_t)min(k, kcap) * jpad + base + 32 * s4;
+                                sum = __dadd_rn(sum, lutX[at]);
+                                gpus += lutG[at];
+                            }
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            gpus += __shfl_xor_sync(0xFFFFFFFFu, gpus, off);
+        }
+        if (lane == 0) {
+            const int32_t over = gpus > capacity ? gpus - capacity : 0;
+            F[cand] = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            if (G) G[cand] = gpus;
+        }
+    }
+}
+
+cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, Tables t, int32_t capacity,
+                                  double penalty, double* F, int32_t* G, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const size_t lut_bytes = (size_t)(t.k1 + 1) * t.jpad * 12;
+    const bool big = n >= kSMs * 32;
+    const int threads = big ? 1024 : 256;
+    const int wpb = threads / 32;
+    int64_t blocks = ((int64_t)n + wpb - 1) / wpb;
+    if (lut_bytes <= (size_t)kMaxSmemPerBlock) {
+        int per_sm = (int)(kMaxSmemPerBlock / (lut_bytes + 1024));
+        if (per_sm < 1) per_sm = 1;
+        const int by_threads = 2048 / threads;
+        if (per_sm > by_threads) per_sm = by_threads;
+        if (blocks > (int64_t)kSMs * per_sm) blocks = (int64_t)kSMs * per_sm;
+        cudaError_t e = cudaFuncSetAttribute(k_fitness_packed<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kMaxSmemPerBlock);
+        if (e != cudaSuccess) return e;
+        k_fitness_packed<true, 4><<<(int)blocks, threads, lut_bytes, s>>>(rows, ld8, n, t, capacity, penalty, F, G);
+    } else {
+        if (blocks > (int64_t)kSMs * (2048 / threads)) blocks = (int64_t)kSMs * (2048 / threads);
+        k_fitness_packed<false, 4><<<(int)blocks, threads, 0, s>>>(rows, ld8, n, t, capacity, penalty, F, G);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Top-e selection (score descending, index ascending): per-block partial lists, then one block
 // merges them.  Scores are mapped to order-preserving 64-bit keys; NaN ranks lowest.
 // ---------------------------------------------------------------------------------------------

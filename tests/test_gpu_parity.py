@@ -469,6 +469,60 @@ def test_per_gpu_refresh_limits(ones):
     assert ((g.get_population() >= -1) & (g.get_population() < 4)).all()
 
 
+# ---- packed candidates: one byte per gene --------------------------------------------------------------
+def _pack_numpy(rows, J):
+    """The packed layout restated: tiles of 512 genes, byte 16*l + 4*b + s = gene 128*b + 4*l + s of the tile."""
+    n = rows.shape[0]
+    ld8 = (J + 511) // 512 * 512
+    genes = np.full((n, ld8), 255, dtype=np.int64)
+    genes[:, :J] = np.where((rows[:, :J] < 0) | (rows[:, :J] > 254), 255, rows[:, :J])
+    j = np.arange(ld8)
+    tile, r = j // 512, j % 512
+    b, q = r // 128, r % 128
+    where = tile * 512 + 16 * (q // 4) + 4 * b + q % 4
+    out = np.zeros((n, ld8), dtype=np.uint8)
+    out[:, where] = genes[:, j].astype(np.uint8)
+    return out
+
+
+@pytest.mark.parametrize("J,N", [(1, 3), (5, 9), (127, 40), (129, 33), (511, 20), (513, 70), (700, 5000), (2048, 300)])
+def test_packed_candidates_score_like_int32_rows(ones, J, N):
+    w = inputs.custom(J, max(4, J), N, 1, seed=J + N, kmax=7, kmin_max=2)
+    g, o = _pair(ones, w)
+    ld = (J + 3) // 4 * 4 + 8
+    rows = inputs.random_genomes(w.jobs, N, ld=ld, seed=J, waiting_fraction=0.05)
+    rows[0, :J] = 9                      # above every job's limit: a zero table entry, not a waiting job
+    rows[N // 2, J // 2] = 300           # out of the byte range: stored as "waits"
+    dev = torch.from_numpy(rows).cuda()
+    packed = g.pack(dev)
+    assert packed.shape == (N, (J + 511) // 512 * 512)
+    assert (packed.cpu().numpy() == _pack_numpy(rows, J)).all()
+    Fp, Gp = g.evaluate_packed(packed)
+    Fi, Gi = g.evaluate(dev)
+    Fo, Go = o.evaluate(rows)
+    assert (Fp.cpu().numpy() == Fi.cpu().numpy()).all() and (Gp.cpu().numpy() == Gi.cpu().numpy()).all()
+    assert (Gp.cpu().numpy() == Go).all() and _rel_err(Fp.cpu().numpy(), Fo) <= REL_TOL
+    assert (Fp.cpu().numpy() == Fo).all()
+    # the handle's own population
+    g.randomize(3)
+    o.randomize(3)
+    F2, G2 = g.evaluate_packed(g.pack())
+    assert (F2.cpu().numpy() == o.evaluate()[0]).all() and (G2.cpu().numpy() == o.evaluate()[1]).all()
+
+
+def test_packed_candidates_errors(ones):
+    w = inputs.tiny()
+    g = ones.Search(w.jobs, w.capacity, w.pop)
+    bad = torch.zeros((4, 1000), dtype=torch.uint8, device="cuda")    # stride not a multiple of 512
+    with pytest.raises(ones.OnesError) as err:
+        g.evaluate_packed(bad)
+    assert err.value.code == -4
+    p = ones.Search(w.jobs, w.capacity, w.pop, inputs.SearchParams(flags=16))
+    with pytest.raises(ones.OnesError) as err:
+        p.pack()
+    assert err.value.code == -3
+
+
 # ---- a6: best and repair ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "paper", "mid"])
 def test_best_and_repair_parity(ones, name):
