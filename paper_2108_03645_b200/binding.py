@@ -143,7 +143,7 @@ class Search:
     """One ``ones_ctx``: a population of candidate schedules on the current CUDA device."""
 
     def __init__(self, jobs: np.ndarray, capacity: int, pop: int, params: SearchParams | None = None, *,
-                 n_jobs_max: int | None = None):
+                 n_jobs_max: int | None = None, guard_bytes: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self._h = C.c_void_p()
@@ -162,13 +162,23 @@ class Search:
         if nbytes == 0:
             raise OnesError(-3, "ones_workspace_bytes")
         self.device = torch.device("cuda", torch.cuda.current_device())
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        # guard_bytes > 0 (a multiple of 256): the workspace sits between two guard areas filled with a
+        # pattern, and guards_intact() tells whether any kernel wrote outside the workspace it was given
+        assert guard_bytes % 256 == 0
+        self._guard = int(guard_bytes)
+        self._arena = torch.full((nbytes + 2 * self._guard,), 0xA5, dtype=torch.uint8, device=self.device)
+        self.workspace = self._arena[self._guard:self._guard + nbytes]
         prm = ones_params(p.elitism, p.tournament, p.p_mut, p.penalty, p.flags)
         rc = lib().ones_create(C.byref(self._h), _np_ptr(jobs), self.J, capacity, pop, C.byref(prm),
                                _t_ptr(self.workspace), nbytes, _stream_ptr())
         if rc:
             self._h = C.c_void_p()
             raise OnesError(rc, "ones_create")
+
+    def guards_intact(self) -> bool:
+        torch.cuda.synchronize()
+        g = self._guard
+        return g == 0 or bool((self._arena[:g] == 0xA5).all() and (self._arena[-g:] == 0xA5).all())
 
     # -- lifetime ---------------------------------------------------------------
     def close(self):

@@ -584,6 +584,39 @@ def test_update_jobs_parity(ones):
     assert err.value.code == -5
 
 
+# ---- no kernel writes outside the memory it was given ------------------------------------------------
+@pytest.mark.parametrize("flags,J,gpus,N", [(0, 37, 48, 101), (0, 300, 256, 6000), (2, 129, 64, 257), (8, 260, 128, 1025),
+                                            (4, 130, 64, 257), (16, 37, 130, 101), (16, 300, 257, 129), (1, 64, 64, 500)])
+def test_workspace_and_output_guards(ones, flags, J, gpus, N):
+    """Every launch sequence with the workspace and the caller's output arrays between guard areas."""
+    w = inputs.custom(J, gpus, N, 2, seed=J + N, kmax=6, kmin_max=1)
+    g = ones.Search(w.jobs, gpus, N, inputs.SearchParams(flags=flags), n_jobs_max=J + 40, guard_bytes=4096)
+    g.randomize(1)
+    g.evolve(3, 1)
+    g.best(repair=not flags & 16)
+    jobs2 = np.concatenate([w.jobs[5:], inputs.custom(9, gpus, 4, 1, seed=3, kmax=2).jobs])
+    remap = np.concatenate([np.arange(5, J), np.full(9, -1)]).astype(np.int32)
+    g.update_jobs(jobs2, remap, gpus)
+    g.evolve(2, 2)
+    g.best()
+    # outputs of ones_evaluate between guards of their own
+    W = g.W
+    ld = (W + 3) // 4 * 4
+    rows = g.get_population(on_device=True, ld=ld)
+    Fbig = torch.full((N + 64,), 7.25, dtype=torch.float64, device="cuda")
+    Gbig = torch.full((N + 64,), -77, dtype=torch.int32, device="cuda")
+    g.evaluate(rows, out=(Fbig[32:32 + N], Gbig[32:32 + N]))
+    torch.cuda.synchronize()
+    assert (Fbig[:32] == 7.25).all() and (Fbig[32 + N:] == 7.25).all()
+    assert (Gbig[:32] == -77).all() and (Gbig[32 + N:] == -77).all()
+    if not flags & 16:
+        packed = g.pack()
+        g.evaluate_packed(packed, out=(Fbig[32:32 + N], Gbig[32:32 + N]))
+        torch.cuda.synchronize()
+        assert (Fbig[:32] == 7.25).all() and (Fbig[32 + N:] == 7.25).all()
+    assert g.guards_intact()
+
+
 # ---- errors ------------------------------------------------------------------------------------
 def test_errors_are_codes_not_faults(ones):
     w = inputs.tiny()
