@@ -312,6 +312,22 @@ def test_truncation_selection_parity(ones, J, N, kw):
     assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"]
 
 
+def test_truncation_selection_parity_large_job_table(ones):
+    """The paper's scheme on the benchmark's job table with a pool larger than L2 (4 x 32768 rows of 2048 genes =
+    1 GiB per buffer): every survivor, score and GPU count of one generation against the oracle."""
+    import dataclasses
+    w = dataclasses.replace(inputs.large(), pop=32768)
+    g, o = _pair(ones, w, flags=4)
+    g.randomize(w.seed)
+    o.randomize(w.seed)
+    g.evolve(1, w.seed)
+    o.evolve(1, w.seed)
+    pg, _ = g.last_parents()
+    po, _ = o.last_parents()
+    assert (pg == po).all()
+    _same_state(g, o)
+
+
 def test_truncation_selection_with_many_ties(ones):
     # identical candidates: every score ties, survivors are decided by row order alone
     w = inputs.tiny()
