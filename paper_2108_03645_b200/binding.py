@@ -166,7 +166,10 @@ class Search:
         # pattern, and guards_intact() tells whether any kernel wrote outside the workspace it was given
         assert guard_bytes % 256 == 0
         self._guard = int(guard_bytes)
-        self._arena = torch.full((nbytes + 2 * self._guard,), 0xA5, dtype=torch.uint8, device=self.device)
+        self._arena = torch.empty(nbytes + 2 * self._guard, dtype=torch.uint8, device=self.device)
+        if self._guard:
+            self._arena[:self._guard].fill_(0xA5)
+            self._arena[-self._guard:].fill_(0xA5)
         self.workspace = self._arena[self._guard:self._guard + nbytes]
         prm = ones_params(p.elitism, p.tournament, p.p_mut, p.penalty, p.flags)
         rc = lib().ones_create(C.byref(self._h), _np_ptr(jobs), self.J, capacity, pop, C.byref(prm),
