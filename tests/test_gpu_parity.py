@@ -167,15 +167,28 @@ def test_evolve_parity_named_workloads(ones, name, gens, flags):
     assert bg["total_gpus"] <= w.capacity
 
 
-def test_evolve_parity_mid_sampled_generations(ones):
+def test_evolve_parity_mid_all_generations(ones):
+    """The mid workload for all of its 200 generations: parents, elites, genomes, GPU demand and scores against the
+    oracle at generations 1, 2, 10, 50 and 200 (near-ties between fp64 scores decide tournaments, and only a long
+    run at scale meets many of them)."""
     w = inputs.mid()
     g, o = _pair(ones, w)
-    g.randomize(3)
-    o.randomize(3)
-    for step in (1, 2):
-        g.evolve(step, 3)
-        o.evolve(step, 3)
+    g.randomize(w.seed)
+    o.randomize(w.seed)
+    done = 0
+    for upto in (1, 2, 10, 50, w.generations):
+        g.evolve(upto - done, w.seed)
+        o.evolve(upto - done, w.seed)
+        done = upto
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all(), upto
         _same_state(g, o)
+        assert g.generation == o.generation == done
+    bg, bo = g.best(True), o.best(True)
+    for key in ("genome", "gpus_per_job", "rate_per_job"):
+        assert (bg[key] == bo[key]).all(), key
+    assert bg["fitness"] == bo["fitness"] and bg["total_gpus"] == bo["total_gpus"] <= w.capacity
 
 
 @pytest.mark.parametrize("kw", [dict(elitism=0), dict(elitism=1), dict(elitism=5, tournament=1),
@@ -657,19 +670,20 @@ def test_errors_are_codes_not_faults(ones):
 
 
 # ---- full size, in the configuration the benchmark times --------------------------------------------
-@pytest.mark.parametrize("flags", [0, 2])  # children scored inside the evolve kernel / by a separate pass
-def test_large_config_parity_full_population(ones, flags):
+@pytest.mark.parametrize("flags,gens", [(0, 3), (2, 1)])  # children scored inside the evolve kernel / by a separate pass
+def test_large_config_parity_full_population(ones, flags, gens):
     w = inputs.large()
     g, o = _pair(ones, w, flags=flags)
     g.randomize(w.seed)
     o.randomize(w.seed)
     assert (g.get_population() == o.get_population()).all()
-    g.evolve(1, w.seed)
-    o.evolve(1, w.seed)
-    pg, eg = g.last_parents()
-    po, eo = o.last_parents()
-    assert (pg == po).all() and (eg == eo).all()
-    _same_state(g, o)
+    for _ in range(gens):
+        g.evolve(1, w.seed)
+        o.evolve(1, w.seed)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
     # invariants that hold at any size
     P = g.get_population()
     assert (P >= w.jobs["kmin"][None, :]).all() and (P <= w.jobs["kmax"][None, :]).all()
@@ -678,3 +692,48 @@ def test_large_config_parity_full_population(ones, flags):
     assert g.best()["fitness"] >= b0
     rep = g.best(True)
     assert rep["total_gpus"] <= w.capacity
+
+
+def test_large_config_generation_200_recomputed_from_generation_199(ones):
+    """The last generation of the large workload (2048 jobs, population 65536, 200 generations), in the launch
+    sequence the benchmark times.  The random draws are keyed by (seed, generation, row, job), so any generation
+    can be recomputed on its own: the oracle is given the GPU's population of generation 199 and the generation
+    counter, scores it, and derives generation 200, which must equal the GPU's row for row (every tournament,
+    elite, child gene, GPU demand and score).  On top, sampled pairs are re-derived from the oracle's stateless
+    steps alone (tournament over the GPU's scores of generation 199; score of the GPU's child rows)."""
+    w = inputs.large()
+    p = w.params
+    g, o = _pair(ones, w)
+    g.randomize(w.seed)
+    g.evolve(w.generations - 1, w.seed)
+    P199 = g.get_population()
+    F199 = g.evaluate()[0].cpu().numpy()
+    o.set_population(P199)
+    o.set_generation(w.generations - 1)
+    Fo, _ = o.evaluate()
+    assert (F199 == Fo).all()
+    # after 199 generations the search has moved well away from its start
+    g0, _ = _pair(ones, w)
+    g0.randomize(w.seed)
+    assert F199.max() > g0.evaluate()[0].max().item()
+    g.evolve(1, w.seed)
+    o.evolve(1, w.seed)
+    assert g.generation == o.generation == w.generations
+    pg, eg = g.last_parents()
+    po, eo = o.last_parents()
+    assert (pg == po).all() and (eg == eo).all()
+    _same_state(g, o)
+    # stateless re-derivation of sampled pairs
+    P200 = g.get_population()
+    F200, G200 = (t.cpu().numpy() for t in g.evaluate())
+    rng = np.random.default_rng(200)
+    pairs = pg.shape[0]
+    for q in [0, pairs - 1] + rng.integers(0, pairs, size=254).tolist():
+        for side, stream in ((0, oracle.STREAM_SEL_A), (1, oracle.STREAM_SEL_B)):
+            assert pg[q, side] == oracle.tournament(F199, p.tournament, w.seed, w.generations - 1, q, stream)
+        for row in (p.elitism + 2 * q, p.elitism + 2 * q + 1):
+            Fr, Gr = oracle.fitness(w.jobs, w.capacity, p.penalty, P200[row])
+            assert F200[row] == Fr and G200[row] == Gr
+            assert np.isin(P200[row], [0, 1, 2, 3, 4, 5, 6, 7]).all()
+    for r in range(p.elitism):
+        assert (P200[r] == P199[eg[r]]).all()

@@ -137,3 +137,28 @@ def test_online_loop_gpu_matches_oracle():
     for (ra, ia, ga), (rb, ib, gb) in zip(a.deployed, b.deployed):
         assert ra == rb and ia == ib and (ga == gb).all()
     assert (a.jct == b.jct).all()
+
+
+@pytest.mark.gpu
+def test_online_loop_full_trace_gpu_matches_oracle():
+    """The online workload as specified: 2000 jobs, 256 GPUs, population 4096, 50 generations per round, every
+    round of the trace.  Deployed schedules, GPU totals, best score per round and the completion time of every
+    job must equal the oracle's."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2108_03645_b200 import binding
+
+    def gpu_engine(jobs, capacity, pop, params, n_jobs_max):
+        return binding.Search(jobs, capacity, pop, params, n_jobs_max=n_jobs_max)
+
+    tr = inputs.online_trace()
+    assert tr.jobs.shape[0] == 2000 and tr.capacity == 256 and tr.pop == 4096 and tr.generations == 50
+    a = online.simulate(tr, gpu_engine, keep_schedules=True, sync=torch.cuda.synchronize)
+    b = online.simulate(tr, oracle_engine, keep_schedules=True)
+    assert a.rounds == b.rounds > 900 and a.active == b.active
+    assert a.gpus_used == b.gpus_used and max(a.gpus_used) <= tr.capacity
+    assert a.best_fitness == b.best_fitness
+    for (ra, ia, ga), (rb, ib, gb) in zip(a.deployed, b.deployed):
+        assert ra == rb and ia == ib and (ga == gb).all(), ra
+    assert np.isfinite(a.jct).all() and (a.jct == b.jct).all()
