@@ -122,14 +122,34 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------
 # CPU oracle on a bounded sample of the workload
 # ----------------------------------------------------------------------------------------------
-def oracle_sample(w, pop_sample: int, gens: int):
-    """Seconds for `gens` generations of a `pop_sample`-candidate population (single thread)."""
+def host_info():
+    """The host the CPU figures were taken on: logical cores and the CPU model string."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for ln in fh:
+                if ln.lower().startswith(("model name", "cpu model", "cpu\t")):
+                    model = ln.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"host_cores": os.cpu_count(), "host_cpu": model}
+
+
+def oracle_search(w, pop_sample: int):
+    """An oracle handle over a `pop_sample`-candidate population, randomised and scored (set-up, not timed)."""
     import oracle
     p = w.params
     s = oracle.Search(w.jobs, w.capacity, pop_sample, elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut,
                       penalty=p.penalty, flags=p.flags)
     s.randomize(w.seed)
     s.evaluate()
+    return s
+
+
+def oracle_sample(w, pop_sample: int, gens: int):
+    """Seconds for `gens` generations of a `pop_sample`-candidate population (single thread)."""
+    s = oracle_search(w, pop_sample)
     t0 = time.perf_counter()
     s.evolve(gens, w.seed)
     dt = time.perf_counter() - t0
@@ -142,35 +162,39 @@ def cpu_baseline(w, pop_sample=8192, gens=None):
     if w.params.flags & 16:
         # per-GPU genome: the oracle's reorder costs slots x jobs per row (about 3.5 ms at 4096 x 2048)
         pop_sample, gens = min(pop_sample, 1024), 4
-    if gens is None:  # about 1e8 gene evaluations: seconds of single-thread work
-        gens = int(min(2000, max(8, 1.3e8 / (pop_sample * w.n_jobs))))
+    if gens is None:  # about 3e8 gene evaluations: 10-20 s of single-thread work
+        gens = int(min(2000, max(8, 3e8 / (pop_sample * w.n_jobs))))
     dt = oracle_sample(w, pop_sample, gens)
-    return {"value": pop_sample * gens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{gens} generations of a {pop_sample}-candidate population (of {w.pop}), "
-                      f"{w.n_jobs} jobs, same job table and parameters; {dt:.1f} s"}
+    return dict({"value": pop_sample * gens / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                 "sample": f"{gens} generations of a {pop_sample}-candidate population (of {w.pop}), "
+                           f"{w.n_jobs} jobs, same job table and parameters; {dt:.1f} s"}, **host_info())
 
 
 def run_reference(args, w):
-    """The reference arm: the CPU oracle as it stands, each step a bounded sample."""
+    """The reference arm: the CPU oracle as it stands; each step is one generation of a bounded sample of the
+    population.  Handle creation, the random initial population and its first scoring are set-up and stay
+    outside the clock, as they do in the GPU arm and in `cpu_baseline`."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     pop_sample = min(8192, w.pop)
-    for _ in range(min(args.warmup, 1)):
-        oracle_sample(w, pop_sample, 1)
-    steps = max(1, min(args.steps, 20))
+    s = oracle_search(w, pop_sample)
+    warm = min(max(args.warmup, 0), 5)
+    s.evolve(warm, w.seed)
+    steps = max(1, min(args.steps, 40))
     t0 = time.perf_counter()
-    for _ in range(steps):
-        oracle_sample(w, pop_sample, 1)
+    s.evolve(steps, w.seed)
     dt = time.perf_counter() - t0
+    s.close()
     value = pop_sample * steps / dt
     sample = (f"each step = 1 generation of a {pop_sample}-candidate population (of {w.pop}), {w.n_jobs} jobs, "
-              f"single thread; {steps} steps timed (capped at 20)")
+              f"single thread; {steps} steps timed (capped at 40), {warm} warm-up (capped at 5)")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps,
+            "steps": steps, "warmup": warm, "ms_per_step": 1e3 * dt / steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "jobs": w.n_jobs, "population": w.pop, "capacity": w.capacity},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": config_of(w, max(args.gpus, 1)),
+            "cpu_baseline": dict({"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+                                 **host_info()),
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -179,11 +203,12 @@ def run_reference(args, w):
 # ----------------------------------------------------------------------------------------------
 # online loop: per-round search latency and simulated job completion time
 # ----------------------------------------------------------------------------------------------
-def run_online(args):
+def online_figures(oracle_rounds: int):
+    """The 2000-job trace through the library (every round), and its first `oracle_rounds` rounds through the
+    CPU oracle (0: skipped).  Returns the figures of the online workload as a dict."""
     import torch
     from paper_2108_03645_b200 import binding, online
 
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     trace = inputs.online_trace()
 
     def gpu_engine(jobs, capacity, pop, params, n_jobs_max):
@@ -197,50 +222,156 @@ def run_online(args):
     online.simulate(trace, gpu_engine, max_rounds=20, sync=torch.cuda.synchronize)  # warm-up
     res = online.simulate(trace, gpu_engine, keep_schedules=True, sync=torch.cuda.synchronize)
     lat = np.array(res.latency_s) * 1e3
-    line = {"metric": "online_round_latency_ms", "value": float(lat.mean()), "unit": "ms per scheduling round "
+    out = {"what": "ones_update_jobs + 50 generations of a 4096-candidate population + ones_best with repair, per "
+                   "60 s scheduling round of the 2000-job trace on 256 GPUs (host wall clock around the three calls)",
+           "rounds": res.rounds, "mean_ms": float(lat.mean()), "p50_ms": float(np.percentile(lat, 50)),
+           "p99_ms": float(np.percentile(lat, 99)), "max_ms": float(lat.max()),
+           "mean_active_jobs": float(np.mean(res.active)), "max_active_jobs": int(max(res.active)),
+           "mean_jct_s": res.mean_jct, "jobs_finished": int(np.isfinite(res.jct).sum()),
+           "trace_jobs": int(trace.jobs.shape[0]), "capacity": trace.capacity, "population": trace.pop,
+           "generations_per_round": trace.generations, "period_s": trace.period_s}
+    if oracle_rounds > 0:
+        t0 = time.perf_counter()
+        ref = online.simulate(trace, cpu_engine, max_rounds=oracle_rounds, keep_schedules=True)
+        dt = time.perf_counter() - t0
+        same = len(ref.deployed) == min(oracle_rounds, res.rounds) and all(
+            ra == rb and ia == ib and (ga == gb).all() for (ra, ia, ga), (rb, ib, gb) in zip(res.deployed, ref.deployed))
+        same = same and ref.best_fitness == res.best_fitness[:len(ref.best_fitness)]
+        out["cpu_oracle"] = dict({"mean_ms": 1e3 * float(np.mean(ref.latency_s)), "rounds": ref.rounds, "cores": 1,
+                                  "kind": "oracle", "sample": f"first {ref.rounds} rounds of the same trace; {dt:.1f} s",
+                                  "schedules_identical_to_gpu": bool(same)}, **host_info())
+    return out
+
+
+def run_online(args):
+    import torch
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    f = online_figures(0 if args.no_cpu_baseline else 100)
+    line = {"metric": "online_round_latency_ms", "value": f["mean_ms"], "unit": "ms per scheduling round "
             "(ones_update_jobs + 50 generations of a 4096-candidate population + ones_best with repair)",
             "n_gpus": 1, "higher_is_better": False, "data": "synthetic", "dtype": "f64",
-            "config": {"workload": "online", "trace_jobs": int(trace.jobs.shape[0]), "capacity": trace.capacity,
-                       "population": trace.pop, "generations_per_round": trace.generations,
-                       "period_s": trace.period_s},
-            "rounds": res.rounds, "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
-            "max_ms": float(lat.max()), "mean_active_jobs": float(np.mean(res.active)),
-            "max_active_jobs": int(max(res.active)), "mean_jct_s": res.mean_jct,
-            "jobs_finished": int(np.isfinite(res.jct).sum())}
-    if not args.no_cpu_baseline:
-        k = 12
-        t0 = time.perf_counter()
-        ref = online.simulate(trace, cpu_engine, max_rounds=k, keep_schedules=True)
-        dt = time.perf_counter() - t0
-        same = all(ia == ib and (ga == gb).all() for (_, ia, ga), (_, ib, gb) in zip(res.deployed, ref.deployed))
-        line["cpu_baseline"] = {"value": 1e3 * float(np.mean(ref.latency_s)), "unit": "ms per scheduling round",
-                                "cores": 1, "kind": "oracle",
-                                "sample": f"first {k} rounds of the same trace; {dt:.1f} s",
-                                "schedules_identical_to_gpu": bool(same)}
+            "config": {"workload": "online", "trace_jobs": f["trace_jobs"], "capacity": f["capacity"],
+                       "population": f["population"], "generations_per_round": f["generations_per_round"],
+                       "period_s": f["period_s"]},
+            "rounds": f["rounds"], "p50_ms": f["p50_ms"], "p99_ms": f["p99_ms"], "max_ms": f["max_ms"],
+            "mean_active_jobs": f["mean_active_jobs"], "max_active_jobs": f["max_active_jobs"],
+            "mean_jct_s": f["mean_jct_s"], "jobs_finished": f["jobs_finished"]}
+    if "cpu_oracle" in f:
+        c = f["cpu_oracle"]
+        line["cpu_baseline"] = dict(c, value=c["mean_ms"], unit="ms per scheduling round")
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------------------------
+# timing helpers
+# ----------------------------------------------------------------------------------------------
+def timed_repeats(run_steps, min_s: float, max_repeats: int = 4000):
+    """Time `run_steps()` (which enqueues exactly K steps on the current stream) repeatedly: one untimed
+    call sizes the repeat count so that the timed region lasts at least `min_s`, then every repeat is
+    bracketed by its own pair of CUDA events.  Returns the per-repeat milliseconds."""
+    import torch
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    run_steps()
+    torch.cuda.synchronize()
+    once = max(time.perf_counter() - t0, 1e-6)
+    repeats = int(min(max_repeats, max(3, np.ceil(min_s / once))))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(repeats)]
+    for e0, e1 in evs:
+        e0.record()
+        run_steps()
+        e1.record()
+    torch.cuda.synchronize()
+    return [e0.elapsed_time(e1) for e0, e1 in evs]
+
+
+def small_workload_figures(binding, name: str, min_s: float = 0.25):
+    """Generations/s of one of the cache-resident workloads: repeats of its own generation count."""
+    w = inputs.WORKLOADS[name]()
+    s = binding.Search(w.jobs, w.capacity, w.pop, w.params)
+    s.randomize(w.seed)
+    s.evolve(w.generations, w.seed)
+    l0 = s.kernel_launches
+    ms = timed_repeats(lambda: s.evolve(w.generations, w.seed), min_s)
+    launches = (s.kernel_launches - l0) / (len(ms) + 1)
+    per_gen_ms = statistics.median(ms) / w.generations
+    s.close()
+    return {"jobs": w.n_jobs, "population": w.pop, "generations_per_call": w.generations,
+            "us_per_generation": 1e3 * per_gen_ms, "generations_per_s": 1e3 / per_gen_ms,
+            "candidate_evals_per_s": w.pop * 1e3 / per_gen_ms, "launches_per_call": launches,
+            "timed_calls": len(ms), "hbm": "n/a (population resident in L2 or shared memory)"}
+
+
+def sha16(path: str) -> str:
+    import hashlib
+    with open(path, "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()[:16]
+
+
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of this
-# benchmark's default workload at its full population (profiles/dram_traffic_large_pop65536.md).  They belong
-# to the kernels as they were when the capture was taken: set an entry to None when its kernel changes.
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("large", 65536, "k_evolve_score"): 403.6e6 + 485.2e6,
-    ("large", 65536, "k_evolve"): 401.6e6 + 483.0e6,
-    ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
+# benchmark's default workload at its full population.  A figure belongs to the kernel source it was
+# captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
+# traffic as null whenever the file it runs differs from it.
+NCU_TRAFFIC = {
+    "captured_at": "b88a7a4",
+    "source_sha16": "",
+    "bytes_per_launch": {
+        ("large", 65536, "k_evolve_score"): 403.6e6 + 485.2e6,
+        ("large", 65536, "k_evolve"): 401.6e6 + 483.0e6,
+        ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
+    },
 }
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2108_03645_b200", "csrc", "ones_kernels.cu")
+
+
+def ncu_traffic(workload: str, pop: int, kernel: str):
+    """(bytes per launch or None, commit of the capture)."""
+    try:
+        current = sha16(KERNEL_SOURCE)
+    except OSError:
+        current = None
+    if current != NCU_TRAFFIC["source_sha16"]:
+        return None, NCU_TRAFFIC["captured_at"]
+    return NCU_TRAFFIC["bytes_per_launch"].get((workload, pop, kernel)), NCU_TRAFFIC["captured_at"]
+
+
+def roofline_entry(kernel, nbytes, t_ms, peak, peak_kind, traffic, captured_at, **more):
+    """HBM roofline of one kernel: `achieved` counts the algorithmic bytes; where an ncu capture of the DRAM
+    bytes of this very kernel exists, the rate on those bytes is reported beside it (`dram_*`)."""
+    a = nbytes / (t_ms * 1e-3) / 1e9
+    r = {"kernel": kernel, "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
+         "peak_kind": f"of {peak_kind}", "traffic": traffic, "traffic_captured_at": captured_at,
+         "bytes_per_launch": nbytes, "ms_per_launch": t_ms, "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS}
+    if traffic:
+        d = traffic / (t_ms * 1e-3) / 1e9
+        r.update({"dram_achieved": d, "dram_frac": d / peak, "dram_frac_of_nominal_8TBs": d / NOMINAL_HBM_GBS})
+    r.update(more)
+    return r
+
+
+def config_of(w, world: int):
+    return {"workload": w.name, "jobs": w.n_jobs, "population": w.pop, "capacity": w.capacity,
+            "elitism": w.params.elitism, "tournament": w.params.tournament, "p_mut": w.params.p_mut,
+            "genome_table_bytes": w.pop * w.n_jobs * 4,
+            "l2": "inputs larger than L2 (two population buffers of genome_table_bytes each against 126 MB)"
+                  if w.pop * w.n_jobs * 4 > 2 * 126e6 else "population fits L2: cache-resident",
+            "parallelism": "replicas" if world > 1 else "single GPU"}
 
 
 # ----------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(inputs.WORKLOADS) + ["online"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-events", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the figures of the other workloads")
+    ap.add_argument("--min-seconds", type=float, default=0.5,
+                    help="the K timed steps are repeated until the timed region lasts this long")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (profiling a smaller case)")
     ap.add_argument("--scheme", default="tournament", choices=["tournament", "truncation", "per_gpu"],
                     help="truncation = the paper's best-K-of-4K selection (ONES_FLAG_TRUNCATION); per_gpu = the "
@@ -274,8 +405,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     warmup = max(args.warmup, 3)
     steps = max(args.steps, 1)
+    solo = rank == 0 and world == 1
 
-    base = cpu_baseline(w) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    base = cpu_baseline(w) if (solo and not args.no_cpu_baseline) else None
 
     seed = rank_seed(w.seed, rank)
     s = binding.Search(w.jobs, w.capacity, w.pop, w.params)
@@ -283,62 +415,64 @@ def main():
     s.evolve(warmup, seed)
     torch.cuda.synchronize()
 
-    # ---- device-resident timed region: K generations ----
-    if not args.no_kernel_events:
-        s.set_profiling(8 if steps >= 64 else 1)  # event pairs around every 8th generation's kernels
-        s.stage_times()
-    sampler = ClockSampler(local)
+    # ---- device-resident timed region: repeats of exactly K generations, each repeat between its own
+    # pair of CUDA events on the handle's stream; no per-kernel events are recorded inside it ----
+    sampler = ClockSampler(local, period_s=0.002)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = s.kernel_launches
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
-    ev0.record()
-    s.evolve(steps, seed)
-    ev1.record()
+    t_wall = time.perf_counter()
+    rep_ms = timed_repeats(lambda: s.evolve(steps, seed), args.min_seconds)
     torch.cuda.synchronize()
+    timed_region_s = time.perf_counter() - t_wall
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
-    ms = ev0.elapsed_time(ev1)
-    launches = s.kernel_launches - launches0
+    launches = (s.kernel_launches - launches0) / (len(rep_ms) + 1)  # per K steps (one untimed sizing call)
+    ms = max_over_ranks(statistics.median(rep_ms), "cuda")
+
+    # ---- per-kernel durations: a separate pass with an event pair around every kernel ----
     stage_ms, stage_n = ({}, {})
     if not args.no_kernel_events:
+        s.set_profiling(1)
+        s.stage_times()
+        s.evolve(max(steps, 100) if w.pop * w.n_jobs >= (1 << 24) else steps, seed)
         stage_ms, stage_n = s.stage_times()
         s.set_profiling(False)
-    ms = max_over_ranks(ms, "cuda")
 
     # ---- end to end: every step uploads the job table and reads the best schedule back ----
     J, N, E = w.n_jobs, w.pop, w.params.elitism
-    e2e_steps = 0 if args.no_e2e else min(steps, 100)
     identity = np.arange(J, dtype=np.int32)
     jobs_pinned = torch.from_numpy(w.jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
     jobs_host = jobs_pinned.numpy().view(inputs.JOB_DTYPE)
     out = {"fitness": None}
-    e2e_s = float("nan")
-    if e2e_steps:
-        for _ in range(3):
-            s.update_jobs(jobs_host, identity, w.capacity)
-            s.evolve(1, seed)
-            s.best(False)
+    e2e_ms, e2e_reps = float("nan"), 0
+    if not args.no_e2e:
+        def e2e_steps():
+            for _ in range(steps):
+                s.update_jobs(jobs_host, identity, w.capacity)
+                s.evolve(1, seed)
+                out.update(s.best(False))
+        e2e_steps()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        t0 = time.perf_counter()
-        for _ in range(e2e_steps):
-            s.update_jobs(jobs_host, identity, w.capacity)
-            s.evolve(1, seed)
-            out = s.best(False)
-        torch.cuda.synchronize()
-        e2e_s = time.perf_counter() - t0
-        e2e_s = max_over_ranks(e2e_s, "cuda")
+        reps = []
+        t_all = time.perf_counter()
+        while len(reps) < 3 or (time.perf_counter() - t_all < 0.6 * args.min_seconds and len(reps) < 500):
+            t0 = time.perf_counter()
+            e2e_steps()  # ones_best synchronises: the host clock brackets the device work
+            reps.append(time.perf_counter() - t0)
+        e2e_ms = max_over_ranks(1e3 * statistics.median(reps), "cuda")
+        e2e_reps = len(reps)
     h2d = J * 48 + J * 4
-    d2h = J * (4 + 4 + 8) + 24 + 4
+    d2h = J * (4 + 4 + 8) + 64
 
     # ---- the two separate kernels (crossover/mutation, fitness) on the same workload ----
     sep = None
-    if rank == 0 and world == 1 and not args.no_kernel_events and args.scheme == "tournament":
+    if solo and not args.no_kernel_events and args.scheme == "tournament":
         import dataclasses
         s.close()
         del s
@@ -349,7 +483,7 @@ def main():
         s2.evolve(warmup, seed)
         s2.set_profiling(True)
         s2.stage_times()
-        s2.evolve(min(steps, 200), seed)
+        s2.evolve(min(max(steps, 50), 200), seed)
         sep = s2.stage_times()
         s2.set_profiling(False)
         # the score step on packed rows (one byte per gene); two copies read in turn so that a launch never
@@ -368,6 +502,14 @@ def main():
         packed_bytes = packs[0].shape[0] * (packs[0].shape[1] + 12)
         del packs
         s2.close()
+        del s2
+        torch.cuda.empty_cache()
+
+    # ---- the other workloads, measured in the same run ----
+    others = None
+    if solo and not args.no_workloads and args.scheme == "tournament" and not args.pop:
+        others = {name: small_workload_figures(binding, name) for name in ("tiny", "paper", "mid") if name != w.name}
+        others["online"] = online_figures(0 if args.no_cpu_baseline else 100)
 
     if rank != 0:
         if world > 1:
@@ -379,53 +521,52 @@ def main():
         "metric": METRIC, "value": whole_job_rate(world, N, steps, ms), "unit": UNIT, "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "jobs": J, "population": N, "capacity": w.capacity,
-                   "elitism": E, "tournament": w.params.tournament, "p_mut": w.params.p_mut,
-                   "genome_table_bytes": N * J * 4, "l2": "inputs larger than L2 (two 512 MiB population buffers)",
-                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "config": config_of(w, world),
         "generations_per_s": world * steps / (ms * 1e-3),
-        "gpu_launches": launches,
+        "gpu_launches": int(round(launches)),
+        "timing": {"timed_repeats": len(rep_ms), "steps_per_repeat": steps, "ms_per_repeat_median": ms,
+                   "ms_per_repeat_min": min(rep_ms), "ms_per_repeat_max": max(rep_ms),
+                   "timed_region_s": timed_region_s,
+                   "how": "the K steps are repeated back to back until the timed region lasts --min-seconds; each "
+                          "repeat has its own CUDA-event pair on the launching stream, the median repeat is reported; "
+                          "per-kernel events are recorded in a separate pass afterwards"},
         "clocks": clocks,
-        "e2e": None if not e2e_steps else {"value": world * N * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs)",
-                "best_fitness": out["fitness"]},
+        "e2e": None if not e2e_reps else {
+            "value": world * N * steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": steps, "ms_per_step": e2e_ms / steps, "timed_repeats": e2e_reps,
+            "what": "per step: ones_update_jobs(host job table) + ones_evolve(1) + ones_best(host outputs); host wall "
+                    "clock, median repeat",
+            "best_fitness": out["fitness"]},
     }
     if args.scheme == "per_gpu":
         Wg = w.capacity
         line["config"]["scheme"] = f"per-GPU genome: {Wg} slots per candidate, reorder after crossover and mutation"
         if stage_n.get("evolve"):
-            peak, peak_kind = measured_peak()
             rows = {"k_evolve": ("evolve", 8 * Wg * N),
                     "k_per_gpu<reorder, score>": ("fitness", N * (8 * Wg + 12)),
                     "k_select_stage": ("select", 8 * N)}
             line["kernels"] = {}
             for name, (stage, nbytes) in rows.items():
-                t_ms = stage_ms[stage] / stage_n[stage]
-                a = nbytes / (t_ms * 1e-3) / 1e9
-                line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                                         "bytes_per_generation": nbytes, "ms_per_generation": t_ms}
-            dom = max(line["kernels"].items(), key=lambda kv: kv[1]["ms_per_generation"])
-            line["roofline"] = dict(dom[1], kernel=dom[0], peak_kind=f"of {peak_kind}", traffic=None)
+                line["kernels"][name] = roofline_entry(name, nbytes, stage_ms[stage] / stage_n[stage], peak, peak_kind,
+                                                       None, None)
+            dom = max(line["kernels"].values(), key=lambda kv: kv["ms_per_launch"])
+            line["roofline"] = dict(dom)
     if args.scheme == "truncation":
         line["config"]["scheme"] = "truncation: pool of 4N rows, 3N new candidates scored per generation"
         line["new_candidates_per_s"] = 3 * line["value"]
         if stage_n.get("evolve"):
-            peak, peak_kind = measured_peak()
             if stage_n.get("fitness"):  # children written first, scored by a separate pass
                 rows = {"children (k_trunc_draws + k_trunc_children)": ("evolve", 6 * N * J * 4),
                         "k_fitness over the 3N new rows": ("fitness", 3 * N * (4 * J + 12))}
             else:  # 3N children written and scored in one pass: 3N row reads, 3N row writes, (F, G) of each
                 rows = {"children + scores (k_trunc_draws + k_trunc_children_score)": ("evolve", 6 * N * J * 4 + 3 * N * 12)}
-            rows["selection (radix threshold, compaction, k_trunc_gather)"] = ("select", 2 * N * J * 4 + 4 * N * 8 * 10)
+            rows["selection (threshold search, compaction, k_trunc_gather)"] = ("select", 2 * N * J * 4 + 4 * N * 8 * 3)
             line["kernels"] = {}
             for name, (stage, nbytes) in rows.items():
-                t_ms = stage_ms[stage] / stage_n[stage]
-                a = nbytes / (t_ms * 1e-3) / 1e9
-                line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                                         "bytes_per_generation": nbytes, "ms_per_generation": t_ms}
-            dom = max(line["kernels"].items(), key=lambda kv: kv[1]["ms_per_generation"])
-            line["roofline"] = dict(dom[1], kernel=dom[0], peak_kind=f"of {peak_kind}", traffic=None)
+                line["kernels"][name] = roofline_entry(name, nbytes, stage_ms[stage] / stage_n[stage], peak, peak_kind,
+                                                       None, None)
+            dom = max(line["kernels"].values(), key=lambda kv: kv["ms_per_launch"])
+            line["roofline"] = dict(dom)
     if stage_n.get("evolve") and args.scheme == "tournament":
         ev_ms = stage_ms["evolve"] / stage_n["evolve"]
         sel_ms = stage_ms["select"] / stage_n["select"] if stage_n.get("select") else 0.0
@@ -433,20 +574,17 @@ def main():
         # the elite rows, the pair/elite indices, and F and G of every candidate (scored in the same kernel)
         evolve_bytes = 8 * J * (N - E) + 8 * J * E + 8 * ((N - E + 1) // 2) + 4 * E
         fused_bytes = evolve_bytes + 12 * N
-        ach = fused_bytes / (ev_ms * 1e-3) / 1e9
         gens_per_launch = steps if launches < steps else 1  # the cluster path runs a whole call in one launch
         one_launch = launches <= steps
         kernel = "k_evolve_cluster" if launches < steps else ("k_generation" if one_launch else "k_evolve_score")
-        ach = fused_bytes * gens_per_launch / (ev_ms * 1e-3) / 1e9
-        line["roofline"] = {"kernel": kernel, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                            "frac": ach / peak, "peak_kind": f"of {peak_kind}",
-                            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, N, kernel)),
-                            "bytes_per_launch": fused_bytes * gens_per_launch, "ms_per_launch": ev_ms,
-                            "generations_per_launch": gens_per_launch,
-                            "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
-                            "note": "crossover + mutation + scoring of the children in one pass (dominant kernel of the "
-                                    "generation); shapes that fit one cluster's shared memory are latency-bound, their "
-                                    "fraction of the HBM rate is informational; the unfused kernels are under 'kernels'"}
+        traffic, at = ncu_traffic(w.name, N, kernel)
+        line["roofline"] = roofline_entry(
+            kernel, fused_bytes * gens_per_launch, ev_ms, peak, peak_kind, traffic, at,
+            generations_per_launch=gens_per_launch,
+            note="crossover + mutation + scoring of the children in one pass (dominant kernel of the generation), timed "
+                 "with an event pair around every launch in a pass of its own; shapes that fit one cluster's shared "
+                 "memory are latency-bound, their fraction of the HBM rate is informational; the unfused kernels are "
+                 "under 'kernels'")
         line["kernels"] = {"k_select_stage": {"ms_per_launch": sel_ms}} if sel_ms else {}
         if sep is not None:
             sep_ms, sep_n = sep
@@ -454,19 +592,16 @@ def main():
             f_ms = sep_ms["fitness"] / sep_n["fitness"]
             fitness_bytes = 4 * J * N + 12 * N
             for name, nbytes, t_ms in (("k_evolve", evolve_bytes, e_ms), ("k_fitness", fitness_bytes, f_ms)):
-                a = nbytes / (t_ms * 1e-3) / 1e9
-                line["kernels"][name] = {"bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                                         "bytes_per_launch": nbytes, "ms_per_launch": t_ms,
-                                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((w.name, N, name)),
-                                         "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
-                                         "how": "same workload with ONES_FLAG_UNFUSED (separate scoring pass)"}
-            a = packed_bytes / (packed_ms * 1e-3) / 1e9
-            line["kernels"]["k_fitness_packed"] = {
-                "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                "bytes_per_launch": packed_bytes, "ms_per_launch": packed_ms, "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
-                "candidate_evals_per_s": N / (packed_ms * 1e-3),
-                "how": "ones_evaluate_packed on the same population stored as one byte per gene (a variant beside the "
-                       "int32 contract); 20 launches back to back, two packed copies read in turn"}
+                traffic, at = ncu_traffic(w.name, N, name)
+                line["kernels"][name] = roofline_entry(name, nbytes, t_ms, peak, peak_kind, traffic, at,
+                                                       how="same workload with ONES_FLAG_UNFUSED (separate scoring pass)")
+            line["kernels"]["k_fitness_packed"] = roofline_entry(
+                "k_fitness_packed", packed_bytes, packed_ms, peak, peak_kind, None, None,
+                candidate_evals_per_s=N / (packed_ms * 1e-3),
+                how="ones_evaluate_packed on the same population stored as one byte per gene (a variant beside the "
+                    "int32 contract); 20 launches back to back, two packed copies read in turn")
+    if others is not None:
+        line["workloads"] = others
     if base is not None:
         line["cpu_baseline"] = base
     print(json.dumps(line))
