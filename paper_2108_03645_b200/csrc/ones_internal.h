@@ -57,7 +57,8 @@ cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t 
                              cudaStream_t s);
 cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, Tables t, int32_t capacity,
                                   double penalty, double* F, int32_t* G, cudaStream_t s);
-// tournaments + top-e in one launch; *done must be 0 at launch (the kernel leaves it 0)
+// tournaments + top-e in one launch; *done must be 0 at launch (the kernel leaves it 0); done[1] is cleared for
+// the work-item counter of launch_evolve_score
 cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,
                                 uint64_t gen, int32_t* parents, int32_t e, int32_t* elites, void* scratch,
                                 unsigned int* done, cudaStream_t s);
@@ -67,12 +68,13 @@ cudaError_t launch_top(const double* F, int32_t n, int32_t e, int32_t* idx_out, 
 cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                           int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                           Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s);
-// crossover + mutation + scoring of the children in one pass; needs evolve_score_smem(t) <= kMaxSmemPerBlock
+// crossover + mutation + scoring of the children in one pass; needs evolve_score_smem(t) <= kMaxSmemPerBlock;
+// *work: counter that is zero at launch (launch_select_stage clears done[1])
 size_t evolve_score_smem(Tables t);
 cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                                 int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                                 Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                double penalty, double* F, int32_t* G, cudaStream_t s);
+                                double penalty, double* F, int32_t* G, unsigned int* work, cudaStream_t s);
 // One launch per generation (tournaments + crossover + mutation + scoring + the next generation's elites).
 struct GenerationShape {
     int blocks, threads;  // blocks == 0: not applicable, use the multi-launch sequence

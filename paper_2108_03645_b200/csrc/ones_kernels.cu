@@ -828,6 +828,7 @@ k_select_stage(const double* __restrict__ F, int32_t n, int32_t tournament, int3
                int32_t top_blocks, int32_t per_block, Rec* __restrict__ partial, int32_t* __restrict__ elites,
                unsigned int* __restrict__ done) {
     grid_dependency_wait();  // the scores come from the kernel before
+    if (blockIdx.x == 0 && threadIdx.x == 0) done[1] = 0u;  // work-item counter of the evolve kernel that follows
     if ((int32_t)blockIdx.x >= top_blocks) {
         const int32_t i = ((int32_t)blockIdx.x - top_blocks) * blockDim.x + threadIdx.x;
         if (i < 2 * pairs) tournament_thread(F, n, tournament, i, keys, gen_lo, (i & 1) ? c3b : c3a, parents);
@@ -986,6 +987,9 @@ k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld,
     }
 }
 
+#ifndef ONES_EV_UNROLL
+#define ONES_EV_UNROLL 2
+#endif
 cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                           int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                           Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, cudaStream_t s) {
@@ -996,10 +1000,10 @@ cudaError_t launch_evolve(const int32_t* src, int32_t* dst, int64_t ld, int32_t 
     if (blocks > 0x7FFFFFFF) blocks = 0x7FFFFFFF;
     const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
     if (thr16 >= 65536u)
-        k_evolve<2, true><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+        k_evolve<ONES_EV_UNROLL, true><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
                                                       (uint32_t)gen, counter3(STREAM_MUT, gen), thr32);
     else
-        k_evolve<2, false><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
+        k_evolve<ONES_EV_UNROLL, false><<<(int)blocks, 256, 0, s>>>(src, dst, ld, n, n_jobs, elitism, pairs, parents, elites, t, keys,
                                                        (uint32_t)gen, counter3(STREAM_MUT, gen), thr32);
     return cudaGetLastError();
 }
@@ -1025,34 +1029,112 @@ __device__ __forceinline__ void score4(const int4 g, int32_t base, uint32_t kcap
     sum = __dadd_rn(sum, sX[i3]); gpus += sG[i3];
 }
 
+// What the pass is built around (each point measured at 2048 jobs x 65536 candidates):
+//   - the 16-bit g planes are stored so that, for each of the four genes of a lane, the 32 lanes of a warp
+//     read 32 different 4-byte bank words whatever their exponents: genes 0/1 and 2/3 of a lane share a word
+//     (entry position within a plane: block * 128 + (sub >> 1) * 64 + lane * 2 + (sub & 1));
+//   - work items (pairs of children, then survivors) are handed out through a counter in global memory after
+//     the first round, so a warp whose parents came from DRAM does not hold the others up (a static
+//     round-robin costs the same crossover pass 8 %);
+//   - the next int4 of both parents (after a pair's last block: the first of the next pair's parents) is in
+//     flight while the current one is worked on, the next pair's parent indices are fetched an item ahead, and
+//     every fourth block the following four blocks of both parent rows are asked into L2 (asking further ahead
+//     only adds DRAM reads: the lines are gone again before they are used);
+//   - a child's mutated value is computed without a branch and selected.
+// FULL: the row length is a multiple of 128 genes, so no lane ever falls outside a row.
+#ifndef ONES_ES_THREADS
+#define ONES_ES_THREADS 768  // threads per CTA when there are more items than warps
+#endif
+#ifndef ONES_ES_L2PF
+#define ONES_ES_L2PF 2  // blocks of 128 genes asked into L2 at a time, that far ahead of the loads (0: off)
+#endif
+
+__device__ __forceinline__ void l2_prefetch(const unsigned char* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+__device__ __forceinline__ int32_t g16_pos(int32_t slot) {  // position of table slot `slot` inside a 16-bit g plane
+    return (slot & ~127) + ((slot >> 6) & 1) * 64 + (slot & 31) * 2 + ((slot >> 5) & 1);
+}
+
+// c = mutate ? kmin + hi32(frac * range) : c, with mutate = key < thr32 (or always)
+template <bool ALWAYS>
+__device__ __forceinline__ void mutate_gene(int32_t& c, uint32_t key, uint32_t thr32, uint32_t frac, int32_t range,
+                                            int32_t kmin) {
+    const int32_t m = kmin + (int32_t)__umulhi(frac, (uint32_t)range);
+    c = (ALWAYS || key < thr32) ? m : c;
+}
+
+template <bool ALWAYS>
+__device__ __forceinline__ void sibling_pair(uint32_t W, int32_t a, int32_t b, int32_t kmin, int32_t range,
+                                             uint32_t thr32, int32_t& c0, int32_t& c1) {
+    const bool flip = (W & 1u) != 0u;
+    const uint32_t R = __funnelshift_l(W, W, 16);  // halves swapped: even child's field on top
+    c0 = flip ? b : a;
+    c1 = flip ? a : b;
+    mutate_gene<ALWAYS>(c0, R, thr32, W * 0x9E360001u, range, kmin);
+    mutate_gene<ALWAYS>(c1, W, thr32, R * 0x85EB0001u, range, kmin);
+}
+
+// One gene's table look-ups: xrow/grow point at the lane's entries of this gene in plane 0, strideX/strideG
+// are the plane strides in bytes.
+__device__ __forceinline__ void score_gene(int32_t k, uint32_t kcap, uint32_t strideX, uint32_t strideG,
+                                           const unsigned char* __restrict__ xrow, const unsigned char* __restrict__ grow,
+                                           double& sum, int32_t& gpus) {
+    const uint32_t p = min((uint32_t)k, kcap);
+    sum = __dadd_rn(sum, *reinterpret_cast<const double*>(xrow + p * strideX));
+    gpus += *reinterpret_cast<const uint16_t*>(grow + p * strideG);
+}
+
+__device__ __forceinline__ void score_int4(const int4 g, uint32_t kcap, uint32_t strideX, uint32_t strideG,
+                                           const unsigned char* __restrict__ xrow, const unsigned char* __restrict__ grow,
+                                           double& sum, int32_t& gpus) {
+    score_gene(g.x, kcap, strideX, strideG, xrow, grow, sum, gpus);
+    score_gene(g.y, kcap, strideX, strideG, xrow + 256, grow + 2, sum, gpus);
+    score_gene(g.z, kcap, strideX, strideG, xrow + 512, grow + 128, sum, gpus);
+    score_gene(g.w, kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
+}
+
+__device__ __forceinline__ int4 ld_row(const unsigned char* p) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
 // Shared memory: X planes (fp64), g planes narrowed to 16 bits (the host checks that every GPU count
-// fits), kmin and range per job (int32).
-template <int THREADS, int UNROLL, bool ALWAYS>
+// fits), kmin and range per job (int32).  `work` is the item counter: zero at launch (the selection stage
+// clears it), it ends above the number of items.
+template <int THREADS, bool ALWAYS, bool FULL>
 __global__ void __launch_bounds__(THREADS, 1)
 k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
                int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents,
                const int32_t* __restrict__ elites, Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3,
-               uint32_t thr32, int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G) {
+               uint32_t thr32, int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G,
+               unsigned int* __restrict__ work) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int32_t planes = t.k1 + 1;
     const int32_t jpad = t.jpad;
-    double* sX = reinterpret_cast<double*>(smem_raw);
-    uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + (size_t)planes * jpad * 8);
-    int4* sKmin = reinterpret_cast<int4*>(smem_raw + (size_t)planes * jpad * 10);
-    int4* sRange = sKmin + jpad / 4;
+    unsigned char* sX = smem_raw;
+    unsigned char* sG = smem_raw + (size_t)planes * jpad * 8;
+    const int4* sKmin = reinterpret_cast<const int4*>(smem_raw + (size_t)planes * jpad * 10);
+    const int4* sRange = sKmin + jpad / 4;
     {
         const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
         const int4* gX = reinterpret_cast<const int4*>(t.X);
         const int4* gG = reinterpret_cast<const int4*>(t.G);
         for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
         for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
-            const int4 g = gG[i];
-            reinterpret_cast<uint2*>(sG)[i] = make_uint2((uint32_t)g.x | ((uint32_t)g.y << 16),
-                                                         (uint32_t)g.z | ((uint32_t)g.w << 16));
+            const int4 g = gG[i];  // slots 4i..4i+3 of one plane: same block and gene, four neighbouring lanes
+            const int32_t plane = (4 * i) / jpad, slot = (4 * i) % jpad;
+            uint16_t* to = reinterpret_cast<uint16_t*>(sG) + plane * jpad + g16_pos(slot);
+            to[0] = (uint16_t)g.x;
+            to[2] = (uint16_t)g.y;
+            to[4] = (uint16_t)g.z;
+            to[6] = (uint16_t)g.w;
         }
         for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
-            sKmin[i] = reinterpret_cast<const int4*>(t.kmin)[i];
-            sRange[i] = reinterpret_cast<const int4*>(t.range)[i];
+            const_cast<int4*>(sKmin)[i] = reinterpret_cast<const int4*>(t.kmin)[i];
+            const_cast<int4*>(sRange)[i] = reinterpret_cast<const int4*>(t.range)[i];
         }
         __syncthreads();
     }
@@ -1061,66 +1143,115 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
     // kernel measured 3 % slower at the largest population.
     grid_dependency_wait();
     const int lane = threadIdx.x & 31;
-    const int32_t warps_per_block = blockDim.x >> 5;
-    const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
+    const int32_t warps_per_block = THREADS >> 5;
+    const int32_t total_warps = (int32_t)gridDim.x * warps_per_block;
     const int32_t nvec = (int32_t)(ld >> 2);
+    const int32_t nblk = (nvec + 31) >> 5;
     const uint32_t kcap = (uint32_t)t.k1;
+    const uint32_t strideX = (uint32_t)jpad * 8u, strideG = (uint32_t)jpad * 2u;
+    const int64_t row_bytes = ld * 4;
+    const unsigned char* srcb = reinterpret_cast<const unsigned char*>(src) + lane * 16;
+    unsigned char* dstb = reinterpret_cast<unsigned char*>(dst) + lane * 16;
+    const unsigned char* xlane = sX + lane * 8;
+    const unsigned char* glane = sG + lane * 4;
+    const int2* pp = reinterpret_cast<const int2*>(parents);
+    const bool row_lane = FULL || lane < nvec;  // a lane past a short row's end never loads in block 0
 
-    for (int64_t w = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); w < (int64_t)pairs + elitism;
-         w += total_warps) {
+    // Items [0, pairs) are pairs of children, [pairs, pairs + elitism) survivors.  A warp's first item is its own
+    // number; when there are more items than warps, every later one comes from the counter: lane 0 asks for a
+    // ticket an item ahead and the warp reads it (one shuffle) half-way through the item it is working on, in
+    // time to fetch the next pair's parent indices before that pair's first loads.
+    const int32_t items = pairs + elitism;
+    const bool dynamic = items > total_warps;
+    unsigned int ticket = 0;
+    auto ask = [&]() {
+        if (dynamic && lane == 0) ticket = atomicAdd(work, 1u);
+    };
+    auto take = [&]() { return dynamic ? total_warps + (int32_t)__shfl_sync(0xFFFFFFFFu, ticket, 0) : items; };
+    int32_t w = (int32_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    ask();
+    int2 par = make_int2(0, 0);
+    int4 a0 = make_int4(0, 0, 0, 0), b0 = a0, a1 = a0, b1 = a0;
+    if (w < pairs) {
+        par = pp[w];
+        if (row_lane) {
+            a0 = ld_row(srcb + par.x * row_bytes);
+            b0 = ld_row(srcb + par.y * row_bytes);
+        }
+    }
+    // One step = one int4 of each parent -> one int4 of each child, scored.
+    auto step = [&](const int32_t blk, const int32_t slot0, const bool has1, unsigned char* __restrict__ C,
+                    const int4& cura, const int4& curb, double& sum0, double& sum1, int32_t& gp0, int32_t& gp1) {
+        const int32_t v = blk * 32 + lane;
+        if (FULL || v < nvec) {
+            const int4 kmin = sKmin[v];
+            const int4 range = sRange[v];
+            const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+            int4 c0, c1;
+            sibling_pair<ALWAYS>(W.x, cura.x, curb.x, kmin.x, range.x, thr32, c0.x, c1.x);
+            sibling_pair<ALWAYS>(W.y, cura.y, curb.y, kmin.y, range.y, thr32, c0.y, c1.y);
+            sibling_pair<ALWAYS>(W.z, cura.z, curb.z, kmin.z, range.z, thr32, c0.z, c1.z);
+            sibling_pair<ALWAYS>(W.w, cura.w, curb.w, kmin.w, range.w, thr32, c0.w, c1.w);
+            unsigned char* to = C + blk * 512;
+            *reinterpret_cast<int4*>(to) = c0;
+            if (has1) *reinterpret_cast<int4*>(to + row_bytes) = c1;
+            const unsigned char* xrow = xlane + blk * 1024;
+            const unsigned char* grow = glane + blk * 256;
+            score_int4(c0, kcap, strideX, strideG, xrow, grow, sum0, gp0);
+            score_int4(c1, kcap, strideX, strideG, xrow, grow, sum1, gp1);
+        }
+    };
+    const int32_t take_at = (nblk / 2) & ~1;  // the block (even) at which the next item's number is read
+    while (w < pairs) {
+        const unsigned char* A = srcb + par.x * row_bytes;
+        const unsigned char* B = srcb + par.y * row_bytes;
+        const int32_t slot0 = elitism + 2 * w;
+        const bool has1 = slot0 + 1 < n;
+        unsigned char* C = dstb + slot0 * row_bytes;
+        int32_t w_next = items;
+        bool more = false;
         double sum0 = 0.0, sum1 = 0.0;
         int32_t gp0 = 0, gp1 = 0;
-        int32_t slot0, slot1;
-        bool has1;
-        if (w >= pairs) {  // survivor: copy unchanged and score again
-            slot0 = (int32_t)(w - pairs);
-            slot1 = slot0;
-            has1 = false;
-            const int4* from = reinterpret_cast<const int4*>(src + (int64_t)elites[slot0] * ld);
-            int4* to = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
-            for (int32_t v = lane; v < nvec; v += 32) {
-                const int4 g = from[v];
-                to[v] = g;
-                score4(g, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
-            }
-        } else {
-            const int32_t q = (int32_t)w;
-            const int32_t pa = parents[2 * q], pb = parents[2 * q + 1];
-            slot0 = elitism + 2 * q;
-            slot1 = slot0 + 1;
-            has1 = slot1 < n;
-            const int4* A = reinterpret_cast<const int4*>(src + (int64_t)pa * ld);
-            const int4* B = reinterpret_cast<const int4*>(src + (int64_t)pb * ld);
-            int4* C0 = reinterpret_cast<int4*>(dst + (int64_t)slot0 * ld);
-            int4* C1 = reinterpret_cast<int4*>(dst + (int64_t)slot1 * ld);
-            for (int32_t v0 = 0; v0 < nvec; v0 += 32 * UNROLL) {
-                int4 a[UNROLL], b[UNROLL];
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int32_t v = v0 + u * 32 + lane;
-                    if (v < nvec) {
-                        a[u] = A[v];
-                        b[u] = B[v];
-                    }
+        // Fetch block `nb` of this pair's parents, or (after the last block) block 0 of the next pair's.
+        auto fetch = [&](const int32_t nb, int4& na, int4& nb4) {
+            na = make_int4(0, 0, 0, 0);
+            nb4 = na;
+            if (nb < nblk) {
+                if (FULL || nb * 32 + lane < nvec) {
+                    na = ld_row(A + nb * 512);
+                    nb4 = ld_row(B + nb * 512);
                 }
+#if ONES_ES_L2PF > 0
+                if ((nb % ONES_ES_L2PF) == 0 && nb + ONES_ES_L2PF < nblk) {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int32_t v = v0 + u * 32 + lane;
-                    if (v < nvec) {
-                        const int4 kmin = sKmin[v];
-                        const int4 range = sRange[v];
-                        const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
-                        int4 c0, c1;
-                        sibling_int4<ALWAYS>(W, a[u], b[u], kmin, range, thr32, has1, c0, c1);
-                        C0[v] = c0;
-                        const int32_t base = (v >> 5) * 128 + lane;
-                        score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
-                        if (has1) {
-                            C1[v] = c1;
-                            score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
+                    for (int d = 0; d < ONES_ES_L2PF; ++d) {
+                        if (nb + ONES_ES_L2PF + d < nblk) {
+                            l2_prefetch(A + (nb + ONES_ES_L2PF + d) * 512);
+                            l2_prefetch(B + (nb + ONES_ES_L2PF + d) * 512);
                         }
                     }
                 }
+#endif
+            } else if (more && row_lane) {
+                na = ld_row(srcb + par.x * row_bytes);
+                nb4 = ld_row(srcb + par.y * row_bytes);
+            }
+        };
+        for (int32_t blk = 0; blk < nblk; blk += 2) {
+            if (blk == take_at) {
+                w_next = take();
+                ask();
+                more = w_next < pairs;
+                if (more) par = pp[w_next];  // A and B keep this pair's rows
+            }
+            fetch(blk + 1, a1, b1);
+            step(blk, slot0, has1, C, a0, b0, sum0, sum1, gp0, gp1);
+            if (blk + 1 < nblk) {
+                fetch(blk + 2, a0, b0);
+                step(blk + 1, slot0, has1, C, a1, b1, sum0, sum1, gp0, gp1);
+            } else {  // odd number of blocks: the next pair's first block sits in the other buffer
+                a0 = a1;
+                b0 = b1;
             }
         }
 #pragma unroll
@@ -1136,10 +1267,39 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             G[slot0] = gp0;
             if (has1) {
                 const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
-                F[slot1] = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
-                G[slot1] = gp1;
+                F[slot0 + 1] = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                G[slot0 + 1] = gp1;
             }
         }
+        w = w_next;
+    }
+    // ---- survivors: copied unchanged and scored again ----
+    while (w < items) {
+        const int32_t w_next = take();
+        ask();
+        const int32_t r = w - pairs;
+        const unsigned char* from = srcb + elites[r] * row_bytes;
+        unsigned char* to = dstb + r * row_bytes;
+        double sum = 0.0;
+        int32_t gp = 0;
+        for (int32_t blk = 0; blk < nblk; ++blk) {
+            if (FULL || blk * 32 + lane < nvec) {
+                const int4 g = *reinterpret_cast<const int4*>(from + blk * 512);
+                *reinterpret_cast<int4*>(to + blk * 512) = g;
+                score_int4(g, kcap, strideX, strideG, xlane + blk * 1024, glane + blk * 256, sum, gp);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            gp += __shfl_xor_sync(0xFFFFFFFFu, gp, off);
+        }
+        if (lane == 0) {
+            const int32_t over = gp > capacity ? gp - capacity : 0;
+            F[r] = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            G[r] = gp;
+        }
+        w = w_next;
     }
 }
 
@@ -1551,20 +1711,32 @@ size_t evolve_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (
 cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                                 int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                                 Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                double penalty, double* F, int32_t* G, cudaStream_t s) {
+                                double penalty, double* F, int32_t* G, unsigned int* work, cudaStream_t s) {
     const int64_t warps = (int64_t)pairs + elitism;
     if (warps <= 0) return cudaSuccess;
     const size_t smem = evolve_score_smem(t);
     if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
-    constexpr int kThreads = 1024;  // one CTA per SM; measured best with one int4 per parent in flight per lane
-    int64_t blocks = (warps + kThreads / 32 - 1) / (kThreads / 32);
-    if (blocks > kSMs) blocks = kSMs;
     const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
-    auto kern = thr16 >= 65536u ? k_evolve_score<kThreads, 1, true> : k_evolve_score<kThreads, 1, false>;
+    const bool always = thr16 >= 65536u, full = (ld & 127) == 0;
+    // One persistent CTA per SM.  32 warps when that gives every item a warp of its own; otherwise 24 warps with
+    // 80 registers each (measured 3 % faster than 32 x 64 at 2048 jobs x 65536 candidates).
+    const bool wide = warps <= (int64_t)kSMs * 32;
+    const int threads = wide ? 1024 : ONES_ES_THREADS;
+    int64_t blocks = (warps + threads / 32 - 1) / (threads / 32);
+    if (blocks > kSMs) blocks = kSMs;
+    void (*kern)(const int32_t*, int32_t*, int64_t, int32_t, int32_t, int32_t, int32_t, const int32_t*, const int32_t*,
+                 Tables, RoundKeys, uint32_t, uint32_t, uint32_t, int32_t, double, double*, int32_t*, unsigned int*);
+    if (wide)
+        kern = always ? (full ? k_evolve_score<1024, true, true> : k_evolve_score<1024, true, false>)
+                      : (full ? k_evolve_score<1024, false, true> : k_evolve_score<1024, false, false>);
+    else
+        kern = always ? (full ? k_evolve_score<ONES_ES_THREADS, true, true> : k_evolve_score<ONES_ES_THREADS, true, false>)
+                      : (full ? k_evolve_score<ONES_ES_THREADS, false, true> : k_evolve_score<ONES_ES_THREADS, false, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
-    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, src, dst, ld, n, n_jobs, elitism, pairs, parents,
-                                 elites, t, keys, (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G);
+    return launch_after_previous(kern, (int)blocks, threads, smem, s, src, dst, ld, n, n_jobs, elitism, pairs, parents,
+                                 elites, t, keys, (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G,
+                                 work);
 }
 
 // ---------------------------------------------------------------------------------------------
