@@ -54,7 +54,11 @@ typedef struct {
 /* Search parameters.  elitism: candidates that survive unchanged per generation;
  * tournament: draws per parent; p_mut: mutation rate theta per gene ("Uniform
  * mutation"); penalty: score lost per GPU above the cluster's capacity (Eq. 4 as a
- * soft constraint).  NULL where a ones_params* is expected means {2, 4, 0.1, 1e3, 0}. */
+ * soft constraint).  NULL where a ones_params* is expected means {2, 4, 0.1, 1e3, 0}.
+ * p_mut is applied with a resolution of 1/65536: a gene mutates when a uniform 16-bit field is below
+ * lround(p_mut * 65536), so the effective rate is that threshold / 65536 (0.1 -> 6554/65536).  A positive
+ * p_mut that rounds to a threshold of 0 (below 2^-17) is rejected with ONES_ERR_BAD_PARAM rather than
+ * silently switching mutation off. */
 typedef struct {
     int32_t elitism, tournament;
     double p_mut, penalty;
@@ -253,7 +257,10 @@ int ones_select_top(const double* d_fitness, int32_t n, int32_t e, int32_t* d_in
  *   d_fitness, d_index  device, as for ones_select_top.   1 <= e <= min(n, ONES_NOALLOC_MAX_TOP);
  *   a larger e returns ONES_ERR_WORKSPACE (use ones_select_top with your own scratch).
  * The first call on each device looks up the array's device address (that device must be
- * current); make that first call before any stream capture begins.  All calls on a device share
+ * current); make that first call before any stream capture begins.  The address is kept for the
+ * life of the process: after cudaDeviceReset (or any other teardown of the device's primary
+ * context) it no longer points at the array, so do not call this entry point again in a process
+ * that reset the device.  All calls on a device share
  * the one array, which keeps whatever the last call left in it: no part of it needs clearing
  * (each call overwrites every record it later reads), but two calls whose kernels may overlap on
  * the GPU — different streams, or different threads — race on it; serialise them.

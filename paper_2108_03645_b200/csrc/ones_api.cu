@@ -182,6 +182,7 @@ int check_params(const ones_params& p, int32_t pop) {
     if (p.elitism < 0 || p.elitism > ONES_MAX_ELITES || p.tournament < 1) return ONES_ERR_BAD_PARAM;
     if (pop < p.elitism + 1) return ONES_ERR_BAD_PARAM;
     if (!(p.p_mut >= 0.0 && p.p_mut <= 1.0)) return ONES_ERR_BAD_PARAM;
+    if (p.p_mut > 0.0 && lround(p.p_mut * 65536.0) == 0) return ONES_ERR_BAD_PARAM;  // below the 16-bit resolution
     if (!isfinite(p.penalty)) return ONES_ERR_BAD_PARAM;
     return ONES_OK;
 }

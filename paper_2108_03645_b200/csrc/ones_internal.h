@@ -7,7 +7,9 @@
 
 namespace ones {
 
-constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
+constexpr int kSMsDefault = 148;          // B200: 2 dies x 74 SMs (used only when the device cannot be asked)
+constexpr int kSMsMax = 192;              // bound on the SM count that per-SM scratch lists are sized for
+int sm_count();                           // SMs of the current device, at most kSMsMax
 constexpr int kMaxSmemPerBlock = 232448;  // 227 KiB opt-in dynamic shared memory per CTA
 constexpr int kTopBlocksMax = 128;        // partial top-k blocks
 

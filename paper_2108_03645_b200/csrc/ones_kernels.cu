@@ -16,6 +16,20 @@
 
 namespace ones {
 
+// SMs of the current device (read once per device): persistent grids are sized from it.
+int sm_count() {
+    constexpr int kDevices = 64;
+    static int cached[kDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDevices) return kSMsDefault;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return kSMsDefault;
+        cached[dev] = n < kSMsMax ? n : kSMsMax;
+    }
+    return cached[dev];
+}
+
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11).  Round keys are precomputed on the host.
 // ---------------------------------------------------------------------------------------------
@@ -170,7 +184,7 @@ __global__ void k_fill_min(int32_t* __restrict__ pop, int64_t ld, int32_t n, int
 cudaError_t launch_fill_min(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t, cudaStream_t s) {
     const int64_t total = (int64_t)n * ld;
     const int64_t grid = (total + 255) / 256;
-    k_fill_min<<<(int)(grid < kSMs * 8 ? grid : kSMs * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t);
+    k_fill_min<<<(int)(grid < sm_count() * 8 ? grid : sm_count() * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t);
     return cudaGetLastError();
 }
 
@@ -200,7 +214,7 @@ cudaError_t launch_randomize(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs
                              RoundKeys keys, cudaStream_t s) {
     const int64_t total = (int64_t)n * (ld >> 2);
     const int64_t grid = (total + 255) / 256;
-    k_randomize<<<(int)(grid < kSMs * 8 ? grid : kSMs * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t, keys);
+    k_randomize<<<(int)(grid < sm_count() * 8 ? grid : sm_count() * 8), 256, 0, s>>>(pop, ld, n, n_jobs, t, keys);
     return cudaGetLastError();
 }
 
@@ -221,7 +235,7 @@ cudaError_t launch_copy_rows(const int32_t* src, int64_t ld_src, int32_t* dst, i
     const int64_t total = (int64_t)n * (zero_pad ? ld_dst : n_jobs);
     const int64_t grid = (total + 255) / 256;
     if (grid == 0) return cudaSuccess;
-    k_copy_rows<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs,
+    k_copy_rows<<<(int)(grid < sm_count() * 16 ? grid : sm_count() * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs,
                                                                           zero_pad);
     return cudaGetLastError();
 }
@@ -250,7 +264,7 @@ cudaError_t launch_remap(const int32_t* src, int64_t ld_src, int32_t* dst, int64
                          const int32_t* range_new, cudaStream_t s) {
     const int64_t total = (int64_t)n * ld_dst;
     const int64_t grid = (total + 255) / 256;
-    k_remap<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs_new,
+    k_remap<<<(int)(grid < sm_count() * 16 ? grid : sm_count() * 16), 256, 0, s>>>(src, ld_src, dst, ld_dst, n, n_jobs_new,
                                                                       remap, kmin_new, range_new);
     return cudaGetLastError();
 }
@@ -341,7 +355,7 @@ cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_
                            int32_t capacity, double penalty, double* F, int32_t* G, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     const size_t lut_bytes = (size_t)(t.k1 + 1) * t.jpad * 12;
-    const bool big = n >= kSMs * 32;
+    const bool big = n >= sm_count() * 32;
     const int threads = big ? 1024 : 256;
     const int wpb = threads / 32;
     int64_t blocks = ((int64_t)n + wpb - 1) / wpb;
@@ -350,14 +364,14 @@ cudaError_t launch_fitness(const int32_t* genomes, int64_t ld, int32_t n, int32_
         if (per_sm < 1) per_sm = 1;
         const int by_threads = 2048 / threads;
         if (per_sm > by_threads) per_sm = by_threads;
-        if (blocks > (int64_t)kSMs * per_sm) blocks = (int64_t)kSMs * per_sm;
+        if (blocks > (int64_t)sm_count() * per_sm) blocks = (int64_t)sm_count() * per_sm;
         cudaError_t e = cudaFuncSetAttribute(k_fitness<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kMaxSmemPerBlock);
         if (e != cudaSuccess) return e;
         k_fitness<true, 4><<<(int)blocks, threads, lut_bytes, s>>>(genomes, ld, n, n_jobs, t, capacity, penalty, F, G);
     } else {
         // tables too large for shared memory: read them through L1/L2
-        if (blocks > (int64_t)kSMs * (2048 / threads)) blocks = (int64_t)kSMs * (2048 / threads);
+        if (blocks > (int64_t)sm_count() * (2048 / threads)) blocks = (int64_t)sm_count() * (2048 / threads);
         k_fitness<false, 4><<<(int)blocks, threads, 0, s>>>(genomes, ld, n, n_jobs, t, capacity, penalty, F, G);
     }
     return cudaGetLastError();
@@ -404,7 +418,7 @@ cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t 
     if (n <= 0) return cudaSuccess;
     const int64_t total = (int64_t)n * (ld8 >> 4);
     const int64_t grid = (total + 255) / 256;
-    k_pack_rows<<<(int)(grid < kSMs * 16 ? grid : kSMs * 16), 256, 0, s>>>(src, ld, n, n_jobs, dst, ld8);
+    k_pack_rows<<<(int)(grid < sm_count() * 16 ? grid : sm_count() * 16), 256, 0, s>>>(src, ld, n, n_jobs, dst, ld8);
     return cudaGetLastError();
 }
 
@@ -484,7 +498,7 @@ cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, T
                                   double penalty, double* F, int32_t* G, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     const size_t lut_bytes = (size_t)(t.k1 + 1) * t.jpad * 12;
-    const bool big = n >= kSMs * 32;
+    const bool big = n >= sm_count() * 32;
     const int threads = big ? 1024 : 256;
     const int wpb = threads / 32;
     int64_t blocks = ((int64_t)n + wpb - 1) / wpb;
@@ -493,13 +507,13 @@ cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, T
         if (per_sm < 1) per_sm = 1;
         const int by_threads = 2048 / threads;
         if (per_sm > by_threads) per_sm = by_threads;
-        if (blocks > (int64_t)kSMs * per_sm) blocks = (int64_t)kSMs * per_sm;
+        if (blocks > (int64_t)sm_count() * per_sm) blocks = (int64_t)sm_count() * per_sm;
         cudaError_t e = cudaFuncSetAttribute(k_fitness_packed<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kMaxSmemPerBlock);
         if (e != cudaSuccess) return e;
         k_fitness_packed<true, 4><<<(int)blocks, threads, lut_bytes, s>>>(rows, ld8, n, t, capacity, penalty, F, G);
     } else {
-        if (blocks > (int64_t)kSMs * (2048 / threads)) blocks = (int64_t)kSMs * (2048 / threads);
+        if (blocks > (int64_t)sm_count() * (2048 / threads)) blocks = (int64_t)sm_count() * (2048 / threads);
         k_fitness_packed<false, 4><<<(int)blocks, threads, 0, s>>>(rows, ld8, n, t, capacity, penalty, F, G);
     }
     return cudaGetLastError();
@@ -1422,7 +1436,7 @@ cudaError_t launch_remap_score(const int32_t* src, int64_t ld_src, int32_t* dst,
     cudaError_t e = cudaFuncSetAttribute(k_remap_score, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
     int64_t blocks = ((int64_t)n + 31) / 32;
-    if (blocks > kSMs) blocks = kSMs;
+    if (blocks > sm_count()) blocks = sm_count();
     k_remap_score<<<(int)blocks, 1024, smem, s>>>(src, ld_src, dst, ld_dst, n, n_jobs_new, remap, t, capacity, penalty, F, G);
     return cudaGetLastError();
 }
@@ -1661,7 +1675,7 @@ k_generation(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t
     if (threadIdx.x == 0) *done = 0u;
 }
 
-size_t generation_scratch_bytes(int32_t e) { return (size_t)kSMs * (size_t)e * sizeof(Rec); }
+size_t generation_scratch_bytes(int32_t e) { return (size_t)kSMsMax * (size_t)e * sizeof(Rec); }
 
 // Launch shape of k_generation for this problem, or blocks = 0 when it does not apply (tables or the
 // score queue do not fit shared memory, or the merge scratch would overflow).
@@ -1672,11 +1686,11 @@ GenerationShape generation_shape(Tables t, int32_t pairs, int32_t elitism) {
     // Large populations are HBM-bound and measured faster as two launches (k_select_stage, then
     // k_evolve_score with the parents known up front); the single launch pays off when the generation is
     // launch-latency-bound.
-    if (warps >= (int64_t)kSMs * 16) return g;
+    if (warps >= (int64_t)sm_count() * 16) return g;
     g.threads = 256;
     const int wpb = g.threads / 32;
     int64_t blocks = (warps + wpb - 1) / wpb;
-    if (blocks > kSMs) blocks = kSMs;  // the merge scratch holds kSMs lists (generation_scratch_bytes)
+    if (blocks > sm_count()) blocks = sm_count();  // the merge scratch holds up to kSMsMax lists (generation_scratch_bytes)
     const int64_t total_warps = blocks * wpb;
     const int64_t per_warp = (warps + total_warps - 1) / total_warps;
     g.queue_cap = (int32_t)(2 * per_warp * wpb);
@@ -1720,10 +1734,10 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
     const bool always = thr16 >= 65536u, full = (ld & 127) == 0;
     // One persistent CTA per SM.  32 warps when that gives every item a warp of its own; otherwise 24 warps with
     // 80 registers each (measured 3 % faster than 32 x 64 at 2048 jobs x 65536 candidates).
-    const bool wide = warps <= (int64_t)kSMs * 32;
+    const bool wide = warps <= (int64_t)sm_count() * 32;
     const int threads = wide ? 1024 : ONES_ES_THREADS;
     int64_t blocks = (warps + threads / 32 - 1) / (threads / 32);
-    if (blocks > kSMs) blocks = kSMs;
+    if (blocks > sm_count()) blocks = sm_count();
     void (*kern)(const int32_t*, int32_t*, int64_t, int32_t, int32_t, int32_t, int32_t, const int32_t*, const int32_t*,
                  Tables, RoundKeys, uint32_t, uint32_t, uint32_t, int32_t, double, double*, int32_t*, unsigned int*);
     if (wide)
@@ -1993,7 +2007,7 @@ static cudaError_t cluster_config(ClusterShape shape, cudaStream_t s, cudaLaunch
 // large enough for the HBM paths).  rows_per_cta >= 32 keeps every CTA busy.
 ClusterShape cluster_shape(Tables t, int64_t ld, int32_t n, int32_t elitism, int32_t pairs) {
     ClusterShape shape{0, 0, 0, 0, 0};
-    if ((int64_t)pairs + elitism >= (int64_t)kSMs * 16) return shape;
+    if ((int64_t)pairs + elitism >= (int64_t)sm_count() * 16) return shape;
     const int32_t nvec = (int32_t)(ld >> 2);
     int gs = 1;
     while (gs < nvec && gs < 32) gs <<= 1;
@@ -2433,7 +2447,7 @@ cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, in
     if (e != cudaSuccess) return e;
     constexpr int kThreads = 1024;
     int64_t blocks = (2 * (int64_t)k + kThreads / 32 - 1) / (kThreads / 32);
-    if (blocks > kSMs) blocks = kSMs;
+    if (blocks > sm_count()) blocks = sm_count();
     auto kern = thr16 >= 65536u ? k_trunc_children_score<true> : k_trunc_children_score<false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
@@ -2455,7 +2469,7 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
     int32_t* kept = bsum + 2 * 1024;
     cudaError_t e;
     int rb = (n + 2047) / 2048;
-    if (rb > kSMs) rb = kSMs;
+    if (rb > sm_count()) rb = sm_count();
     for (int pass = 0; pass < 8; ++pass) {
         e = launch_after_previous(k_trunc_radix_pass, rb, 256, 0, s, F, n, k, pass, state, pick);
         if (e != cudaSuccess) return e;
@@ -2863,7 +2877,7 @@ static cudaError_t launch_per_gpu_regs_t(int32_t* slots, int64_t ld, int32_t n, 
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int64_t blocks = n;
-    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
     k_per_gpu_regs<PIECE, REORDER, SCORE, RUNS, NARROW><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit,
                                                                                         F, G);
     return cudaGetLastError();
@@ -2899,7 +2913,7 @@ static cudaError_t launch_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_t
     cudaError_t e = cudaFuncSetAttribute(k_per_gpu<REORDER, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int64_t blocks = n;
-    if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+    if (blocks > (int64_t)sm_count() * 8) blocks = (int64_t)sm_count() * 8;
     k_per_gpu<REORDER, SCORE><<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_jobs, t, fit, F, G);
     return cudaGetLastError();
 }
@@ -3393,7 +3407,7 @@ cudaError_t launch_refresh_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_
     e = cudaFuncSetAttribute(k_refresh_per_gpu, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int64_t blocks = n;
-    if (blocks > (int64_t)kSMs * 4) blocks = (int64_t)kSMs * 4;
+    if (blocks > (int64_t)sm_count() * 4) blocks = (int64_t)sm_count() * 4;
     k_refresh_per_gpu<<<(int)blocks, 256, smem, s>>>(slots, ld, n, n_gpus, n_old, n_jobs, t, fit, remap, inv, newcum,
                                                       refresh_sort_len(n_jobs));
     return cudaGetLastError();

@@ -654,7 +654,8 @@ def test_errors_are_codes_not_faults(ones):
     with pytest.raises(ones.OnesError) as err:
         ones.Search(bad, 16, 32)
     assert err.value.code == -2
-    for kw, code in ((dict(elitism=40), -3), (dict(tournament=0), -3), (dict(p_mut=-0.1), -3)):
+    for kw, code in ((dict(elitism=40), -3), (dict(tournament=0), -3), (dict(p_mut=-0.1), -3),
+                     (dict(p_mut=2.0 ** -18), -3)):   # a rate below the 16-bit resolution would switch mutation off
         with pytest.raises(ones.OnesError) as err:
             ones.Search(w.jobs, 16, 32, inputs.SearchParams(**kw))
         assert err.value.code == code

@@ -42,10 +42,9 @@ def test_philox_matches_independent_implementation():
         ctr[1] = 0xFFFFFFFF
         ctr[2] = (1, 0, 0, 0)
         ctr[3] = (0, 0, 0, 1)
-        try:
-            ref = _triton_philox(seed, ctr[:, 0], ctr[:, 1], ctr[:, 2], ctr[:, 3])
-        except Exception as exc:  # interpreter not usable in this environment
-            pytest.skip(f"triton interpreter unavailable: {exc}")
+        # no skip here: if the independent implementation cannot run, the generator is unpinned and the run
+        # must not pass as if it had been checked
+        ref = _triton_philox(seed, ctr[:, 0], ctr[:, 1], ctr[:, 2], ctr[:, 3])
         key = [seed & 0xFFFFFFFF, seed >> 32]
         for i in range(n):
             assert (oracle.philox(ctr[i], key) == ref[i]).all(), (seed, i)

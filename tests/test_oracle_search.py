@@ -345,6 +345,20 @@ def test_sibling_children_mutate_independently():
         both = int(((kids[0::2] != 0) & (kids[1::2] != 0)).sum())
         n = kids[0::2].size
         assert abs(both - n * rate * rate) < 6 * (n * rate * rate) ** 0.5 + 3
+    # p = 0.1: where both siblings redraw the same gene (both 16-bit fields of the word are below the threshold,
+    # a thin slice of the word's values) the two new values must still be jointly uniform.  Parents wait at
+    # every gene (-1), so each redraw is visible.
+    big = inputs.custom(48, 10 ** 6, 8193, 1, seed=8, kmax=5)
+    s = _search(big, p_mut=0.1, elitism=1)
+    s.set_population(np.full((big.pop, 48), -1, dtype=np.int32))
+    s.evolve(1, 23)
+    kids = s.get_population()[1:]
+    even, odd = kids[0::2].ravel(), kids[1::2].ravel()
+    hit = (even >= 0) & (odd >= 0)
+    assert abs(int(hit.sum()) - even.size * 0.01) < 6 * (even.size * 0.01) ** 0.5   # both redraw: p * p
+    joint = np.bincount(even[hit] * 6 + odd[hit], minlength=36)
+    exp = int(hit.sum()) / 36
+    assert exp > 40 and ((joint - exp) ** 2 / exp).sum() < 80  # 35 dof, p ~ 2e-5
 
 
 def test_checkpoint_and_resume():

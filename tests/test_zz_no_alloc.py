@@ -49,3 +49,22 @@ def test_noalloc_selection_rejects_sizes_beyond_its_scratch():
     with pytest.raises(binding.OnesError) as err:
         binding.select_top_noalloc(scores[:3], 4, out)
     assert err.value.code == -3
+
+
+def test_noalloc_selection_on_a_stream_of_the_callers():
+    """The entry point enqueues on the stream it is given; a caller's own stream (not the default one) must see
+    the same result, again on two calls in a row."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2108_03645_b200 import binding
+    scores = _scores(50_000, 4)
+    want = binding.select_top(scores, 7)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    out = torch.full((binding.NOALLOC_MAX_TOP,), -7, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            got = binding.select_top_noalloc(scores, 7, out)[:7]
+            stream.synchronize()
+            assert torch.equal(got, want)
