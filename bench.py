@@ -505,6 +505,25 @@ def main():
         del s2
         torch.cuda.empty_cache()
 
+    # ---- the generation on one-byte genes (ONES_FLAG_PACKED): a variant beside the int32 contract ----
+    packed_gen = None
+    if solo and not args.no_kernel_events and args.scheme == "tournament":
+        import dataclasses
+        p3 = dataclasses.replace(w.params, flags=w.params.flags | binding.FLAG_PACKED)
+        s3 = binding.Search(w.jobs, w.capacity, w.pop, p3)
+        s3.randomize(seed)
+        s3.evolve(warmup, seed)
+        rep3 = timed_repeats(lambda: s3.evolve(steps, seed), 0.5 * args.min_seconds)
+        s3.set_profiling(1)
+        s3.stage_times()
+        s3.evolve(max(steps, 50), seed)
+        ms3, n3 = s3.stage_times()
+        s3.set_profiling(False)
+        packed_gen = (statistics.median(rep3) / steps, ms3["evolve"] / n3["evolve"], ms3["select"] / n3["select"], len(rep3))
+        s3.close()
+        del s3
+        torch.cuda.empty_cache()
+
     # ---- the other workloads, measured in the same run ----
     others = None
     if solo and not args.no_workloads and args.scheme == "tournament" and not args.pop:
@@ -600,6 +619,17 @@ def main():
                 candidate_evals_per_s=N / (packed_ms * 1e-3),
                 how="ones_evaluate_packed on the same population stored as one byte per gene (a variant beside the "
                     "int32 contract); 20 launches back to back, two packed copies read in turn")
+    if packed_gen is not None and "kernels" in line:
+        gen_ms, k_ms, sel_ms3, reps3 = packed_gen
+        # one parent byte read and one child byte written per child gene, the elite rows, indices, F and G
+        pbytes = 2 * J * (N - E) + 2 * J * E + 8 * ((N - E + 1) // 2) + 4 * E + 12 * N
+        line["kernels"]["k_evolve_score_packed"] = roofline_entry(
+            "k_evolve_score_packed", pbytes, k_ms, peak, peak_kind, None, None,
+            ms_per_generation=gen_ms, generations_per_s=1e3 / gen_ms, candidate_evals_per_s=N * 1e3 / gen_ms,
+            timed_repeats=reps3,
+            how="same workload on a handle with ONES_FLAG_PACKED (population kept as one byte per gene; identical "
+                "children, scores and selections): ms_per_generation from repeats of the K steps without per-kernel "
+                "events, ms_per_launch from an event pass of its own")
     if others is not None:
         line["workloads"] = others
     if base is not None:

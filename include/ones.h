@@ -103,6 +103,19 @@ typedef struct {
  * Not combinable with ONES_FLAG_TRUNCATION.  Size the workspace with ones_workspace_bytes_per_gpu. */
 #define ONES_FLAG_PER_GPU 16u
 
+/* The handle keeps its population as packed rows (one byte per gene, the tile layout described at
+ * ones_pack_population) and ones_evolve reads parents and writes children as bytes: 2 bytes of device-memory
+ * traffic per child gene instead of 8.  Random draws, operators, summation order and therefore children, scores
+ * and selections are those of the int32 rows (Section 3.2.2 "Uniform crossover", "Uniform mutation"; Alg. 1's
+ * score step).  Everything else keeps its interface: ones_set_population / ones_get_population take and return
+ * int32 rows (converted on the way; a gene outside [0, 254] is stored as "waits" and reads back as -1),
+ * ones_best and ones_update_jobs work as before, ones_pack_population(NULL) returns the rows as they are.
+ * Needs model tables that fit the shared memory of one thread block (about 2300 jobs at kmax 7; otherwise
+ * ones_create / ones_update_jobs return ONES_ERR_BAD_PARAM).  Not combinable with ONES_FLAG_TRUNCATION or
+ * ONES_FLAG_PER_GPU; ONES_FLAG_UNFUSED and ONES_FLAG_NO_CLUSTER have no effect.  Size the workspace with
+ * ones_workspace_bytes_flags. */
+#define ONES_FLAG_PACKED 32u
+
 #define ONES_MAX_EXPONENT 15  /* kmax <= 15 */
 #define ONES_MAX_ELITES 256   /* elitism <= 256 */
 

@@ -21,6 +21,7 @@ FLAG_UNFUSED = 2
 FLAG_TRUNCATION = 4
 FLAG_NO_CLUSTER = 8
 FLAG_PER_GPU = 16
+FLAG_PACKED = 32
 MAX_ELITES = 256
 
 ERRORS = {0: "ONES_OK", -1: "ONES_ERR_NULL", -2: "ONES_ERR_BAD_JOB", -3: "ONES_ERR_BAD_PARAM",

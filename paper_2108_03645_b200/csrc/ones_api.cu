@@ -26,11 +26,12 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, refresh, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+    size_t pop0, pop1, P0, P1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, refresh, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
         status, total;
 };
 
-Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus = 0 /* > 0: per-GPU genome */) {
+Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus = 0 /* > 0: per-GPU genome */,
+                   bool packed = false /* the population also as one byte per gene */) {
     Layout L;
     size_t at = 0;
     auto take = [&](size_t bytes) {
@@ -45,6 +46,9 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus =
     const size_t pairs = trunc ? 3 * (size_t)pop : ((size_t)pop + 1) / 2;  // 2K parents + K mutant sources
     L.pop0 = take(rows * ldm * 4);
     L.pop1 = take(rows * ldm * 4);
+    const size_t p8 = packed ? rows * (((size_t)jmax + 511) / 512 * 512) : 16;
+    L.P0 = take(p8);
+    L.P1 = take(p8);
     L.F = take(rows * 8);
     L.F1 = take(rows * 8);
     L.G = take(rows * 4);
@@ -104,6 +108,10 @@ struct ones_ctx {
     bool trunc = false;     // ONES_FLAG_TRUNCATION
     bool per_gpu = false;   // ONES_FLAG_PER_GPU: one gene per GPU (a job id) instead of one per job
     bool narrow = false;    // per-GPU genome: capacity * max_per_gpu < 2^31 for every job (32-bit exponent search)
+    bool packed = false;    // ONES_FLAG_PACKED: the population lives as packed rows, the int32 buffers are scratch
+    int pcur = 0;           // packed buffer in force
+    int64_t ld8 = 0;        // stride of the packed rows
+    bool int_valid = false; // packed handle: pop(cur) holds the unpacked population
     int32_t W = 0;          // genes per candidate
     Tables tabS{};          // as tab, with the limits of a slot (any job id) for the shared operators
     int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
@@ -122,6 +130,7 @@ struct ones_ctx {
     size_t staging_bytes = 0;
 
     int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
+    uint8_t* P(int which) { return reinterpret_cast<uint8_t*>(ws + (which ? L.P1 : L.P0)); }
     double* Fbuf(int which) { return reinterpret_cast<double*>(ws + (which ? L.F1 : L.F)); }
     double* F() { return Fbuf(fcur); }
     int32_t* Gbuf(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.G1 : L.G)); }
@@ -220,7 +229,7 @@ void set_tables(ones_ctx* c, const ones_job* jobs, int32_t n_jobs) {
         c->fused = false;  // scoring a per-GPU candidate needs its job counts: separate kernel
     }
     c->cshape = ClusterShape{0, 0, 0, 0, 0};
-    if (c->fused && !c->trunc && !(c->prm.flags & ONES_FLAG_NO_CLUSTER))
+    if (c->fused && !c->trunc && !c->packed && !(c->prm.flags & ONES_FLAG_NO_CLUSTER))
         c->cshape = cluster_shape(c->tab, ld_of(n_jobs), c->N, c->prm.elitism, c->pairs);
 }
 
@@ -265,6 +274,8 @@ int run_fitness(ones_ctx* c) {
     if (rc) return rc;
     if (c->per_gpu)
         CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->narrow, c->F(), c->G(), c->stream));
+    else if (c->packed)
+        CU(c, launch_fitness_packed(c->P(c->pcur), c->ld8, c->N, c->tab, c->cap, c->prm.penalty, c->F(), c->G(), c->stream));
     else
         CU(c, launch_fitness(c->pop(c->cur), c->ld, c->N, c->J, c->tab, c->cap, c->prm.penalty, c->F(), c->G(),
                              c->stream));
@@ -272,6 +283,22 @@ int run_fitness(ones_ctx* c) {
     c->f_valid = true;
     c->elites_valid = false;
     return prof_end(c);
+}
+
+// Packed handle: the int32 buffer in force -> packed rows, and back.
+int pack_from_int(ones_ctx* c) {
+    c->ld8 = (int64_t)(((size_t)c->J + 511) / 512 * 512);
+    CU(c, launch_pack_rows(c->pop(c->cur), c->ld, c->N, c->J, c->P(c->pcur), c->ld8, c->stream));
+    c->launches += 1;
+    return ONES_OK;
+}
+
+int unpack_to_int(ones_ctx* c) {
+    if (c->int_valid) return ONES_OK;
+    CU(c, launch_unpack_rows(c->P(c->pcur), c->ld8, c->N, c->J, c->pop(c->cur), c->ld, nullptr, c->stream));
+    c->launches += 1;
+    c->int_valid = true;
+    return ONES_OK;
 }
 
 int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const int32_t* h_remap = nullptr) {
@@ -329,7 +356,9 @@ size_t ones_workspace_bytes_flags(int32_t n_jobs_max, int32_t pop, uint32_t flag
     const bool trunc = (flags & ONES_FLAG_TRUNCATION) != 0;
     if (trunc && pop > kPopLimit / 4) return 0;
     if (flags & ONES_FLAG_PER_GPU) return 0;  // needs the cluster size: ones_workspace_bytes_per_gpu
-    return make_layout(n_jobs_max, pop, trunc).total;
+    const bool packed = (flags & ONES_FLAG_PACKED) != 0;
+    if (packed && trunc) return 0;
+    return make_layout(n_jobs_max, pop, trunc, 0, packed).total;
 }
 
 size_t ones_workspace_bytes_per_gpu(int32_t n_jobs, int32_t pop, int32_t capacity) {
@@ -352,15 +381,17 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     if ((reinterpret_cast<uintptr_t>(d_workspace) & (kAlign - 1)) != 0) return ONES_ERR_ALIGN;
     const bool trunc = (p.flags & ONES_FLAG_TRUNCATION) != 0;
     const bool per_gpu = (p.flags & ONES_FLAG_PER_GPU) != 0;
+    const bool packed = (p.flags & ONES_FLAG_PACKED) != 0;
     if (trunc && (pop > kPopLimit / 4 || per_gpu)) return ONES_ERR_BAD_PARAM;
+    if (packed && (trunc || per_gpu)) return ONES_ERR_BAD_PARAM;
     if (per_gpu && capacity > kJobsLimit) return ONES_ERR_BAD_PARAM;
     const int32_t gpus = per_gpu ? capacity : 0;
-    if (workspace_bytes < make_layout(n_jobs, pop, trunc, gpus).total) return ONES_ERR_WORKSPACE;
+    if (workspace_bytes < make_layout(n_jobs, pop, trunc, gpus, packed).total) return ONES_ERR_WORKSPACE;
     // the largest job count this workspace can hold
     int32_t lo = n_jobs, hi = kJobsLimit;
     while (lo < hi) {
         const int32_t mid = lo + (hi - lo + 1) / 2;
-        if (make_layout(mid, pop, trunc, gpus).total <= workspace_bytes) lo = mid;
+        if (make_layout(mid, pop, trunc, gpus, packed).total <= workspace_bytes) lo = mid;
         else hi = mid - 1;
     }
     ones_ctx* c = new (std::nothrow) ones_ctx();
@@ -369,6 +400,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     c->J = n_jobs;
     c->Jmax = lo;
     c->per_gpu = per_gpu;
+    c->packed = packed;
     c->W = per_gpu ? capacity : n_jobs;
     c->N = pop;
     c->cap = capacity;
@@ -378,7 +410,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
     c->pairs = trunc ? pop : (pop - p.elitism + 1) / 2;
     c->ld = ld_of(c->W);
     c->ws = reinterpret_cast<char*>(d_workspace);
-    c->L = make_layout(c->Jmax, pop, trunc, gpus);
+    c->L = make_layout(c->Jmax, pop, trunc, gpus, packed);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) {
         free_ctx(c);
@@ -404,11 +436,16 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
         c->launches += 1;
         if (e != cudaSuccess) rc = cuda_fail(c, e);
     }
+    c->cur = 0;
+    if (rc == ONES_OK && packed) {
+        // the one-byte rows need the tables in shared memory (no separate scoring pass exists for them)
+        rc = c->fused ? pack_from_int(c) : ONES_ERR_BAD_PARAM;
+        c->int_valid = true;
+    }
     if (rc != ONES_OK) {
         free_ctx(c);
         return rc;
     }
-    c->cur = 0;
     c->f_valid = false;
     c->elites_valid = false;
     *out = c;
@@ -428,6 +465,10 @@ int ones_randomize(ones_ctx* c, uint64_t seed) {
     c->launches += 1;
     c->f_valid = false;
     c->elites_valid = false;
+    if (c->packed) {
+        c->int_valid = true;
+        return pack_from_int(c);
+    }
     return ONES_OK;
 }
 
@@ -446,6 +487,10 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
     }
     c->f_valid = false;
     c->elites_valid = false;
+    if (c->packed) {  // genes outside [0, 254] become "waits": what is read back comes from the packed rows
+        c->int_valid = false;
+        return pack_from_int(c);
+    }
     return ONES_OK;
 }
 
@@ -453,6 +498,10 @@ int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device
     DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
     if (ld < c->W) return ONES_ERR_BAD_PARAM;
+    if (c->packed) {
+        int rc = unpack_to_int(c);
+        if (rc) return rc;
+    }
     if (on_device) {
         CU(c, launch_copy_rows(c->pop(c->cur), c->ld, genomes, ld, c->N, c->W, 0, c->stream));
         c->launches += 1;
@@ -498,6 +547,14 @@ int ones_pack_population(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int3
     DeviceScope scope(c);
     if (!c || !d_packed) return ONES_ERR_NULL;
     if (c->per_gpu) return ONES_ERR_BAD_PARAM;  // job ids do not fit a byte
+    if (!d_genomes && c->packed) {  // the handle's own rows are packed already
+        if (ld8 < c->ld8) return ONES_ERR_BAD_PARAM;
+        if ((ld8 & 511) != 0 || !aligned16(d_packed)) return ONES_ERR_ALIGN;
+        if (ld8 != c->ld8) CU(c, cudaMemsetAsync(d_packed, 0xFF, (size_t)c->N * ld8, c->stream));
+        CU(c, cudaMemcpy2DAsync(d_packed, (size_t)ld8, c->P(c->pcur), (size_t)c->ld8, (size_t)c->ld8, (size_t)c->N,
+                                cudaMemcpyDeviceToDevice, c->stream));
+        return ONES_OK;
+    }
     if (!d_genomes) {
         d_genomes = c->pop(c->cur);
         ld = c->ld;
@@ -572,6 +629,30 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         return ONES_OK;
     }
     const int32_t E = c->prm.elitism;
+    if (c->packed) {
+        // parents read and children written as bytes: selection stage, then crossover + mutation + scoring
+        unsigned int* pdone = reinterpret_cast<unsigned int*>(c->status() + 1);
+        for (int32_t it = 0; it < generations; ++it) {
+            c->prof.sample = it % c->prof.every == 0;
+            if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
+            CU(c, launch_select_stage(c->F(), c->N, c->prm.tournament, c->pairs, keys, c->gen, c->parents(), E,
+                                      c->elites(0), c->ws + c->L.top, pdone, c->stream));
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+            if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
+            CU(c, launch_evolve_score_packed(c->P(c->pcur), c->P(c->pcur ^ 1), c->ld8, c->N, c->J, E, c->pairs, c->parents(),
+                                             c->elites(0), c->tab, keys, c->gen, c->thr16, c->cap, c->prm.penalty, c->F(),
+                                             c->G(), pdone + 1, c->stream));
+            if ((rc = prof_end(c)) != ONES_OK) return rc;
+            c->launches += 2;
+            c->pcur ^= 1;
+            c->gen += 1;
+        }
+        c->elast = 0;
+        c->elites_valid = false;
+        c->int_valid = false;
+        c->prof.sample = true;
+        return ONES_OK;
+    }
     if (c->cshape.cluster > 0) {
         // small population: every generation of this call inside one cluster launch
         if ((rc = prof_begin(c, 2)) != ONES_OK) return rc;
@@ -668,6 +749,10 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
     double* d_rate = reinterpret_cast<double*>(pack + 64);
     int32_t* d_genome = reinterpret_cast<int32_t*>(pack + 64 + J * 8);
     int32_t* d_gpus = reinterpret_cast<int32_t*>(pack + 64 + J * 12);
+    if (c->packed && !c->int_valid) {  // only the best row is needed as int32
+        CU(c, launch_unpack_rows(c->P(c->pcur), c->ld8, 1, c->J, c->pop(c->cur), c->ld, c->best_idx(), c->stream));
+        c->launches += 1;
+    }
     if (c->per_gpu)
         CU(c, launch_best_per_gpu(c->pop(c->cur), c->ld, c->W, c->J, c->best_idx(), c->tab,
                                   reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec,
@@ -704,9 +789,11 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
         if (capacity != c->cap) return ONES_ERR_BAD_PARAM;  // a candidate has one gene per GPU of the cluster
         if (refresh_smem(c->W, n_jobs) > (size_t)kMaxSmemPerBlock - 1024) return ONES_ERR_WORKSPACE;
     }
+    if (c->packed && (rc = unpack_to_int(c)) != ONES_OK) return rc;  // the column map works on the int32 rows
     const int64_t old_ld = c->ld;
     const int32_t old_J = c->J;
     rc = rebuild_tables(c, jobs, n_jobs, remap);
+    if (rc == ONES_OK && c->packed && !c->fused) rc = ONES_ERR_BAD_PARAM;  // tables of the new set do not fit shared memory
     if (rc != ONES_OK) {
         // put the tables of the job set in force back; the population is untouched
         const std::vector<ones_job> keep = c->h_jobs;
@@ -744,6 +831,10 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
     c->cap = capacity;
     c->f_valid = scored;
     c->elites_valid = false;
+    if (c->packed) {
+        c->int_valid = true;
+        return pack_from_int(c);
+    }
     return ONES_OK;
 }
 

@@ -59,6 +59,14 @@ cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t 
                              cudaStream_t s);
 cudaError_t launch_fitness_packed(const uint8_t* rows, int64_t ld8, int32_t n, Tables t, int32_t capacity,
                                   double penalty, double* F, int32_t* G, cudaStream_t s);
+// packed rows -> int32 rows (0xFF -> -1); row_index != NULL: only row *row_index, into the same row of dst
+cudaError_t launch_unpack_rows(const uint8_t* src, int64_t ld8, int32_t n, int32_t n_jobs, int32_t* dst, int64_t ld,
+                               const int32_t* row_index, cudaStream_t s);
+// crossover + mutation + scoring on packed rows (as launch_evolve_score: same tables, same counter)
+cudaError_t launch_evolve_score_packed(const uint8_t* src, uint8_t* dst, int64_t ld8, int32_t n, int32_t n_jobs, int32_t elitism,
+                                       int32_t pairs, const int32_t* parents, const int32_t* elites, Tables t,
+                                       RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity, double penalty,
+                                       double* F, int32_t* G, unsigned int* work, cudaStream_t s);
 // tournaments + top-e in one launch; *done must be 0 at launch (the kernel leaves it 0); done[1] is cleared for
 // the work-item counter of launch_evolve_score
 cudaError_t launch_select_stage(const double* F, int32_t n, int32_t tournament, int32_t pairs, RoundKeys keys,

@@ -422,6 +422,42 @@ cudaError_t launch_pack_rows(const int32_t* src, int64_t ld, int32_t n, int32_t 
     return cudaGetLastError();
 }
 
+// Packed rows back to int32 rows (0xFF -> -1, the waiting state).  One thread per int4 of the int32 row: its four
+// genes are one aligned 32-bit word of the tile.  row_index != NULL: only row *row_index is unpacked, into the
+// same row of dst.  Columns from n_jobs up to ld are written as 0.
+__global__ void __launch_bounds__(256)
+k_unpack_rows(const uint8_t* __restrict__ src, int64_t ld8, int32_t n, int32_t n_jobs, int32_t* __restrict__ dst, int64_t ld,
+              const int32_t* __restrict__ row_index) {
+    const int32_t nvec = (int32_t)(ld >> 2);
+    const int64_t total = (int64_t)n * nvec;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = row_index ? (int64_t)*row_index : i / nvec;
+        const int32_t j0 = 4 * (int32_t)(i % nvec);
+        const int32_t tile = j0 >> 9, b = (j0 >> 7) & 3, l = (j0 >> 2) & 31;
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(src + row * ld8 + (int64_t)tile * 512 + 16 * l + 4 * b);
+        int4 g;
+        g.x = (int32_t)(w & 0xFFu);
+        g.y = (int32_t)((w >> 8) & 0xFFu);
+        g.z = (int32_t)((w >> 16) & 0xFFu);
+        g.w = (int32_t)(w >> 24);
+        g.x = j0 < n_jobs ? (g.x == 255 ? -1 : g.x) : 0;
+        g.y = j0 + 1 < n_jobs ? (g.y == 255 ? -1 : g.y) : 0;
+        g.z = j0 + 2 < n_jobs ? (g.z == 255 ? -1 : g.z) : 0;
+        g.w = j0 + 3 < n_jobs ? (g.w == 255 ? -1 : g.w) : 0;
+        *reinterpret_cast<int4*>(dst + row * ld + j0) = g;
+    }
+}
+
+cudaError_t launch_unpack_rows(const uint8_t* src, int64_t ld8, int32_t n, int32_t n_jobs, int32_t* dst, int64_t ld,
+                               const int32_t* row_index, cudaStream_t s) {
+    if (row_index) n = 1;
+    if (n <= 0) return cudaSuccess;
+    const int64_t total = (int64_t)n * (ld >> 2);
+    const int64_t grid = (total + 255) / 256;
+    k_unpack_rows<<<(int)(grid < sm_count() * 16 ? grid : sm_count() * 16), 256, 0, s>>>(src, ld8, n, n_jobs, dst, ld, row_index);
+    return cudaGetLastError();
+}
+
 // Fitness of packed candidates: one candidate per warp, one 16-byte load per lane and tile (UNROLL tiles in
 // flight), tables in shared memory as for k_fitness.
 template <bool SMEM, int UNROLL>
@@ -1315,6 +1351,242 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
         }
         w = w_next;
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same pass on packed candidates (one byte per gene, tiles of 512 genes, see k_pack_rows): parents read and
+// children written as bytes, 2 bytes of HBM traffic per child gene instead of 8.  One 16-byte load gives a lane
+// the genes 4l..4l+3 of four consecutive 128-gene blocks; each of its four words is one block's int4 of the
+// int32 rows, so the random words (one Philox call per block and lane, counter = the int4's index), the
+// operators and the fixed summation order are those of k_evolve_score and the children equal the packed
+// int32 children byte for byte.  Crossover takes the four genes of a word at once (a byte mask from bit 0 of
+// the four random words); a mutated gene is inserted into its byte.  A parent byte of 0xFF (the job waits) is
+// inherited as it is.  Work items and shared-memory tables as in k_evolve_score.
+// ---------------------------------------------------------------------------------------------
+template <bool ALWAYS>
+__device__ __forceinline__ void mutate_byte(uint32_t& word, int s, uint32_t key, uint32_t thr32, uint32_t frac,
+                                            int32_t range, int32_t kmin) {
+    const uint32_t m = (uint32_t)(kmin + (int32_t)__umulhi(frac, (uint32_t)range));
+    const uint32_t with = (word & ~(0xFFu << (8 * s))) | (m << (8 * s));
+    word = (ALWAYS || key < thr32) ? with : word;
+}
+
+__device__ __forceinline__ void score_word(uint32_t w, uint32_t kcap, uint32_t strideX, uint32_t strideG,
+                                           const unsigned char* __restrict__ xrow, const unsigned char* __restrict__ grow,
+                                           double& sum, int32_t& gpus) {
+    score_gene((int32_t)(w & 0xFFu), kcap, strideX, strideG, xrow, grow, sum, gpus);
+    score_gene((int32_t)((w >> 8) & 0xFFu), kcap, strideX, strideG, xrow + 256, grow + 2, sum, gpus);
+    score_gene((int32_t)((w >> 16) & 0xFFu), kcap, strideX, strideG, xrow + 512, grow + 128, sum, gpus);
+    score_gene((int32_t)(w >> 24), kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
+}
+
+template <int THREADS, bool ALWAYS>
+__global__ void __launch_bounds__(THREADS, 1)
+k_evolve_score_packed(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int64_t ld8, int32_t n,
+                      int32_t n_jobs, int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents,
+                      const int32_t* __restrict__ elites, Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3,
+                      uint32_t thr32, int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G,
+                      unsigned int* __restrict__ work) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int32_t planes = t.k1 + 1;
+    const int32_t jpad = t.jpad;
+    unsigned char* sX = smem_raw;
+    unsigned char* sG = smem_raw + (size_t)planes * jpad * 8;
+    const int4* sKmin = reinterpret_cast<const int4*>(smem_raw + (size_t)planes * jpad * 10);
+    const int4* sRange = sKmin + jpad / 4;
+    {
+        const int32_t nX = planes * jpad / 2, nG = planes * jpad / 4;
+        const int4* gX = reinterpret_cast<const int4*>(t.X);
+        const int4* gG = reinterpret_cast<const int4*>(t.G);
+        for (int32_t i = threadIdx.x; i < nX; i += blockDim.x) reinterpret_cast<int4*>(sX)[i] = gX[i];
+        for (int32_t i = threadIdx.x; i < nG; i += blockDim.x) {
+            const int4 g = gG[i];
+            const int32_t plane = (4 * i) / jpad, slot = (4 * i) % jpad;
+            uint16_t* to = reinterpret_cast<uint16_t*>(sG) + plane * jpad + g16_pos(slot);
+            to[0] = (uint16_t)g.x;
+            to[2] = (uint16_t)g.y;
+            to[4] = (uint16_t)g.z;
+            to[6] = (uint16_t)g.w;
+        }
+        for (int32_t i = threadIdx.x; i < jpad / 4; i += blockDim.x) {
+            int4 lo = reinterpret_cast<const int4*>(t.kmin)[i];
+            // columns past the last job keep their 0xFF through a redraw (range 1, lower limit 255)
+            if (4 * i >= n_jobs) lo.x = 255;
+            if (4 * i + 1 >= n_jobs) lo.y = 255;
+            if (4 * i + 2 >= n_jobs) lo.z = 255;
+            if (4 * i + 3 >= n_jobs) lo.w = 255;
+            const_cast<int4*>(sKmin)[i] = lo;
+            const_cast<int4*>(sRange)[i] = reinterpret_cast<const int4*>(t.range)[i];
+        }
+        __syncthreads();
+    }
+    grid_dependency_wait();
+    const int lane = threadIdx.x & 31;
+    const int32_t warps_per_block = THREADS >> 5;
+    const int32_t total_warps = (int32_t)gridDim.x * warps_per_block;
+    const int32_t tiles = (int32_t)(ld8 >> 9);
+    const int32_t nblk = jpad >> 7;  // blocks of 128 genes that hold jobs; the blocks after them are copied
+    const uint32_t kcap = (uint32_t)t.k1;
+    const uint32_t strideX = (uint32_t)jpad * 8u, strideG = (uint32_t)jpad * 2u;
+    const unsigned char* srcb = src + lane * 16;
+    unsigned char* dstb = dst + lane * 16;
+    const unsigned char* xlane = sX + lane * 8;
+    const unsigned char* glane = sG + lane * 4;
+    const int2* pp = reinterpret_cast<const int2*>(parents);
+
+    const int32_t items = pairs + elitism;
+    const bool dynamic = items > total_warps;
+    unsigned int ticket = 0;
+    auto ask = [&]() {
+        if (dynamic && lane == 0) ticket = atomicAdd(work, 1u);
+    };
+    auto take = [&]() { return dynamic ? total_warps + (int32_t)__shfl_sync(0xFFFFFFFFu, ticket, 0) : items; };
+    auto ld_tile = [&](const unsigned char* p) {
+        const int4 v = ld_row(p);
+        return make_uint4((uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w);
+    };
+    int32_t w = (int32_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    ask();
+    int2 par = make_int2(0, 0);
+    uint4 qa = make_uint4(0, 0, 0, 0), qb = qa;
+    if (w < pairs) {
+        par = pp[w];
+        qa = ld_tile(srcb + par.x * ld8);
+        qb = ld_tile(srcb + par.y * ld8);
+    }
+    const int32_t take_at = tiles / 2;
+    while (w < pairs) {
+        const unsigned char* A = srcb + par.x * ld8;
+        const unsigned char* B = srcb + par.y * ld8;
+        const uint32_t slot0 = (uint32_t)(elitism + 2 * w);
+        const bool has1 = (int32_t)slot0 + 1 < n;
+        unsigned char* C = dstb + slot0 * ld8;
+        int32_t w_next = items;
+        bool more = false;
+        double sum0 = 0.0, sum1 = 0.0;
+        int32_t gp0 = 0, gp1 = 0;
+        for (int32_t tile = 0; tile < tiles; ++tile) {
+            if (tile == take_at) {
+                w_next = take();
+                ask();
+                more = w_next < pairs;
+                if (more) par = pp[w_next];  // A and B keep this pair's rows
+            }
+            // the next tile of both parents (after the last tile: the first of the next pair's) while this one is worked on
+            uint4 na = make_uint4(0, 0, 0, 0), nb = na;
+            if (tile + 1 < tiles) {
+                na = ld_tile(A + (tile + 1) * 512);
+                nb = ld_tile(B + (tile + 1) * 512);
+            } else if (more) {
+                na = ld_tile(srcb + par.x * ld8);
+                nb = ld_tile(srcb + par.y * ld8);
+            }
+            const uint32_t aw[4] = {qa.x, qa.y, qa.z, qa.w}, bw[4] = {qb.x, qb.y, qb.z, qb.w};
+            uint32_t c0w[4], c1w[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int32_t blk = tile * 4 + b;
+                c0w[b] = aw[b];
+                c1w[b] = bw[b];
+                if (blk < nblk) {  // warp-uniform
+                    const int32_t v = blk * 32 + lane;
+                    const int4 kmin = sKmin[v];
+                    const int4 range = sRange[v];
+                    const uint4 W = philox((uint32_t)v, slot0, gen_lo, c3, keys);
+                    // byte s of the even child comes from the second parent where bit 0 of random word s is set
+                    const uint32_t flips = (W.x & 1u) | ((W.y & 1u) << 8) | ((W.z & 1u) << 16) | ((W.w & 1u) << 24);
+                    const uint32_t m = flips * 0xFFu;
+                    c0w[b] = (aw[b] & ~m) | (bw[b] & m);
+                    c1w[b] = (bw[b] & ~m) | (aw[b] & m);
+                    const uint32_t Ws[4] = {W.x, W.y, W.z, W.w};
+                    const int32_t kmins[4] = {kmin.x, kmin.y, kmin.z, kmin.w}, ranges[4] = {range.x, range.y, range.z, range.w};
+#pragma unroll
+                    for (int s4 = 0; s4 < 4; ++s4) {
+                        const uint32_t R = __funnelshift_l(Ws[s4], Ws[s4], 16);  // halves swapped: even child's field on top
+                        mutate_byte<ALWAYS>(c0w[b], s4, R, thr32, Ws[s4] * 0x9E360001u, ranges[s4], kmins[s4]);
+                        mutate_byte<ALWAYS>(c1w[b], s4, Ws[s4], thr32, R * 0x85EB0001u, ranges[s4], kmins[s4]);
+                    }
+                    const unsigned char* xrow = xlane + blk * 1024;
+                    const unsigned char* grow = glane + blk * 256;
+                    score_word(c0w[b], kcap, strideX, strideG, xrow, grow, sum0, gp0);
+                    score_word(c1w[b], kcap, strideX, strideG, xrow, grow, sum1, gp1);
+                }
+            }
+            unsigned char* to = C + tile * 512;
+            *reinterpret_cast<uint4*>(to) = make_uint4(c0w[0], c0w[1], c0w[2], c0w[3]);
+            if (has1) *reinterpret_cast<uint4*>(to + ld8) = make_uint4(c1w[0], c1w[1], c1w[2], c1w[3]);
+            qa = na;
+            qb = nb;
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
+            gp0 += __shfl_xor_sync(0xFFFFFFFFu, gp0, off);
+            sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
+            gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
+        }
+        if (lane == 0) {
+            const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
+            F[slot0] = __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
+            G[slot0] = gp0;
+            if (has1) {
+                const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
+                F[slot0 + 1] = __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
+                G[slot0 + 1] = gp1;
+            }
+        }
+        w = w_next;
+    }
+    // ---- survivors: copied unchanged and scored again ----
+    while (w < items) {
+        const int32_t w_next = take();
+        ask();
+        const int32_t r = w - pairs;
+        const unsigned char* from = srcb + elites[r] * ld8;
+        unsigned char* to = dstb + r * ld8;
+        double sum = 0.0;
+        int32_t gp = 0;
+        for (int32_t tile = 0; tile < tiles; ++tile) {
+            const uint4 q = *reinterpret_cast<const uint4*>(from + tile * 512);
+            *reinterpret_cast<uint4*>(to + tile * 512) = q;
+            const uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int32_t blk = tile * 4 + b;
+                if (blk < nblk) score_word(qw[b], kcap, strideX, strideG, xlane + blk * 1024, glane + blk * 256, sum, gp);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            sum = __dadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, off));
+            gp += __shfl_xor_sync(0xFFFFFFFFu, gp, off);
+        }
+        if (lane == 0) {
+            const int32_t over = gp > capacity ? gp - capacity : 0;
+            F[r] = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+            G[r] = gp;
+        }
+        w = w_next;
+    }
+}
+
+cudaError_t launch_evolve_score_packed(const uint8_t* src, uint8_t* dst, int64_t ld8, int32_t n, int32_t n_jobs, int32_t elitism,
+                                       int32_t pairs, const int32_t* parents, const int32_t* elites, Tables t,
+                                       RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity, double penalty,
+                                       double* F, int32_t* G, unsigned int* work, cudaStream_t s) {
+    const int64_t warps = (int64_t)pairs + elitism;
+    if (warps <= 0) return cudaSuccess;
+    const size_t smem = evolve_score_smem(t);
+    if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
+    const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
+    constexpr int kThreads = 1024;
+    int64_t blocks = (warps + kThreads / 32 - 1) / (kThreads / 32);
+    if (blocks > sm_count()) blocks = sm_count();
+    auto kern = thr16 >= 65536u ? k_evolve_score_packed<kThreads, true> : k_evolve_score_packed<kThreads, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
+    if (e != cudaSuccess) return e;
+    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, src, dst, ld8, n, n_jobs, elitism, pairs, parents, elites, t,
+                                 keys, (uint32_t)gen, counter3(STREAM_MUT, gen), thr32, capacity, penalty, F, G, work);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -552,6 +552,98 @@ def test_packed_candidates_errors(ones):
     assert err.value.code == -3
 
 
+# ---- the generation on one-byte genes (ONES_FLAG_PACKED) ------------------------------------------------
+@pytest.mark.parametrize("J,N,kw", [(1, 3, {}), (5, 4, {}), (127, 33, {}), (129, 64, {}), (513, 70, dict(p_mut=1.0)),
+                                    (700, 2000, {}), (2048, 300, dict(p_mut=0.02, tournament=8)),
+                                    (100, 1024, dict(elitism=0)), (260, 1025, dict(elitism=5, tournament=1)),
+                                    (512, 9000, dict(p_mut=0.0)), (37, 101, dict(flags=33))])
+def test_packed_generation_parity(ones, J, N, kw):
+    """ones_evolve on packed rows: parents, elites, genomes, GPU demand and scores equal the oracle's after 1, 2
+    and 10 generations, and the packed rows equal the packed form of the oracle's population byte for byte."""
+    w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, kmin_max=2, pinned=J // 5)
+    kw = dict(kw)
+    if kw.get("flags", 0) & 1:
+        w.jobs["weight"] = np.random.default_rng(J).uniform(1e3, 1e6, J)
+    flags = kw.pop("flags", 32)
+    g, o = _pair(ones, w, flags=flags, **kw)
+    _same_state(g, o)  # every job at its smallest batch
+    g.randomize(1)
+    o.randomize(1)
+    _same_state(g, o)
+    for step in (1, 1, 8):
+        g.evolve(step, 2 ** 33 + 5)
+        o.evolve(step, 2 ** 33 + 5)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+    assert (g.pack().cpu().numpy() == _pack_numpy(o.get_population(), J)).all()
+    for repair in (False, True):
+        bg, bo = g.best(repair), o.best(repair)
+        # (with the SRUF score the library reports the per-job score terms, the oracle the throughputs)
+        for key in ("genome", "gpus_per_job") + (() if flags & 1 else ("rate_per_job",)):
+            assert (bg[key] == bo[key]).all(), (key, repair)
+        assert bg["fitness"] == bo["fitness"] and bg["total_gpus"] == bo["total_gpus"] and bg["index"] == bo["index"]
+
+
+def test_packed_generation_waiting_genes_and_job_set_change(ones):
+    """Waiting jobs (-1) are inherited through crossover on packed rows, and a job-set change converts, remaps and
+    packs again."""
+    w = inputs.custom(300, 256, 1500, 2, seed=5, kmax=6, kmin_max=1)
+    p = inputs.SearchParams(flags=32)
+    g = ones.Search(w.jobs, w.capacity, w.pop, p, n_jobs_max=400, guard_bytes=4096)
+    o = oracle.Search(w.jobs, w.capacity, w.pop, elitism=p.elitism, tournament=p.tournament, p_mut=p.p_mut,
+                      penalty=p.penalty)
+    rows = inputs.random_genomes(w.jobs, w.pop, seed=9, waiting_fraction=0.1)
+    g.set_population(rows)
+    o.set_population(rows)
+    _same_state(g, o)
+    g.evolve(3, 7)
+    o.evolve(3, 7)
+    _same_state(g, o)
+    assert (g.get_population() == -1).any()
+    rng = np.random.default_rng(3)
+    jobs = w.jobs
+    for rnd in range(2):
+        jobs2, remap = _changed_job_set(rng, jobs, 40, 55, seed=60 + rnd, kmax_new=rnd)
+        g.update_jobs(jobs2, remap, w.capacity)
+        o.update_jobs(jobs2, remap, w.capacity)
+        _same_state(g, o)
+        g.evolve(2, rnd)
+        o.evolve(2, rnd)
+        _same_state(g, o)
+        jobs = jobs2
+    assert g.guards_intact()
+    with pytest.raises(ones.OnesError) as err:   # not combinable with the truncation scheme
+        ones.Search(w.jobs, w.capacity, 64, inputs.SearchParams(flags=32 | 4))
+    assert err.value.code == -3
+
+
+def test_packed_generation_large_config(ones):
+    """The large workload on packed rows: two generations against the oracle, then 60 more against the int32 rows
+    of a second handle (same seeds: populations, scores and selections must stay identical)."""
+    w = inputs.large()
+    g, o = _pair(ones, w, flags=32)
+    h, _ = _pair(ones, w)
+    for s in (g, o, h):
+        s.randomize(w.seed)
+    for _ in range(2):
+        g.evolve(1, w.seed)
+        o.evolve(1, w.seed)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+    h.evolve(2, w.seed)
+    g.evolve(60, w.seed)
+    h.evolve(60, w.seed)
+    assert torch.equal(g.evaluate()[0], h.evaluate()[0]) and torch.equal(g.evaluate()[1], h.evaluate()[1])
+    assert torch.equal(g.get_population(on_device=True), h.get_population(on_device=True))
+    pg, eg = g.last_parents()
+    ph, eh = h.last_parents()
+    assert (pg == ph).all() and (eg == eh).all()
+
+
 # ---- a6: best and repair ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "paper", "mid"])
 def test_best_and_repair_parity(ones, name):
@@ -615,7 +707,8 @@ def test_update_jobs_parity(ones):
 
 # ---- no kernel writes outside the memory it was given ------------------------------------------------
 @pytest.mark.parametrize("flags,J,gpus,N", [(0, 37, 48, 101), (0, 300, 256, 6000), (2, 129, 64, 257), (8, 260, 128, 1025),
-                                            (4, 130, 64, 257), (16, 37, 130, 101), (16, 300, 257, 129), (1, 64, 64, 500)])
+                                            (4, 130, 64, 257), (16, 37, 130, 101), (16, 300, 257, 129), (1, 64, 64, 500), (32, 300, 256, 6000),
+                                            (32, 37, 48, 101)])
 def test_workspace_and_output_guards(ones, flags, J, gpus, N):
     """Every launch sequence with the workspace and the caller's output arrays between guard areas."""
     w = inputs.custom(J, gpus, N, 2, seed=J + N, kmax=6, kmin_max=1)
