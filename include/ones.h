@@ -223,7 +223,15 @@ int ones_best(ones_ctx* ctx, int repair, int32_t* h_genome, int32_t* h_gpus_per_
  * jobs leave, new jobs arrive, limits R_j move).  Column j of the new population is
  * column remap[j] of the old one clamped into the new [kmin_j, kmax_j], or kmin_j
  * when remap[j] == -1; the model tables are rebuilt.  jobs, remap: host, n_jobs
- * entries; n_jobs must fit the workspace.  Asynchronous apart from argument checks.
+ * entries; n_jobs must fit the workspace.  Asynchronous apart from argument checks: the job rows are checked on
+ * the host (limits as at ones_create, and a positive, finite throughput for every exponent; else
+ * ONES_ERR_BAD_JOB and the search is untouched).  The table kernel repeats the throughput check on the device;
+ * should it ever disagree, ONES_ERR_BAD_JOB comes from the next call that synchronises (ones_best,
+ * ones_get_population to host memory, ones_last_parents), like any asynchronous fault.
+ * When the new set has the same jobs in the same columns (remap[j] == j) and no job's [kmin, kmax] shrinks, no
+ * gene can move: the population is left where it is (after ones_set_population the full pass runs, since the
+ * caller's genes may lie outside the limits), the tables are rebuilt and the scores are recomputed when next
+ * needed; an identical job table and capacity change nothing at all.
  *
  * With ONES_FLAG_PER_GPU the candidates hold job ids, and every candidate goes through the four steps of
  * "Refresh" (Fig. 5) and then "Reorder":

@@ -112,6 +112,8 @@ struct ones_ctx {
     int pcur = 0;           // packed buffer in force
     int64_t ld8 = 0;        // stride of the packed rows
     bool int_valid = false; // packed handle: pop(cur) holds the unpacked population
+    bool flag_pending = false;  // the device-side job-table flag of the last ones_update_jobs has not been read yet
+    bool in_limits = false;     // every gene of the population is known to lie in its job's [kmin, kmax]
     int32_t W = 0;          // genes per candidate
     Tables tabS{};          // as tab, with the limits of a slot (any job id) for the shared operators
     int ecur = 0;           // elites buffer holding the elites of the population in force (if elites_valid)
@@ -183,6 +185,25 @@ int check_jobs(const ones_job* jobs, int32_t n) {
         if (((int64_t)q.b0 << q.kmax) >= ((int64_t)1 << 31)) return ONES_ERR_BAD_JOB;
         if (!(q.a >= 0.0) || !(q.c >= 0.0) || !(q.d >= 0.0)) return ONES_ERR_BAD_JOB;
         if (!isfinite(q.a) || !isfinite(q.c) || !isfinite(q.d) || !isfinite(q.weight)) return ONES_ERR_BAD_JOB;
+    }
+    return ONES_OK;
+}
+
+// Argument check: does every exponent of every job give a positive, finite throughput?  The tables themselves
+// are built on the device (which sets a flag under the same condition); this check only lets ones_update_jobs
+// reject a bad job table without waiting for the device.  Rows with ordinary magnitudes are accepted at
+// once (seconds per iteration >= a > 0, everything far from the ends of the double range); the rest are
+// evaluated exponent by exponent.
+int check_throughput(const ones_job* jobs, int32_t n) {
+    for (int32_t j = 0; j < n; ++j) {
+        const ones_job& q = jobs[j];
+        if (q.a > 1e-290 && q.a < 1e290 && q.c < 1e290 && q.d < 1e290) continue;
+        for (int32_t k = 0; k <= q.kmax; ++k) {
+            const int64_t b = (int64_t)q.b0 << k, m = q.max_per_gpu, g = (b + m - 1) / m;
+            const double sec = (q.a + q.c * ((double)b / (double)g)) + q.d * log2((double)g);
+            const double X = (double)b / sec;
+            if (!(X > 0.0) || X > 1.7976931348623157e308) return ONES_ERR_BAD_JOB;
+        }
     }
     return ONES_OK;
 }
@@ -301,7 +322,8 @@ int unpack_to_int(ones_ctx* c) {
     return ONES_OK;
 }
 
-int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const int32_t* h_remap = nullptr) {
+int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const int32_t* h_remap = nullptr,
+                   bool wait_for_flag = true) {
     const size_t jb = sizeof(ones_job) * (size_t)n_jobs, rb = h_remap ? (size_t)n_jobs * 4 : 0;
     int rc = ensure_staging(c, jb + rb);
     if (rc) return rc;
@@ -312,16 +334,38 @@ int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const in
     set_tables(c, h_jobs, n_jobs);
     CU(c, launch_build_tables(c->jobs(), n_jobs, c->prm.flags, c->tab, c->status(), c->stream));
     c->launches += 1;
-    int32_t bad = 0;
-    CU(c, cudaMemcpyAsync(&bad, c->status(), 4, cudaMemcpyDeviceToHost, c->stream));
-    CU(c, cudaStreamSynchronize(c->stream));
-    if (bad) return ONES_ERR_BAD_JOB;  // some job has a non-positive or non-finite throughput
+    if (wait_for_flag) {
+        int32_t bad = 0;
+        CU(c, cudaMemcpyAsync(&bad, c->status(), 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(c, cudaStreamSynchronize(c->stream));
+        if (bad) return ONES_ERR_BAD_JOB;  // some job has a non-positive or non-finite throughput
+        c->flag_pending = false;
+    } else {
+        c->flag_pending = true;  // read at the next call that synchronises (the host check has passed already)
+    }
     try {
         c->h_jobs.assign(h_jobs, h_jobs + n_jobs);
     } catch (...) {
         return ONES_ERR_NOMEM;
     }
     return ONES_OK;
+}
+
+// The job-table flag that ones_update_jobs left unread: fetched by the calls that synchronise anyway.
+int enqueue_flag_read(ones_ctx* c) {
+    if (!c->flag_pending) return ONES_OK;
+    int rc = ensure_staging(c, 64);
+    if (rc) return rc;
+    CU(c, cudaMemcpyAsync(c->staging + c->staging_bytes - 16, c->status(), 4, cudaMemcpyDeviceToHost, c->stream));
+    return ONES_OK;
+}
+
+int flag_after_sync(ones_ctx* c) {
+    if (!c->flag_pending) return ONES_OK;
+    c->flag_pending = false;
+    int32_t bad = 0;
+    memcpy(&bad, c->staging + c->staging_bytes - 16, 4);
+    return bad ? ONES_ERR_BAD_JOB : ONES_OK;
 }
 
 // Work of a handle always goes to the device it was created on, whatever device the caller has current.
@@ -437,6 +481,7 @@ int ones_create(ones_ctx** out, const ones_job* jobs, int32_t n_jobs, int32_t ca
         if (e != cudaSuccess) rc = cuda_fail(c, e);
     }
     c->cur = 0;
+    c->in_limits = !per_gpu;
     if (rc == ONES_OK && packed) {
         // the one-byte rows need the tables in shared memory (no separate scoring pass exists for them)
         rc = c->fused ? pack_from_int(c) : ONES_ERR_BAD_PARAM;
@@ -465,6 +510,7 @@ int ones_randomize(ones_ctx* c, uint64_t seed) {
     c->launches += 1;
     c->f_valid = false;
     c->elites_valid = false;
+    c->in_limits = !c->per_gpu;
     if (c->packed) {
         c->int_valid = true;
         return pack_from_int(c);
@@ -487,6 +533,7 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
     }
     c->f_valid = false;
     c->elites_valid = false;
+    c->in_limits = false;
     if (c->packed) {  // genes outside [0, 254] become "waits": what is read back comes from the packed rows
         c->int_valid = false;
         return pack_from_int(c);
@@ -508,7 +555,10 @@ int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device
     } else {
         CU(c, cudaMemcpy2DAsync(genomes, (size_t)ld * 4, c->pop(c->cur), (size_t)c->ld * 4, (size_t)c->W * 4,
                                 (size_t)c->N, cudaMemcpyDeviceToHost, c->stream));
+        int rc = enqueue_flag_read(c);
+        if (rc) return rc;
         CU(c, cudaStreamSynchronize(c->stream));
+        return flag_after_sync(c);
     }
     return ONES_OK;
 }
@@ -762,9 +812,11 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
                           reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
     c->launches += (uint64_t)nl + 1;
     const size_t bytes = 64 + J * 16;
-    if ((rc = ensure_staging(c, bytes)) != ONES_OK) return rc;
+    if ((rc = ensure_staging(c, bytes + 64)) != ONES_OK) return rc;
     CU(c, cudaMemcpyAsync(c->staging, pack, bytes, cudaMemcpyDeviceToHost, c->stream));
+    if ((rc = enqueue_flag_read(c)) != ONES_OK) return rc;
     CU(c, cudaStreamSynchronize(c->stream));
+    if ((rc = flag_after_sync(c)) != ONES_OK) return rc;
     BestOut rec;
     memcpy(&rec, c->staging, sizeof rec);
     if (h_rate_per_job) memcpy(h_rate_per_job, c->staging + 64, J * 8);
@@ -789,10 +841,31 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
         if (capacity != c->cap) return ONES_ERR_BAD_PARAM;  // a candidate has one gene per GPU of the cluster
         if (refresh_smem(c->W, n_jobs) > (size_t)kMaxSmemPerBlock - 1024) return ONES_ERR_WORKSPACE;
     }
+    if ((rc = check_throughput(jobs, n_jobs)) != ONES_OK) return rc;
+    if (!c->per_gpu && n_jobs == c->J && c->in_limits && (int32_t)c->h_jobs.size() == n_jobs) {
+        // Same jobs in the same columns, and no job's range of exponents shrinks: no gene moves, so the
+        // population stays where it is.  With an unchanged table even the scores stay; otherwise the tables are
+        // rebuilt and the population is scored again when it is next needed.
+        bool same_columns = true, same_table = capacity == c->cap;
+        for (int32_t j = 0; j < n_jobs && same_columns; ++j) {
+            const ones_job& was = c->h_jobs[j];
+            same_columns = remap[j] == j && jobs[j].kmin <= was.kmin && jobs[j].kmax >= was.kmax;
+            same_table = same_table && memcmp(&jobs[j], &was, sizeof(ones_job)) == 0;
+        }
+        if (same_columns) {
+            if (same_table) return ONES_OK;
+            if ((rc = rebuild_tables(c, jobs, n_jobs, nullptr, false)) != ONES_OK) return rc;
+            if (c->packed && !c->fused) return ONES_ERR_BAD_PARAM;
+            c->cap = capacity;
+            c->f_valid = false;
+            c->elites_valid = false;
+            return ONES_OK;
+        }
+    }
     if (c->packed && (rc = unpack_to_int(c)) != ONES_OK) return rc;  // the column map works on the int32 rows
     const int64_t old_ld = c->ld;
     const int32_t old_J = c->J;
-    rc = rebuild_tables(c, jobs, n_jobs, remap);
+    rc = rebuild_tables(c, jobs, n_jobs, remap, c->per_gpu);
     if (rc == ONES_OK && c->packed && !c->fused) rc = ONES_ERR_BAD_PARAM;  // tables of the new set do not fit shared memory
     if (rc != ONES_OK) {
         // put the tables of the job set in force back; the population is untouched
@@ -831,6 +904,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
     c->cap = capacity;
     c->f_valid = scored;
     c->elites_valid = false;
+    c->in_limits = true;  // every gene was clamped into its job's new limits
     if (c->packed) {
         c->int_valid = true;
         return pack_from_int(c);
@@ -845,8 +919,10 @@ int ones_last_parents(ones_ctx* c, int32_t* h_parents, int32_t* h_elites) {
         CU(c, cudaMemcpyAsync(h_parents, c->parents(), (size_t)c->pairs * 8, cudaMemcpyDeviceToHost, c->stream));
     if (h_elites && c->prm.elitism > 0 && !c->trunc)
         CU(c, cudaMemcpyAsync(h_elites, c->elites(c->elast), (size_t)c->prm.elitism * 4, cudaMemcpyDeviceToHost, c->stream));
+    int rc = enqueue_flag_read(c);
+    if (rc) return rc;
     CU(c, cudaStreamSynchronize(c->stream));
-    return ONES_OK;
+    return flag_after_sync(c);
 }
 
 int ones_model_table(ones_ctx* c, double* h_X, int32_t* h_g, int32_t* planes) {

@@ -705,6 +705,52 @@ def test_update_jobs_parity(ones):
     assert err.value.code == -5
 
 
+@pytest.mark.parametrize("flags", [0, 32])
+def test_update_jobs_same_columns(ones, flags):
+    """A job-set change that keeps every job in its column: nothing moves when no range of exponents shrinks (the
+    library then only rebuilds its tables), and the full pass still runs when a range shrinks or when the caller's
+    own genes may lie outside the limits."""
+    w = inputs.custom(300, 256, 6000, 2, seed=4, kmax=5, kmin_max=1)
+    g, o = _pair(ones, w, flags=flags)
+    ident = np.arange(300, dtype=np.int32)
+    g.randomize(2)
+    o.randomize(2)
+    g.evolve(2, 2)
+    o.evolve(2, 2)
+    for s in (g, o):
+        s.update_jobs(w.jobs, ident, w.capacity)           # the same table again
+    _same_state(g, o)
+    jobs2 = w.jobs.copy()
+    jobs2["a"] *= 1.25
+    jobs2["weight"] = 3.0
+    jobs2["kmax"] = np.minimum(jobs2["kmax"] + 1, 7)        # limits grow ("Scale-up")
+    for s in (g, o):
+        s.update_jobs(jobs2, ident, w.capacity + 7)         # capacity moves too
+    _same_state(g, o)
+    g.evolve(2, 3)
+    o.evolve(2, 3)
+    _same_state(g, o)
+    jobs3 = jobs2.copy()
+    jobs3["kmax"] = np.maximum(jobs3["kmax"] - 2, jobs3["kmin"])   # limits shrink: genes are clamped
+    for s in (g, o):
+        s.update_jobs(jobs3, ident, w.capacity)
+    _same_state(g, o)
+    rows = inputs.random_genomes(jobs2, w.pop, seed=8)      # genes up to the old, larger limits
+    for s in (g, o):
+        s.set_population(rows)
+        s.update_jobs(jobs3, ident, w.capacity)             # same table as in force, but the genes must be clamped
+    _same_state(g, o)
+    g.evolve(2, 4)
+    o.evolve(2, 4)
+    _same_state(g, o)
+    bad = jobs3.copy()
+    bad["a"][7] = bad["c"][7] = bad["d"][7] = 0.0            # no throughput: rejected on the host, nothing changes
+    with pytest.raises(ones.OnesError) as err:
+        g.update_jobs(bad, ident, w.capacity)
+    assert err.value.code == -2
+    _same_state(g, o)
+
+
 # ---- no kernel writes outside the memory it was given ------------------------------------------------
 @pytest.mark.parametrize("flags,J,gpus,N", [(0, 37, 48, 101), (0, 300, 256, 6000), (2, 129, 64, 257), (8, 260, 128, 1025),
                                             (4, 130, 64, 257), (16, 37, 130, 101), (16, 300, 257, 129), (1, 64, 64, 500), (32, 300, 256, 6000),
