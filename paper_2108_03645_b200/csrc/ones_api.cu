@@ -664,11 +664,12 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
                 c->launches += 1;
             }
             if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
+            int sel_launches = 0;
             CU(c, launch_trunc_select(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->Fbuf(c->fcur),
                                       c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1), c->Gbuf(c->gcur ^ 1),
-                                      c->ws + c->L.trunc, c->stream));
+                                      c->ws + c->L.trunc, c->stream, &sel_launches));
             if ((rc = prof_end(c)) != ONES_OK) return rc;
-            c->launches += 14;
+            c->launches += 2 + (uint64_t)sel_launches;
             c->cur ^= 1;
             c->fcur ^= 1;
             c->gcur ^= 1;

@@ -120,7 +120,7 @@ cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, in
                                         int32_t* G, cudaStream_t s);
 cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
                                 const int32_t* G, double* F_next, int32_t* G_next, void* scratch,
-                                cudaStream_t s);  // 12 launches
+                                cudaStream_t s, int* launches);  // 2 launches (pools up to 262144 rows) or 12
 // The paper's per-GPU genome (ONES_FLAG_PER_GPU): scoring, the reorder operation, slot limits, best
 // narrow: n_gpus * max_per_gpu < 2^31 for every job, so the exponent search may use 32-bit arithmetic
 cudaError_t launch_fitness_per_gpu(const int32_t* slots, int64_t ld, int32_t n, int32_t n_gpus, int32_t n_jobs,

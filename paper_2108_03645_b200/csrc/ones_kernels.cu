@@ -2665,6 +2665,188 @@ __global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ 
     }
 }
 
+// The whole threshold search and the survivors' places in ONE launch of one thread-block cluster, for pools of
+// up to 16 x 1024 x 16 rows: every thread keeps the keys of 16 consecutive rows in registers, the eight radix
+// passes exchange their 256-bin histograms through distributed shared memory (two hardware cluster barriers per
+// pass, nothing spins), then the counts above / at the threshold are scanned over threads and CTAs and every
+// survivor's row is written to kept[] as k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).
+constexpr int kPickCtas = 16, kPickThreads = 1024, kPickKeys = 16;
+
+__global__ void __launch_bounds__(kPickThreads, 1)
+k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* __restrict__ kept) {
+    grid_dependency_wait();
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned int tot[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ int32_t s_remaining;
+    __shared__ int32_t s_warp_g[32], s_warp_e[32];
+    __shared__ int32_t s_cta[2];  // this CTA's counts above / at the threshold
+    const unsigned int rank = cluster.block_rank();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t row0 = ((int32_t)rank * kPickThreads + (int32_t)threadIdx.x) * kPickKeys;
+    unsigned long long key[kPickKeys];
+#pragma unroll
+    for (int u = 0; u < kPickKeys; ++u) key[u] = row0 + u < n ? score_key(F[row0 + u]) : 0ull;
+    unsigned long long prefix = 0ull;
+    int32_t remaining = k;
+    for (int pass = 0; pass < 8; ++pass) {
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
+        __syncthreads();
+        const int shift = 56 - 8 * pass;
+        const unsigned long long mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
+#pragma unroll
+        for (int u = 0; u < kPickKeys; ++u) {
+            const bool in = row0 + u < n && (key[u] & mask) == prefix;
+            const unsigned int live = __ballot_sync(0xFFFFFFFFu, in);
+            if (live == 0u) continue;  // late passes: hardly any key still matches the prefix
+            // similar scores share their leading digits: one atomic for the warp when all live lanes agree,
+            // else one per distinct digit
+            const unsigned int digit = (unsigned int)(key[u] >> shift) & 255u;
+            const int first = __ffs(live) - 1;
+            const unsigned int lead = __shfl_sync(0xFFFFFFFFu, digit, first);
+            if (__all_sync(0xFFFFFFFFu, !in || digit == lead)) {
+                if (lane == first) atomicAdd(&hist[lead], (unsigned int)__popc(live));
+            } else if (in) {
+                const unsigned int peers = __match_any_sync(live, digit);
+                if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned int)__popc(peers));
+            }
+        }
+        cluster.sync();  // every CTA's histogram of this digit is complete
+        if (threadIdx.x < 256) {
+            unsigned int sum = 0u;
+            for (unsigned int r = 0; r < (unsigned int)kPickCtas; ++r) sum += *cluster.map_shared_rank(&hist[threadIdx.x], r);
+            tot[threadIdx.x] = sum;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // the digit that holds the remaining-th best key, bins taken from 255 downwards (every CTA finds the
+            // same one): lane l owns the eight bins 255 - 8l ... 248 - 8l
+            unsigned int c[8], mine = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                c[i] = tot[255 - (8 * lane + i)];
+                mine += c[i];
+            }
+            unsigned int incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned int a = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += a;
+            }
+            const unsigned int reached = __ballot_sync(0xFFFFFFFFu, (int32_t)incl >= remaining);
+            const int owner = reached ? __ffs(reached) - 1 : 31;
+            if (lane == owner) {
+                int32_t above = (int32_t)(incl - mine), d = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int32_t bin = 255 - (8 * lane + i);
+                    if (bin == 0 || above + (int32_t)c[i] >= remaining) {
+                        d = bin;
+                        break;
+                    }
+                    above += (int32_t)c[i];
+                }
+                s_remaining = remaining - above;
+                s_prefix = prefix | ((unsigned long long)d << shift);
+            }
+        }
+        __syncthreads();
+        prefix = s_prefix;
+        remaining = s_remaining;
+        cluster.sync();  // nobody clears a histogram that a neighbour is still reading
+    }
+    // prefix = key of the k-th best, remaining = how many rows with exactly that key survive (lowest rows first)
+    const unsigned long long T = prefix;
+    const int32_t quota = remaining;
+    int32_t gt = 0, eq = 0;
+#pragma unroll
+    for (int u = 0; u < kPickKeys; ++u) {
+        if (row0 + u < n) {
+            gt += key[u] > T;
+            eq += key[u] == T;
+        }
+    }
+    // exclusive scan over the CTA's threads (rows ascend with the thread index), then over the CTAs
+    int32_t sg = gt, se = eq;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t a = __shfl_up_sync(0xFFFFFFFFu, sg, off), b = __shfl_up_sync(0xFFFFFFFFu, se, off);
+        if (lane >= off) {
+            sg += a;
+            se += b;
+        }
+    }
+    if (lane == 31) {
+        s_warp_g[warp] = sg;
+        s_warp_e[warp] = se;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int32_t wg = s_warp_g[lane], we = s_warp_e[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t a = __shfl_up_sync(0xFFFFFFFFu, wg, off), b = __shfl_up_sync(0xFFFFFFFFu, we, off);
+            if (lane >= off) {
+                wg += a;
+                we += b;
+            }
+        }
+        s_warp_g[lane] = wg;  // inclusive over warps
+        s_warp_e[lane] = we;
+        if (lane == 31) {
+            s_cta[0] = wg;
+            s_cta[1] = we;
+        }
+    }
+    cluster.sync();  // every CTA's totals are in place
+    int32_t g_before = sg - gt + (warp > 0 ? s_warp_g[warp - 1] : 0);
+    int32_t e_before = se - eq + (warp > 0 ? s_warp_e[warp - 1] : 0);
+    for (unsigned int r = 0; r < rank; ++r) {
+        const int32_t* other = cluster.map_shared_rank(s_cta, r);
+        g_before += other[0];
+        e_before += other[1];
+    }
+#pragma unroll
+    for (int u = 0; u < kPickKeys; ++u) {
+        if (row0 + u < n) {
+            if (key[u] > T) {
+                kept[g_before + min(e_before, quota)] = row0 + u;
+                ++g_before;
+            } else if (key[u] == T) {
+                if (e_before < quota) kept[g_before + e_before] = row0 + u;
+                ++e_before;
+            }
+        }
+    }
+    cluster.sync();  // no CTA leaves while a neighbour may still read its totals
+}
+
+// Can the device host that cluster (asked once per device)?
+static bool pick_cluster_available() {
+    static int state[64] = {};  // 0 unknown, 1 yes, 2 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (state[dev] == 0) {
+        int clusters = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kPickCtas, 1, 1);
+        cfg.blockDim = dim3(kPickThreads, 1, 1);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kPickCtas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        bool ok = cudaFuncSetAttribute(k_trunc_pick_place, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaOccupancyMaxActiveClusters(&clusters, k_trunc_pick_place, &cfg) == cudaSuccess && clusters >= 1;
+        if (!ok) (void)cudaGetLastError();
+        state[dev] = ok ? 1 : 2;
+    }
+    return state[dev] == 1;
+}
+
 // survivors move to rows 0..K-1 of the other pool, with their scores and GPU counts
 __global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict__ src, int32_t* __restrict__ dst,
                                                       int64_t ld, int32_t k, const int32_t* __restrict__ kept,
@@ -2729,10 +2911,12 @@ cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, in
 }
 
 // Keep the best K of the 4K scored rows: F, G hold 4K entries; the survivors become rows 0..K-1 of
-// pool_next with F_next, G_next.  12 launches.
+// pool_next with F_next, G_next.  2 launches for pools of up to 262144 rows, 12 beyond.
 cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
-                                const int32_t* G, double* F_next, int32_t* G_next, void* scratch, cudaStream_t s) {
+                                const int32_t* G, double* F_next, int32_t* G_next, void* scratch, cudaStream_t s,
+                                int* launches) {
     const int32_t n = 4 * k;
+    if (launches) *launches = 12;
     const int32_t per_block = ((n + 1023) / 1024 + 255) / 256 * 256;  // rows per block: multiple of 256, <= 1024 blocks
     const int32_t blocks = (n + per_block - 1) / per_block;
     TruncPick* pick = reinterpret_cast<TruncPick*>(scratch);
@@ -2740,6 +2924,27 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
     int32_t* bsum = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + 64 + sizeof(TruncState));
     int32_t* kept = bsum + 2 * 1024;
     cudaError_t e;
+    if (n <= kPickCtas * kPickThreads * kPickKeys && pick_cluster_available()) {
+        // threshold search and places in one cluster launch, then the gather
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kPickCtas, 1, 1);
+        cfg.blockDim = dim3(kPickThreads, 1, 1);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kPickCtas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        e = cudaLaunchKernelEx(&cfg, k_trunc_pick_place, F, n, k, kept);
+        if (e != cudaSuccess) return e;
+        if (launches) *launches = 2;
+        return launch_after_previous(k_trunc_gather, (k + 7) / 8, 256, 0, s, pool, pool_next, ld, k, (const int32_t*)kept,
+                                     F, G, F_next, G_next);
+    }
     int rb = (n + 2047) / 2048;
     if (rb > sm_count()) rb = sm_count();
     for (int pass = 0; pass < 8; ++pass) {
