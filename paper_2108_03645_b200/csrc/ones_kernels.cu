@@ -1143,6 +1143,15 @@ __device__ __forceinline__ void score_int4(const int4 g, uint32_t kcap, uint32_t
     score_gene(g.w, kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
 }
 
+// Parent rows are asked to stay in L2 (tournament winners are read again by other pairs within the generation)
+// and child rows are written as streaming data, so that the 0.5 GB of children do not push the parents out:
+// measured 0.1785 -> 0.163 ms per generation at 2048 jobs x 65536 candidates.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 __device__ __forceinline__ int4 ld_row(const unsigned char* p) {
     int4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
@@ -1150,7 +1159,13 @@ __device__ __forceinline__ int4 ld_row(const unsigned char* p) {
                  : "l"(p));
     return v;
 }
-
+__device__ __forceinline__ int4 ld_row_hint(const unsigned char* p, uint64_t policy) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.s32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(policy));
+    return v;
+}
 // Shared memory: X planes (fp64), g planes narrowed to 16 bits (the host checks that every GPU count
 // fits), kmin and range per job (int32).  `work` is the item counter: zero at launch (the selection stage
 // clears it), it ends above the number of items.
@@ -1206,7 +1221,9 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
     const unsigned char* glane = sG + lane * 4;
     const int2* pp = reinterpret_cast<const int2*>(parents);
     const bool row_lane = FULL || lane < nvec;  // a lane past a short row's end never loads in block 0
-
+    const uint64_t keep = l2_policy_evict_last();
+    auto ldp = [&](const unsigned char* p) { return ld_row_hint(p, keep); };
+    auto stc = [&](unsigned char* p, const int4 v) { __stcs(reinterpret_cast<int4*>(p), v); };
     // Items [0, pairs) are pairs of children, [pairs, pairs + elitism) survivors.  A warp's first item is its own
     // number; when there are more items than warps, every later one comes from the counter: lane 0 asks for a
     // ticket an item ahead and the warp reads it (one shuffle) half-way through the item it is working on, in
@@ -1225,8 +1242,8 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
     if (w < pairs) {
         par = pp[w];
         if (row_lane) {
-            a0 = ld_row(srcb + par.x * row_bytes);
-            b0 = ld_row(srcb + par.y * row_bytes);
+            a0 = ldp(srcb + par.x * row_bytes);
+            b0 = ldp(srcb + par.y * row_bytes);
         }
     }
     // One step = one int4 of each parent -> one int4 of each child, scored.
@@ -1243,8 +1260,8 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             sibling_pair<ALWAYS>(W.z, cura.z, curb.z, kmin.z, range.z, thr32, c0.z, c1.z);
             sibling_pair<ALWAYS>(W.w, cura.w, curb.w, kmin.w, range.w, thr32, c0.w, c1.w);
             unsigned char* to = C + blk * 512;
-            *reinterpret_cast<int4*>(to) = c0;
-            if (has1) *reinterpret_cast<int4*>(to + row_bytes) = c1;
+            stc(to, c0);
+            if (has1) stc(to + row_bytes, c1);
             const unsigned char* xrow = xlane + blk * 1024;
             const unsigned char* grow = glane + blk * 256;
             score_int4(c0, kcap, strideX, strideG, xrow, grow, sum0, gp0);
@@ -1268,8 +1285,8 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             nb4 = na;
             if (nb < nblk) {
                 if (FULL || nb * 32 + lane < nvec) {
-                    na = ld_row(A + nb * 512);
-                    nb4 = ld_row(B + nb * 512);
+                    na = ldp(A + nb * 512);
+                    nb4 = ldp(B + nb * 512);
                 }
 #if ONES_ES_L2PF > 0
                 if ((nb % ONES_ES_L2PF) == 0 && nb + ONES_ES_L2PF < nblk) {
@@ -1283,8 +1300,8 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
                 }
 #endif
             } else if (more && row_lane) {
-                na = ld_row(srcb + par.x * row_bytes);
-                nb4 = ld_row(srcb + par.y * row_bytes);
+                na = ldp(srcb + par.x * row_bytes);
+                nb4 = ldp(srcb + par.y * row_bytes);
             }
         };
         for (int32_t blk = 0; blk < nblk; blk += 2) {
@@ -1441,8 +1458,9 @@ k_evolve_score_packed(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst
         if (dynamic && lane == 0) ticket = atomicAdd(work, 1u);
     };
     auto take = [&]() { return dynamic ? total_warps + (int32_t)__shfl_sync(0xFFFFFFFFu, ticket, 0) : items; };
+    const uint64_t keep = l2_policy_evict_last();
     auto ld_tile = [&](const unsigned char* p) {
-        const int4 v = ld_row(p);
+        const int4 v = ld_row_hint(p, keep);
         return make_uint4((uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w);
     };
     int32_t w = (int32_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
@@ -1513,8 +1531,8 @@ k_evolve_score_packed(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst
                 }
             }
             unsigned char* to = C + tile * 512;
-            *reinterpret_cast<uint4*>(to) = make_uint4(c0w[0], c0w[1], c0w[2], c0w[3]);
-            if (has1) *reinterpret_cast<uint4*>(to + ld8) = make_uint4(c1w[0], c1w[1], c1w[2], c1w[3]);
+            __stcs(reinterpret_cast<uint4*>(to), make_uint4(c0w[0], c0w[1], c0w[2], c0w[3]));
+            if (has1) __stcs(reinterpret_cast<uint4*>(to + ld8), make_uint4(c1w[0], c1w[1], c1w[2], c1w[3]));
             qa = na;
             qb = nb;
         }
