@@ -2444,6 +2444,7 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
     }
     grid_dependency_wait();  // the draws come from the kernel before
     constexpr int UN = 1;  // int4 per source row in flight per lane (2 measured 2 % slower)
+    const uint64_t keep = l2_policy_evict_last();  // the K current candidates are read about three times each
     const int lane = threadIdx.x & 31;
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
@@ -2468,8 +2469,8 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
                 for (int u = 0; u < UN; ++u) {
                     const int32_t v = v0 + 32 * u;
                     if (v < nvec) {
-                        a[u] = A[v];
-                        b[u] = B[v];
+                        a[u] = ld_row_hint(reinterpret_cast<const unsigned char*>(A + v), keep);
+                        b[u] = ld_row_hint(reinterpret_cast<const unsigned char*>(B + v), keep);
                     }
                 }
 #pragma unroll
@@ -2479,8 +2480,8 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
                         const uint4 W = philox((uint32_t)v, (uint32_t)(2 * q), gen_lo, c3cross, keys);
                         int4 c0, c1;
                         sibling_int4<false>(W, a[u], b[u], sKmin[v], sRange[v], 0u, true, c0, c1);  // threshold 0: no mutation
-                        C0[v] = c0;
-                        C1[v] = c1;
+                        __stcs(C0 + v, c0);
+                        __stcs(C1 + v, c1);
                         const int32_t base = (v >> 5) * 128 + lane;
                         score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
                         score4(c1, base, kcap, jpad, sX, sG, sum1, gp1);
@@ -2496,7 +2497,7 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
                 int4 g[UN];
 #pragma unroll
                 for (int u = 0; u < UN; ++u)
-                    if (v0 + 32 * u < nvec) g[u] = S[v0 + 32 * u];
+                    if (v0 + 32 * u < nvec) g[u] = ld_row_hint(reinterpret_cast<const unsigned char*>(S + v0 + 32 * u), keep);
 #pragma unroll
                 for (int u = 0; u < UN; ++u) {
                     const int32_t v = v0 + 32 * u;
@@ -2504,7 +2505,7 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
                         const uint4 W = philox((uint32_t)v, (uint32_t)m, gen_lo, c3mutant, keys);
                         int4 c0, c1;
                         sibling_int4<ALWAYS>(W, g[u], g[u], sKmin[v], sRange[v], thr32, false, c0, c1);  // the even child's draws
-                        C[v] = c0;
+                        __stcs(C + v, c0);
                         score4(c0, (v >> 5) * 128 + lane, kcap, jpad, sX, sG, sum0, gp0);
                     }
                 }
