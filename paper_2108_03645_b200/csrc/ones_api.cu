@@ -761,7 +761,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
         if (c->fused) {
             CU(c, launch_evolve_score(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->J, E, c->pairs,
                                       c->parents(), c->elites(0), c->tab, keys, c->gen, c->thr16, c->cap,
-                                      c->prm.penalty, c->F(), c->G(), done + 1, c->stream));
+                                      c->prm.penalty, c->F(), c->G(), done + 1, c->in_limits, c->stream));
         } else {
             CU(c, launch_evolve(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->W, E, c->pairs, c->parents(),
                                 c->elites(0), c->tabS, keys, c->gen, c->thr16, c->stream));

@@ -84,7 +84,8 @@ size_t evolve_score_smem(Tables t);
 cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                                 int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                                 Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                double penalty, double* F, int32_t* G, unsigned int* work, cudaStream_t s);
+                                double penalty, double* F, int32_t* G, unsigned int* work,
+                                bool in_limits /* every gene lies in its job's [kmin, kmax] */, cudaStream_t s);
 // One launch per generation (tournaments + crossover + mutation + scoring + the next generation's elites).
 struct GenerationShape {
     int blocks, threads;  // blocks == 0: not applicable, use the multi-launch sequence

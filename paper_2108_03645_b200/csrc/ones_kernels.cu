@@ -1126,21 +1126,25 @@ __device__ __forceinline__ void sibling_pair(uint32_t W, int32_t a, int32_t b, i
 
 // One gene's table look-ups: xrow/grow point at the lane's entries of this gene in plane 0, strideX/strideG
 // are the plane strides in bytes.
+// CLAMP = false: the caller knows that every gene lies in [0, k1] (a population whose genes are inside their jobs'
+// limits), so the gene itself is the plane.
+template <bool CLAMP = true>
 __device__ __forceinline__ void score_gene(int32_t k, uint32_t kcap, uint32_t strideX, uint32_t strideG,
                                            const unsigned char* __restrict__ xrow, const unsigned char* __restrict__ grow,
                                            double& sum, int32_t& gpus) {
-    const uint32_t p = min((uint32_t)k, kcap);
+    const uint32_t p = CLAMP ? min((uint32_t)k, kcap) : (uint32_t)k;
     sum = __dadd_rn(sum, *reinterpret_cast<const double*>(xrow + p * strideX));
     gpus += *reinterpret_cast<const uint16_t*>(grow + p * strideG);
 }
 
+template <bool CLAMP = true>
 __device__ __forceinline__ void score_int4(const int4 g, uint32_t kcap, uint32_t strideX, uint32_t strideG,
                                            const unsigned char* __restrict__ xrow, const unsigned char* __restrict__ grow,
                                            double& sum, int32_t& gpus) {
-    score_gene(g.x, kcap, strideX, strideG, xrow, grow, sum, gpus);
-    score_gene(g.y, kcap, strideX, strideG, xrow + 256, grow + 2, sum, gpus);
-    score_gene(g.z, kcap, strideX, strideG, xrow + 512, grow + 128, sum, gpus);
-    score_gene(g.w, kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
+    score_gene<CLAMP>(g.x, kcap, strideX, strideG, xrow, grow, sum, gpus);
+    score_gene<CLAMP>(g.y, kcap, strideX, strideG, xrow + 256, grow + 2, sum, gpus);
+    score_gene<CLAMP>(g.z, kcap, strideX, strideG, xrow + 512, grow + 128, sum, gpus);
+    score_gene<CLAMP>(g.w, kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
 }
 
 // Parent rows are asked to stay in L2 (tournament winners are read again by other pairs within the generation)
@@ -1169,7 +1173,7 @@ __device__ __forceinline__ int4 ld_row_hint(const unsigned char* p, uint64_t pol
 // Shared memory: X planes (fp64), g planes narrowed to 16 bits (the host checks that every GPU count
 // fits), kmin and range per job (int32).  `work` is the item counter: zero at launch (the selection stage
 // clears it), it ends above the number of items.
-template <int THREADS, bool ALWAYS, bool FULL>
+template <int THREADS, bool ALWAYS, bool FULL, bool CLAMP>
 __global__ void __launch_bounds__(THREADS, 1)
 k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
                int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents,
@@ -1264,8 +1268,8 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             if (has1) stc(to + row_bytes, c1);
             const unsigned char* xrow = xlane + blk * 1024;
             const unsigned char* grow = glane + blk * 256;
-            score_int4(c0, kcap, strideX, strideG, xrow, grow, sum0, gp0);
-            score_int4(c1, kcap, strideX, strideG, xrow, grow, sum1, gp1);
+            score_int4<CLAMP>(c0, kcap, strideX, strideG, xrow, grow, sum0, gp0);
+            score_int4<CLAMP>(c1, kcap, strideX, strideG, xrow, grow, sum1, gp1);
         }
     };
     const int32_t take_at = (nblk / 2) & ~1;  // the block (even) at which the next item's number is read
@@ -1353,7 +1357,7 @@ k_evolve_score(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64
             if (FULL || blk * 32 + lane < nvec) {
                 const int4 g = *reinterpret_cast<const int4*>(from + blk * 512);
                 *reinterpret_cast<int4*>(to + blk * 512) = g;
-                score_int4(g, kcap, strideX, strideG, xlane + blk * 1024, glane + blk * 256, sum, gp);
+                score_int4<CLAMP>(g, kcap, strideX, strideG, xlane + blk * 1024, glane + blk * 256, sum, gp);
             }
         }
 #pragma unroll
@@ -2015,7 +2019,8 @@ size_t evolve_score_smem(Tables t) { return (size_t)(t.k1 + 1) * t.jpad * 10 + (
 cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, int32_t n, int32_t n_jobs,
                                 int32_t elitism, int32_t pairs, const int32_t* parents, const int32_t* elites,
                                 Tables t, RoundKeys keys, uint64_t gen, uint32_t thr16, int32_t capacity,
-                                double penalty, double* F, int32_t* G, unsigned int* work, cudaStream_t s) {
+                                double penalty, double* F, int32_t* G, unsigned int* work, bool in_limits,
+                                cudaStream_t s) {
     const int64_t warps = (int64_t)pairs + elitism;
     if (warps <= 0) return cudaSuccess;
     const size_t smem = evolve_score_smem(t);
@@ -2030,12 +2035,16 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
     if (blocks > sm_count()) blocks = sm_count();
     void (*kern)(const int32_t*, int32_t*, int64_t, int32_t, int32_t, int32_t, int32_t, const int32_t*, const int32_t*,
                  Tables, RoundKeys, uint32_t, uint32_t, uint32_t, int32_t, double, double*, int32_t*, unsigned int*);
-    if (wide)
-        kern = always ? (full ? k_evolve_score<1024, true, true> : k_evolve_score<1024, true, false>)
-                      : (full ? k_evolve_score<1024, false, true> : k_evolve_score<1024, false, false>);
-    else
-        kern = always ? (full ? k_evolve_score<ONES_ES_THREADS, true, true> : k_evolve_score<ONES_ES_THREADS, true, false>)
-                      : (full ? k_evolve_score<ONES_ES_THREADS, false, true> : k_evolve_score<ONES_ES_THREADS, false, false>);
+    // the clamp of a gene to the tables' planes is only needed when genes may lie outside their jobs' limits
+    const bool clamp = !in_limits;
+#define ONES_ES_PICK(T)                                                                                              \
+    (always ? (full ? (clamp ? k_evolve_score<T, true, true, true> : k_evolve_score<T, true, true, false>)          \
+                    : (clamp ? k_evolve_score<T, true, false, true> : k_evolve_score<T, true, false, false>))       \
+            : (full ? (clamp ? k_evolve_score<T, false, true, true> : k_evolve_score<T, false, true, false>)        \
+                    : (clamp ? k_evolve_score<T, false, false, true> : k_evolve_score<T, false, false, false>)))
+    if (wide) kern = ONES_ES_PICK(1024);
+    else kern = ONES_ES_PICK(ONES_ES_THREADS);
+#undef ONES_ES_PICK
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
     return launch_after_previous(kern, (int)blocks, threads, smem, s, src, dst, ld, n, n_jobs, elitism, pairs, parents,
