@@ -313,12 +313,14 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "b88a7a4",
-    "source_sha16": "",
+    "captured_at": "dbf12f5",
+    "source_sha16": "6e1d3fd2291016af",
     "bytes_per_launch": {
-        ("large", 65536, "k_evolve_score"): 403.6e6 + 485.2e6,
-        ("large", 65536, "k_evolve"): 401.6e6 + 483.0e6,
-        ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
+        ("large", 65536, "k_evolve_score"): 379.5e6 + 481.2e6,
+        ("large", 65536, "k_evolve"): 401.4e6 + 483.5e6,
+        ("large", 65536, "k_fitness"): 537.1e6 + 1.3e6,
+        ("large", 65536, "k_evolve_score_packed"): 45.3e6 + 74.0e6,
+        ("large", 65536, "k_fitness_packed"): 134.5e6 + 1.0e6,
     },
 }
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2108_03645_b200", "csrc", "ones_kernels.cu")
@@ -621,7 +623,7 @@ def main():
                 line["kernels"][name] = roofline_entry(name, nbytes, t_ms, peak, peak_kind, traffic, at,
                                                        how="same workload with ONES_FLAG_UNFUSED (separate scoring pass)")
             line["kernels"]["k_fitness_packed"] = roofline_entry(
-                "k_fitness_packed", packed_bytes, packed_ms, peak, peak_kind, None, None,
+                "k_fitness_packed", packed_bytes, packed_ms, peak, peak_kind, *ncu_traffic(w.name, N, "k_fitness_packed"),
                 candidate_evals_per_s=N / (packed_ms * 1e-3),
                 how="ones_evaluate_packed on the same population stored as one byte per gene (a variant beside the "
                     "int32 contract); 20 launches back to back, two packed copies read in turn")
@@ -630,7 +632,7 @@ def main():
         # one parent byte read and one child byte written per child gene, the elite rows, indices, F and G
         pbytes = 2 * J * (N - E) + 2 * J * E + 8 * ((N - E + 1) // 2) + 4 * E + 12 * N
         line["kernels"]["k_evolve_score_packed"] = roofline_entry(
-            "k_evolve_score_packed", pbytes, k_ms, peak, peak_kind, None, None,
+            "k_evolve_score_packed", pbytes, k_ms, peak, peak_kind, *ncu_traffic(w.name, N, "k_evolve_score_packed"),
             ms_per_generation=gen_ms, generations_per_s=1e3 / gen_ms, candidate_evals_per_s=N * 1e3 / gen_ms,
             timed_repeats=reps3,
             how="same workload on a handle with ONES_FLAG_PACKED (population kept as one byte per gene; identical "
