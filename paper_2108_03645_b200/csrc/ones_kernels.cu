@@ -2704,7 +2704,7 @@ __global__ void __launch_bounds__(kPickThreads, 1)
 k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* __restrict__ kept) {
     grid_dependency_wait();
     cg::cluster_group cluster = cg::this_cluster();
-    __shared__ unsigned int hist[256];
+    __shared__ unsigned int hist[2][256];  // by pass parity: a histogram is cleared two passes after it was read
     __shared__ unsigned int tot[256];
     __shared__ unsigned long long s_prefix;
     __shared__ int32_t s_remaining;
@@ -2712,19 +2712,23 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     __shared__ int32_t s_cta[2];  // this CTA's counts above / at the threshold
     const unsigned int rank = cluster.block_rank();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int32_t row0 = ((int32_t)rank * kPickThreads + (int32_t)threadIdx.x) * kPickKeys;
+    // every thread owns `kpt` consecutive rows, so that all CTAs share the work whatever the pool's size
+    const int32_t kpt = (n + kPickCtas * kPickThreads - 1) / (kPickCtas * kPickThreads);
+    const int32_t row0 = ((int32_t)rank * kPickThreads + (int32_t)threadIdx.x) * kpt;
     unsigned long long key[kPickKeys];
 #pragma unroll
-    for (int u = 0; u < kPickKeys; ++u) key[u] = row0 + u < n ? score_key(F[row0 + u]) : 0ull;
+    for (int u = 0; u < kPickKeys; ++u) key[u] = (u < kpt && row0 + u < n) ? score_key(F[row0 + u]) : 0ull;
     unsigned long long prefix = 0ull;
     int32_t remaining = k;
     for (int pass = 0; pass < 8; ++pass) {
-        if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
+        unsigned int* myhist = hist[pass & 1];
+        if (threadIdx.x < 256) myhist[threadIdx.x] = 0u;
         __syncthreads();
         const int shift = 56 - 8 * pass;
         const unsigned long long mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
 #pragma unroll
         for (int u = 0; u < kPickKeys; ++u) {
+            if (u >= kpt) break;  // uniform
             const bool in = row0 + u < n && (key[u] & mask) == prefix;
             const unsigned int live = __ballot_sync(0xFFFFFFFFu, in);
             if (live == 0u) continue;  // late passes: hardly any key still matches the prefix
@@ -2734,16 +2738,17 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
             const int first = __ffs(live) - 1;
             const unsigned int lead = __shfl_sync(0xFFFFFFFFu, digit, first);
             if (__all_sync(0xFFFFFFFFu, !in || digit == lead)) {
-                if (lane == first) atomicAdd(&hist[lead], (unsigned int)__popc(live));
+                if (lane == first) atomicAdd(&myhist[lead], (unsigned int)__popc(live));
             } else if (in) {
                 const unsigned int peers = __match_any_sync(live, digit);
-                if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned int)__popc(peers));
+                if (lane == __ffs(peers) - 1) atomicAdd(&myhist[digit], (unsigned int)__popc(peers));
             }
         }
         cluster.sync();  // every CTA's histogram of this digit is complete
         if (threadIdx.x < 256) {
             unsigned int sum = 0u;
-            for (unsigned int r = 0; r < (unsigned int)kPickCtas; ++r) sum += *cluster.map_shared_rank(&hist[threadIdx.x], r);
+#pragma unroll
+            for (unsigned int r = 0; r < (unsigned int)kPickCtas; ++r) sum += *cluster.map_shared_rank(&myhist[threadIdx.x], r);
             tot[threadIdx.x] = sum;
         }
         __syncthreads();
@@ -2782,7 +2787,8 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
         __syncthreads();
         prefix = s_prefix;
         remaining = s_remaining;
-        cluster.sync();  // nobody clears a histogram that a neighbour is still reading
+        // no second barrier: the other histogram is the one cleared next, and every CTA finished reading it before
+        // it arrived at this pass's barrier
     }
     // prefix = key of the k-th best, remaining = how many rows with exactly that key survive (lowest rows first)
     const unsigned long long T = prefix;
@@ -2790,7 +2796,7 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     int32_t gt = 0, eq = 0;
 #pragma unroll
     for (int u = 0; u < kPickKeys; ++u) {
-        if (row0 + u < n) {
+        if (u < kpt && row0 + u < n) {
             gt += key[u] > T;
             eq += key[u] == T;
         }
@@ -2837,7 +2843,7 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     }
 #pragma unroll
     for (int u = 0; u < kPickKeys; ++u) {
-        if (row0 + u < n) {
+        if (u < kpt && row0 + u < n) {
             if (key[u] > T) {
                 kept[g_before + min(e_before, quota)] = row0 + u;
                 ++g_before;
