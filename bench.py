@@ -313,13 +313,13 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "dbf12f5",
-    "source_sha16": "6e1d3fd2291016af",
+    "captured_at": "6ea204c",
+    "source_sha16": "c8c29476ad451082",
     "bytes_per_launch": {
-        ("large", 65536, "k_evolve_score"): 379.5e6 + 481.2e6,
-        ("large", 65536, "k_evolve"): 401.4e6 + 483.5e6,
+        ("large", 65536, "k_evolve_score"): 379.3e6 + 481.6e6,
+        ("large", 65536, "k_evolve"): 401.5e6 + 483.7e6,
         ("large", 65536, "k_fitness"): 537.1e6 + 1.3e6,
-        ("large", 65536, "k_evolve_score_packed"): 45.3e6 + 74.0e6,
+        ("large", 65536, "k_evolve_score_packed"): 45.4e6 + 74.2e6,
         ("large", 65536, "k_fitness_packed"): 134.5e6 + 1.0e6,
     },
 }
