@@ -313,11 +313,11 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "6ea204c",
-    "source_sha16": "c8c29476ad451082",
+    "captured_at": "the commit that applies the L2 policies to k_evolve",
+    "source_sha16": "8790ad6a62d0494e",
     "bytes_per_launch": {
         ("large", 65536, "k_evolve_score"): 379.3e6 + 481.6e6,
-        ("large", 65536, "k_evolve"): 401.5e6 + 483.7e6,
+        ("large", 65536, "k_evolve"): 375.5e6 + 479.8e6,
         ("large", 65536, "k_fitness"): 537.1e6 + 1.3e6,
         ("large", 65536, "k_evolve_score_packed"): 45.4e6 + 74.2e6,
         ("large", 65536, "k_fitness_packed"): 134.5e6 + 1.0e6,

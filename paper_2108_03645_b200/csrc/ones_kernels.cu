@@ -981,12 +981,36 @@ __device__ __forceinline__ void sibling_int4(const uint4 W, const int4 a, const 
     sibling_gene<ALWAYS>(W.w, a.w, b.w, kmin.w, range.w, thr32, has1, c0.w, c1.w);
 }
 
+// Parent rows are asked to stay in L2 (tournament winners are read again by other pairs within the generation)
+// and child rows are written as streaming data, so that the 0.5 GB of children do not push the parents out:
+// measured 0.1785 -> 0.163 ms per generation at 2048 jobs x 65536 candidates.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+__device__ __forceinline__ int4 ld_row(const unsigned char* p) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int4 ld_row_hint(const unsigned char* p, uint64_t policy) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.s32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(policy));
+    return v;
+}
 template <int UNROLL, bool ALWAYS, int MINB = 4>
 __global__ void __launch_bounds__(256, MINB)
 k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld, int32_t n, int32_t n_jobs,
          int32_t elitism, int32_t pairs, const int32_t* __restrict__ parents, const int32_t* __restrict__ elites,
          Tables t, RoundKeys keys, uint32_t gen_lo, uint32_t c3, uint32_t thr32) {
     const int lane = threadIdx.x & 31;
+    const uint64_t keep = l2_policy_evict_last();
     const int32_t warps_per_block = blockDim.x >> 5;
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
     const int32_t nvec = (int32_t)(ld >> 2);
@@ -1016,8 +1040,8 @@ k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld,
             for (int u = 0; u < UNROLL; ++u) {
                 const int32_t v = v0 + u * 32 + lane;
                 if (v < nvec) {
-                    a[u] = A[v];
-                    b[u] = B[v];
+                    a[u] = ld_row_hint(reinterpret_cast<const unsigned char*>(A + v), keep);
+                    b[u] = ld_row_hint(reinterpret_cast<const unsigned char*>(B + v), keep);
                 }
             }
 #pragma unroll
@@ -1029,8 +1053,8 @@ k_evolve(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int64_t ld,
                     const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
                     int4 c0, c1;
                     sibling_int4<ALWAYS>(W, a[u], b[u], kmin, range, thr32, has1, c0, c1);
-                    C0[v] = c0;
-                    if (has1) C1[v] = c1;
+                    __stcs(C0 + v, c0);
+                    if (has1) __stcs(C1 + v, c1);
                 }
             }
         }
@@ -1147,29 +1171,6 @@ __device__ __forceinline__ void score_int4(const int4 g, uint32_t kcap, uint32_t
     score_gene<CLAMP>(g.w, kcap, strideX, strideG, xrow + 768, grow + 130, sum, gpus);
 }
 
-// Parent rows are asked to stay in L2 (tournament winners are read again by other pairs within the generation)
-// and child rows are written as streaming data, so that the 0.5 GB of children do not push the parents out:
-// measured 0.1785 -> 0.163 ms per generation at 2048 jobs x 65536 candidates.
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-
-__device__ __forceinline__ int4 ld_row(const unsigned char* p) {
-    int4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-__device__ __forceinline__ int4 ld_row_hint(const unsigned char* p, uint64_t policy) {
-    int4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.s32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p), "l"(policy));
-    return v;
-}
 // Shared memory: X planes (fp64), g planes narrowed to 16 bits (the host checks that every GPU count
 // fits), kmin and range per job (int32).  `work` is the item counter: zero at launch (the selection stage
 // clears it), it ends above the number of items.
