@@ -313,7 +313,7 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "the commit that applies the L2 policies to k_evolve",
+    "captured_at": "74836ee",
     "source_sha16": "8790ad6a62d0494e",
     "bytes_per_launch": {
         ("large", 65536, "k_evolve_score"): 379.3e6 + 481.6e6,
