@@ -314,7 +314,7 @@ def sha16(path: str) -> str:
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
     "captured_at": "74836ee",
-    "source_sha16": "8790ad6a62d0494e",
+    "source_sha16": "179e4634ec863a72",
     "bytes_per_launch": {
         ("large", 65536, "k_evolve_score"): 379.3e6 + 481.6e6,
         ("large", 65536, "k_evolve"): 375.5e6 + 479.8e6,

@@ -2695,10 +2695,11 @@ __global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ 
 }
 
 // The whole threshold search and the survivors' places in ONE launch of one thread-block cluster, for pools of
-// up to 16 x 1024 x 16 rows: every thread keeps the keys of 16 consecutive rows in registers, the eight radix
-// passes exchange their 256-bin histograms through distributed shared memory (two hardware cluster barriers per
-// pass, nothing spins), then the counts above / at the threshold are scanned over threads and CTAs and every
-// survivor's row is written to kept[] as k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).
+// up to 16 x 1024 x 16 rows: every thread keeps the keys of its (up to 16) consecutive rows in registers, the
+// eight radix passes exchange their 256-bin histograms through distributed shared memory (one hardware cluster
+// barrier per pass, the histograms alternating between two buffers; nothing spins), then the counts above / at
+// the threshold are scanned over threads and CTAs and every survivor's row is written to kept[] as
+// k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).
 constexpr int kPickCtas = 16, kPickThreads = 1024, kPickKeys = 16;
 
 __global__ void __launch_bounds__(kPickThreads, 1)
