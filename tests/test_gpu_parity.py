@@ -241,6 +241,26 @@ def test_evolve_parity_ragged_shapes(ones, J, N, flags):
     _same_state(g, o)
 
 
+@pytest.mark.parametrize("flags", [0, 32])
+@pytest.mark.parametrize("J,N,kw", [(260, 12000, dict(elitism=3)), (700, 20001, {}), (129, 9474, dict(elitism=0, p_mut=1.0)),
+                                    (512, 10000, dict(tournament=2))])
+def test_evolve_parity_more_pairs_than_warps(ones, J, N, kw, flags):
+    """Populations with more pairs of children than the persistent grid has warps (pairs beyond the first round are
+    handed out through the work counter) on ragged rows: an odd and an even number of 128-gene blocks, a partial
+    last block, an odd child count."""
+    w = inputs.custom(J, max(4, J), N, 3, seed=J + N, kmax=6, kmin_max=1, pinned=J // 7)
+    g, o = _pair(ones, w, flags=flags, **kw)
+    g.randomize(4)
+    o.randomize(4)
+    for step in (1, 2):
+        g.evolve(step, 77)
+        o.evolve(step, 77)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+
+
 def test_evolve_non_power_of_two_gpus_stays_within_tolerance(ones):
     # log2 of a non-power-of-two GPU count may differ from the oracle's in the last bit, so only the
     # first generation's scores are comparable gene for gene
