@@ -66,7 +66,9 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus =
     L.Gt = take((size_t)kPlanesMax * jp * 4);
     L.kmin = take(jp * 4);
     L.range = take(jp * 4);
-    L.jobs_in = take((size_t)jmax * (sizeof(ones_job) + 4));  // job rows, then the remap entries of an update
+    // job rows, then the remap entries of an update, then (only for job tables with GPU counts that are not powers
+    // of two) log2 of the GPU count per exponent and job
+    L.jobs_in = take((size_t)jmax * (sizeof(ones_job) + 8) + (size_t)(kPlanesMax - 1) * jmax * 8);
     {
         const size_t a = top_scratch_bytes(pop, ONES_MAX_ELITES), b = generation_scratch_bytes(ONES_MAX_ELITES);
         L.top = take(a > b ? a : b);
@@ -129,6 +131,8 @@ struct ones_ctx {
     int last_cuda = 0;
     Prof prof;
     unsigned char* staging = nullptr;  // small pinned host buffer: uploads and downloads go through it in one copy
+    cudaEvent_t staging_read = nullptr;  // recorded after an upload from the staging buffer: the host waits for it
+                                         // before it writes there again
     size_t staging_bytes = 0;
 
     int32_t* pop(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.pop1 : L.pop0)); }
@@ -154,6 +158,7 @@ int cuda_fail(ones_ctx* c, cudaError_t e);
 
 int ensure_staging(ones_ctx* c, size_t bytes) {
     if (bytes <= c->staging_bytes) return ONES_OK;
+    if (c->staging_read) cudaEventSynchronize(c->staging_read);  // no upload may still be reading the old buffer
     if (c->staging) cudaFreeHost(c->staging);
     c->staging = nullptr;
     c->staging_bytes = 0;
@@ -324,15 +329,39 @@ int unpack_to_int(ones_ctx* c) {
 
 int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const int32_t* h_remap = nullptr,
                    bool wait_for_flag = true) {
-    const size_t jb = sizeof(ones_job) * (size_t)n_jobs, rb = h_remap ? (size_t)n_jobs * 4 : 0;
-    int rc = ensure_staging(c, jb + rb);
+    // log2 of a GPU count that is not a power of two comes from the host's math library and is uploaded with the
+    // job rows: the device routine may differ from it in the last bit, and a last bit decides tournaments
+    int32_t kmax = 0;
+    bool all_pow2 = true;
+    for (int32_t j = 0; j < n_jobs; ++j) {
+        kmax = h_jobs[j].kmax > kmax ? h_jobs[j].kmax : kmax;
+        for (int32_t k = 0; k <= h_jobs[j].kmax && all_pow2; ++k) {
+            const int64_t b = (int64_t)h_jobs[j].b0 << k, m = h_jobs[j].max_per_gpu, g = (b + m - 1) / m;
+            all_pow2 = (g & (g - 1)) == 0;
+        }
+    }
+    const size_t jb = sizeof(ones_job) * (size_t)n_jobs, rb = (size_t)n_jobs * 8;  // remap entries padded to 8 bytes each
+    const size_t lb = all_pow2 ? 0 : (size_t)(kmax + 1) * n_jobs * 8;
+    int rc = ensure_staging(c, jb + rb + lb);
     if (rc) return rc;
+    if (!c->staging_read) CU(c, cudaEventCreateWithFlags(&c->staging_read, cudaEventDisableTiming));
+    CU(c, cudaEventSynchronize(c->staging_read));  // the last upload has left the staging buffer
     memcpy(c->staging, h_jobs, jb);
-    if (h_remap) memcpy(c->staging + jb, h_remap, rb);
+    if (h_remap) memcpy(c->staging + jb, h_remap, (size_t)n_jobs * 4);
+    if (lb) {
+        double* lg = reinterpret_cast<double*>(c->staging + jb + rb);
+        for (int32_t k = 0; k <= kmax; ++k)
+            for (int32_t j = 0; j < n_jobs; ++j) {
+                const int64_t b = (int64_t)h_jobs[j].b0 << (k <= h_jobs[j].kmax ? k : 0), m = h_jobs[j].max_per_gpu;
+                lg[(size_t)k * n_jobs + j] = log2((double)((b + m - 1) / m));
+            }
+    }
     CU(c, cudaMemsetAsync(c->status(), 0, 16, c->stream));
-    CU(c, cudaMemcpyAsync(c->jobs(), c->staging, jb + rb, cudaMemcpyHostToDevice, c->stream));
+    CU(c, cudaMemcpyAsync(c->jobs(), c->staging, (h_remap || lb) ? jb + rb + lb : jb, cudaMemcpyHostToDevice, c->stream));
+    CU(c, cudaEventRecord(c->staging_read, c->stream));
+    const double* d_lg = lb ? reinterpret_cast<const double*>(reinterpret_cast<const unsigned char*>(c->jobs()) + jb + rb) : nullptr;
     set_tables(c, h_jobs, n_jobs);
-    CU(c, launch_build_tables(c->jobs(), n_jobs, c->prm.flags, c->tab, c->status(), c->stream));
+    CU(c, launch_build_tables(c->jobs(), n_jobs, c->prm.flags, c->tab, d_lg, c->status(), c->stream));
     c->launches += 1;
     if (wait_for_flag) {
         int32_t bad = 0;
@@ -384,6 +413,7 @@ void free_ctx(ones_ctx* c) {
     if (!c) return;
     for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
     if (c->staging) cudaFreeHost(c->staging);
+    if (c->staging_read) cudaEventDestroy(c->staging_read);
     delete c;
 }
 

@@ -46,7 +46,10 @@ struct BestOut {  // device record written by the best/repair kernel
     int32_t steps;
 };
 
+// d_log2g: NULL, or log2 of the GPU count per (exponent, job) as double[k1][n_jobs] for job tables whose GPU counts
+// are not all powers of two (computed by the caller's math library so that both sides of a comparison agree)
 cudaError_t launch_build_tables(const ones_job* d_jobs, int32_t n_jobs, uint32_t flags, Tables t,
+                                const double* d_log2g,
                                 int32_t* d_bad /*set to 1 when a throughput is not positive and finite*/,
                                 cudaStream_t s);
 cudaError_t launch_fill_min(int32_t* pop, int64_t ld, int32_t n, int32_t n_jobs, Tables t, cudaStream_t s);

@@ -104,7 +104,7 @@ static cudaError_t launch_after_previous(void (*kernel)(Params...), int blocks, 
 // Model tables: X_j(k), g_j(k) for every job and exponent (throughput model of the job table)
 // ---------------------------------------------------------------------------------------------
 __global__ void k_build_tables(const ones_job* __restrict__ jobs, int32_t n_jobs, uint32_t flags, Tables t,
-                               int32_t* __restrict__ bad) {
+                               const double* __restrict__ log2g, int32_t* __restrict__ bad) {
     const int32_t planes = t.k1 + 1;
     const int64_t total = (int64_t)planes * t.jpad;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
@@ -120,8 +120,12 @@ __global__ void k_build_tables(const ones_job* __restrict__ jobs, int32_t n_jobs
                 const long long m = job.max_per_gpu;
                 const long long g = (b + m - 1) / m;
                 const double local = __ddiv_rn((double)b, (double)g);
-                // log2 of a power of two is its exponent, exactly; otherwise the library routine
-                const double lg = ((g & (g - 1)) == 0) ? (double)(63 - __clzll(g)) : log2((double)g);
+                // log2 of a power of two is its exponent, exactly; otherwise the value the caller supplies (its own
+                // math library's, so that a comparison with host arithmetic is not decided by a last bit), else the
+                // device routine
+                const double lg = ((g & (g - 1)) == 0) ? (double)(63 - __clzll(g))
+                                  : log2g       ? log2g[(int64_t)k * n_jobs + j]
+                                                : log2((double)g);
                 const double sec = __dadd_rn(__dadd_rn(job.a, __dmul_rn(job.c, local)), __dmul_rn(job.d, lg));
                 const double X = __ddiv_rn((double)b, sec);
                 if (!(X > 0.0) || X > 1.7976931348623157e308) atomicOr(bad, 1);  // needs seconds/iteration > 0
@@ -143,10 +147,10 @@ __global__ void k_build_tables(const ones_job* __restrict__ jobs, int32_t n_jobs
 }
 
 cudaError_t launch_build_tables(const ones_job* d_jobs, int32_t n_jobs, uint32_t flags, Tables t,
-                                int32_t* d_bad, cudaStream_t s) {
+                                const double* d_log2g, int32_t* d_bad, cudaStream_t s) {
     const int64_t total = (int64_t)(t.k1 + 1) * t.jpad;
     const int grid = (int)((total + 255) / 256);
-    k_build_tables<<<grid < 1024 ? grid : 1024, 256, 0, s>>>(d_jobs, n_jobs, flags, t, d_bad);
+    k_build_tables<<<grid < 1024 ? grid : 1024, 256, 0, s>>>(d_jobs, n_jobs, flags, t, d_log2g, d_bad);
     return cudaGetLastError();
 }
 
