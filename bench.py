@@ -313,14 +313,14 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "74836ee",
-    "source_sha16": "179e4634ec863a72",
+    "captured_at": "964a7d5",
+    "source_sha16": "2f942f73bf557d81",
     "bytes_per_launch": {
-        ("large", 65536, "k_evolve_score"): 379.3e6 + 481.6e6,
-        ("large", 65536, "k_evolve"): 375.5e6 + 479.8e6,
-        ("large", 65536, "k_fitness"): 537.1e6 + 1.3e6,
-        ("large", 65536, "k_evolve_score_packed"): 45.4e6 + 74.2e6,
-        ("large", 65536, "k_fitness_packed"): 134.5e6 + 1.0e6,
+        ("large", 65536, "k_evolve_score"): 379.7e6 + 481.1e6,
+        ("large", 65536, "k_evolve"): 375.1e6 + 479.1e6,
+        ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
+        ("large", 65536, "k_evolve_score_packed"): 45.1e6 + 73.7e6,
+        ("large", 65536, "k_fitness_packed"): 134.5e6 + 0.3e6,
     },
 }
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2108_03645_b200", "csrc", "ones_kernels.cu")

@@ -44,6 +44,8 @@ typedef struct ones_ctx ones_ctx;
  * grid and b0 << kmax the batch-size limit R_j (Section 3.2.2, "Evolution");
  * a, c, d are the coefficients of the job's profiled throughput X_j (Eq. 5):
  * seconds per iteration t = a + c * (B / g) + d * log2(g) on g GPUs, X = B / t.
+ * log2(g) is the exact integer for a power of two; for any other g it is taken with the host's
+ * math library when the job table is set and uploaded, not computed on the device.
  * weight is the per-job factor Y_processed * (1/rho - 1) of Alg. 1's score; it is
  * used only with ONES_FLAG_SRUF.  48 bytes. */
 typedef struct {
