@@ -586,8 +586,14 @@ def main():
                 rows = {"children (k_trunc_draws + k_trunc_children)": ("evolve", 6 * N * J * 4),
                         "k_fitness over the 3N new rows": ("fitness", 3 * N * (4 * J + 12))}
             else:  # 3N children written and scored in one pass: 3N row reads, 3N row writes, (F, G) of each
-                rows = {"children + scores (k_trunc_draws + k_trunc_children_score)": ("evolve", 6 * N * J * 4 + 3 * N * 12)}
-            rows["selection (threshold search, compaction, k_trunc_gather)"] = ("select", 2 * N * J * 4 + 4 * N * 8 * 3)
+                rows = {"children + scores (k_trunc_children_score)": ("evolve", 6 * N * J * 4 + 3 * N * 12)}
+            if launches == 2 * steps:
+                # fused handle: the pool is used in place, one cluster launch finds the threshold, the survivors'
+                # places and the new row map (scores, GPU counts and the map: no candidate row moves)
+                rows["selection in place (k_trunc_pick_place: threshold, places, row map)"] = \
+                    ("select", 4 * N * 8 + N * 12 * 2 + 4 * N * 4 * 2)
+            else:
+                rows["selection (threshold search, compaction, k_trunc_gather)"] = ("select", 2 * N * J * 4 + 4 * N * 8 * 3)
             line["kernels"] = {}
             for name, (stage, nbytes) in rows.items():
                 line["kernels"][name] = roofline_entry(name, nbytes, stage_ms[stage] / stage_n[stage], peak, peak_kind,

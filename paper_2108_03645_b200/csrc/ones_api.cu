@@ -26,7 +26,7 @@ inline int32_t ld_of(int32_t n_jobs) { return (n_jobs + 3) & ~3; }
 inline int32_t jpad_of(int32_t n_jobs) { return (n_jobs + 127) & ~127; }
 
 struct Layout {
-    size_t pop0, pop1, P0, P1, F, F1, G, G1, trunc, slot_kmin, slot_range, fit, refresh, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
+    size_t pop0, pop1, P0, P1, F, F1, G, G1, trunc, rowmap0, rowmap1, slot_kmin, slot_range, fit, refresh, parents, elites, elites1, best_idx, X, Gt, kmin, range, jobs_in, top, work, out_pack, exp_X, exp_G,
         status, total;
 };
 
@@ -54,6 +54,8 @@ Layout make_layout(int32_t jmax, int32_t pop, bool trunc = false, int32_t gpus =
     L.G = take(rows * 4);
     L.G1 = take(rows * 4);
     L.trunc = take(trunc ? trunc_scratch_bytes(pop) : 16);
+    L.rowmap0 = take(trunc ? rows * 4 : 16);  // pool used in place: logical row -> pool row, two maps in turn
+    L.rowmap1 = take(trunc ? rows * 4 : 16);
     L.slot_kmin = take(sp * 4);
     L.slot_range = take(sp * 4);
     L.fit = take(gpus > 0 ? jp * 16 : 16);  // per-GPU genome: the jobs' limits in the tables' job order
@@ -108,6 +110,8 @@ struct ones_ctx {
     int fcur = 0;           // score buffer in force
     int gcur = 0;           // GPU-count buffer in force (only the truncation scheme alternates it)
     bool trunc = false;     // ONES_FLAG_TRUNCATION
+    bool mapped = false;    // truncation scheme: the pool is in use in place, logical row r lives in pool row rowmap(mcur)[r]
+    int mcur = 0;           // row map in force (if mapped)
     bool per_gpu = false;   // ONES_FLAG_PER_GPU: one gene per GPU (a job id) instead of one per job
     bool narrow = false;    // per-GPU genome: capacity * max_per_gpu < 2^31 for every job (32-bit exponent search)
     bool packed = false;    // ONES_FLAG_PACKED: the population lives as packed rows, the int32 buffers are scratch
@@ -142,6 +146,7 @@ struct ones_ctx {
     int32_t* Gbuf(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.G1 : L.G)); }
     int32_t* G() { return Gbuf(gcur); }
     int32_t* parents() { return reinterpret_cast<int32_t*>(ws + L.parents); }
+    int32_t* rowmap(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.rowmap1 : L.rowmap0)); }
     int32_t* elites(int which) { return reinterpret_cast<int32_t*>(ws + (which ? L.elites1 : L.elites)); }
     int32_t* best_idx() { return reinterpret_cast<int32_t*>(ws + L.best_idx); }
     ones_job* jobs() { return reinterpret_cast<ones_job*>(ws + L.jobs_in); }
@@ -295,8 +300,22 @@ int prof_end(ones_ctx* c) {
     return ONES_OK;
 }
 
+// Truncation scheme with the pool used in place: bring the K candidates, in order, to rows 0..K-1 of the other
+// pool and go on there with logical row = pool row.  Everything that reads or replaces the population as rows
+// calls this first; generations that follow one another never do.
+int compact_pool(ones_ctx* c) {
+    if (!c->mapped) return ONES_OK;
+    CU(c, launch_trunc_compact(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->rowmap(c->mcur), c->stream));
+    c->launches += 1;
+    c->cur ^= 1;
+    c->mapped = false;
+    return ONES_OK;
+}
+
 int run_fitness(ones_ctx* c) {
-    int rc = prof_begin(c, 0);
+    int rc = compact_pool(c);
+    if (rc) return rc;
+    rc = prof_begin(c, 0);
     if (rc) return rc;
     if (c->per_gpu)
         CU(c, launch_fitness_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, c->J, c->tab, c->fit(), c->narrow, c->F(), c->G(), c->stream));
@@ -536,6 +555,7 @@ int ones_destroy(ones_ctx* c) {
 int ones_randomize(ones_ctx* c, uint64_t seed) {
     DeviceScope scope(c);
     if (!c) return ONES_ERR_NULL;
+    c->mapped = false;  // every candidate is replaced
     CU(c, launch_randomize(c->pop(c->cur), c->ld, c->N, c->W, c->tabS, make_round_keys(seed), c->stream));
     c->launches += 1;
     c->f_valid = false;
@@ -552,6 +572,7 @@ int ones_set_population(ones_ctx* c, const int32_t* genomes, int64_t ld, int on_
     DeviceScope scope(c);
     if (!c || !genomes) return ONES_ERR_NULL;
     if (ld < c->W) return ONES_ERR_BAD_PARAM;
+    c->mapped = false;  // every candidate is replaced
     if (on_device) {
         CU(c, launch_copy_rows(genomes, ld, c->pop(c->cur), c->ld, c->N, c->W, 1, c->stream));
         c->launches += 1;
@@ -577,6 +598,10 @@ int ones_get_population(ones_ctx* c, int32_t* genomes, int64_t ld, int on_device
     if (ld < c->W) return ONES_ERR_BAD_PARAM;
     if (c->packed) {
         int rc = unpack_to_int(c);
+        if (rc) return rc;
+    }
+    {
+        int rc = compact_pool(c);
         if (rc) return rc;
     }
     if (on_device) {
@@ -636,6 +661,8 @@ int ones_pack_population(ones_ctx* c, const int32_t* d_genomes, int64_t ld, int3
         return ONES_OK;
     }
     if (!d_genomes) {
+        int rc = compact_pool(c);
+        if (rc) return rc;
         d_genomes = c->pop(c->cur);
         ld = c->ld;
         n = c->N;
@@ -674,6 +701,11 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
     const RoundKeys keys = make_round_keys(seed);
     if (c->trunc) {
         // the paper's scheme: pool of 4K rows, best K survive (elitism and tournament size do not apply)
+        // Fused handles use the pool in place: survivors keep their pool rows, a map of 4K entries says where each
+        // logical row lives, and no candidate is copied between generations (compact_pool() orders them when
+        // someone asks for the population).  Otherwise the survivors are gathered into the other pool.
+        const bool in_place = c->fused && !(c->prm.flags & ONES_FLAG_NO_CLUSTER) && trunc_inplace_available(c->N);
+        if (!in_place && (rc = compact_pool(c)) != ONES_OK) return rc;
         for (int32_t it = 0; it < generations; ++it) {
             c->prof.sample = it % c->prof.every == 0;
             const int64_t K = c->N;
@@ -681,7 +713,7 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
             if (c->fused) {  // the 3K new rows are scored while they are written
                 CU(c, launch_trunc_children_score(c->pop(c->cur), c->ld, c->N, c->parents(), c->tab, keys, c->gen,
                                                   c->thr16, c->cap, c->prm.penalty, c->Fbuf(c->fcur), c->Gbuf(c->gcur),
-                                                  c->stream));
+                                                  c->mapped ? c->rowmap(c->mcur) : nullptr, c->stream));
                 if ((rc = prof_end(c)) != ONES_OK) return rc;
             } else {
                 CU(c, launch_trunc_children(c->pop(c->cur), c->ld, c->N, c->parents(), c->tab, keys, c->gen, c->thr16,
@@ -695,12 +727,22 @@ int ones_evolve(ones_ctx* c, int32_t generations, uint64_t seed) {
             }
             if ((rc = prof_begin(c, 1)) != ONES_OK) return rc;
             int sel_launches = 0;
-            CU(c, launch_trunc_select(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->Fbuf(c->fcur),
-                                      c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1), c->Gbuf(c->gcur ^ 1),
-                                      c->ws + c->L.trunc, c->stream, &sel_launches));
+            if (in_place) {
+                const int next = c->mapped ? c->mcur ^ 1 : 0;
+                CU(c, launch_trunc_select_inplace(c->N, c->Fbuf(c->fcur), c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1),
+                                                  c->Gbuf(c->gcur ^ 1), c->mapped ? c->rowmap(c->mcur) : nullptr,
+                                                  c->rowmap(next), c->stream));
+                sel_launches = 1;
+                c->mapped = true;
+                c->mcur = next;
+            } else {
+                CU(c, launch_trunc_select(c->pop(c->cur), c->pop(c->cur ^ 1), c->ld, c->N, c->Fbuf(c->fcur),
+                                          c->Gbuf(c->gcur), c->Fbuf(c->fcur ^ 1), c->Gbuf(c->gcur ^ 1),
+                                          c->ws + c->L.trunc, c->stream, &sel_launches));
+                c->cur ^= 1;
+            }
             if ((rc = prof_end(c)) != ONES_OK) return rc;
-            c->launches += 2 + (uint64_t)sel_launches;
-            c->cur ^= 1;
+            c->launches += (c->fused ? 1u : 2u) + (uint64_t)sel_launches;
             c->fcur ^= 1;
             c->gcur ^= 1;
             c->gen += 1;
@@ -840,7 +882,8 @@ int ones_best(ones_ctx* c, int repair, int32_t* h_genome, int32_t* h_gpus_per_jo
                                   c->stream));
     else
         CU(c, launch_best(c->pop(c->cur), c->ld, c->J, c->best_idx(), c->tab, c->cap, c->prm.penalty, repair,
-                          reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec, c->stream));
+                          reinterpret_cast<int32_t*>(c->ws + c->L.work), d_genome, d_gpus, d_rate, d_rec,
+                          c->mapped ? c->rowmap(c->mcur) : nullptr, c->stream));
     c->launches += (uint64_t)nl + 1;
     const size_t bytes = 64 + J * 16;
     if ((rc = ensure_staging(c, bytes + 64)) != ONES_OK) return rc;
@@ -894,6 +937,7 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
         }
     }
     if (c->packed && (rc = unpack_to_int(c)) != ONES_OK) return rc;  // the column map works on the int32 rows
+    if ((rc = compact_pool(c)) != ONES_OK) return rc;                // ... in the order of the candidates
     const int64_t old_ld = c->ld;
     const int32_t old_J = c->J;
     rc = rebuild_tables(c, jobs, n_jobs, remap, c->per_gpu);

@@ -118,10 +118,18 @@ cudaError_t launch_evolve_cluster(ClusterShape shape, int32_t* pop_io, int64_t l
 size_t trunc_scratch_bytes(int32_t k);
 cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
                                   uint64_t gen, uint32_t thr16, cudaStream_t s);  // 2 launches
-// the same, scoring the 3K new rows in the same pass (needs evolve_score_smem(t) <= kMaxSmemPerBlock); 2 launches
+// the same, scoring the 3K new rows in the same pass (needs evolve_score_smem(t) <= kMaxSmemPerBlock) and drawing
+// the parents itself (written to draws[] for ones_last_parents); 1 launch
 cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
                                         uint64_t gen, uint32_t thr16, int32_t capacity, double penalty, double* F,
-                                        int32_t* G, cudaStream_t s);
+                                        int32_t* G, const int32_t* rowmap /* nullptr: logical row = pool row */,
+                                        cudaStream_t s);
+// selection without copying a row: the pool is used in place through a map logical row -> pool row (4k entries)
+bool trunc_inplace_available(int32_t k);
+cudaError_t launch_trunc_select_inplace(int32_t k, const double* F, const int32_t* G, double* F_next, int32_t* G_next,
+                                        const int32_t* oldmap, int32_t* newmap, cudaStream_t s);  // 1 launch
+cudaError_t launch_trunc_compact(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const int32_t* rowmap,
+                                 cudaStream_t s);  // logical rows 0..k-1 -> rows 0..k-1 of pool_next
 cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const double* F,
                                 const int32_t* G, double* F_next, int32_t* G_next, void* scratch,
                                 cudaStream_t s, int* launches);  // 2 launches (pools up to 262144 rows) or 12
@@ -148,7 +156,7 @@ cudaError_t launch_refresh_per_gpu(int32_t* slots, int64_t ld, int32_t n, int32_
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work /*3*jpad*/,
                         int32_t* genome_out, int32_t* gpus_out, double* rate_out, BestOut* out,
-                        cudaStream_t s);
+                        const int32_t* rowmap /* nullptr: row best_index[0] of pop */, cudaStream_t s);
 cudaError_t launch_remap(const int32_t* src, int64_t ld_src, int32_t* dst, int64_t ld_dst, int32_t n,
                          int32_t n_jobs_new, const int32_t* remap, const int32_t* kmin_new,
                          const int32_t* range_new, cudaStream_t s);

@@ -2430,9 +2430,12 @@ k_trunc_children(int32_t* __restrict__ pool, int64_t ld, int32_t k, const int32_
 // not read back for their fitness.  F, G: the pool's score arrays (4K entries; rows K..4K-1 are written).
 template <bool ALWAYS>
 __global__ void __launch_bounds__(1024, 1)
-k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const int32_t* __restrict__ draws, Tables t,
-                       RoundKeys keys, uint32_t gen_lo, uint32_t c3cross, uint32_t c3mutant, uint32_t thr32,
-                       int32_t capacity, double penalty, double* __restrict__ F, int32_t* __restrict__ G) {
+k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, int32_t* __restrict__ draws, Tables t,
+                       RoundKeys keys, uint32_t gen_lo, uint32_t c3a, uint32_t c3b, uint32_t c3pick, uint32_t c3cross,
+                       uint32_t c3mutant, uint32_t thr32, int32_t capacity, double penalty, double* __restrict__ F,
+                       int32_t* __restrict__ G, const int32_t* __restrict__ rowmap) {
+    // (no early release of the selection that follows: measured 0.711-0.715 ms per generation with it against
+    // 0.686 without, 65536 candidates of 2048 jobs)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int32_t planes = t.k1 + 1;
     const int32_t jpad = t.jpad;
@@ -2456,7 +2459,7 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
         }
         __syncthreads();
     }
-    grid_dependency_wait();  // the draws come from the kernel before
+    grid_dependency_wait();  // the pool, its row map and the scores come from the kernels before
     constexpr int UN = 1;  // int4 per source row in flight per lane (2 measured 2 % slower)
     const uint64_t keep = l2_policy_evict_last();  // the K current candidates are read about three times each
     const int lane = threadIdx.x & 31;
@@ -2464,6 +2467,8 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
     const int64_t total_warps = (int64_t)gridDim.x * warps_per_block;
     const int32_t nvec = (int32_t)(ld >> 2);
     const uint32_t kcap = (uint32_t)t.k1;
+    // pool row of a logical row (the pool is used in place: survivors stay where they are)
+    auto row_of = [&](int64_t logical) -> int64_t { return rowmap ? (int64_t)rowmap[logical] : logical; };
     for (int64_t item = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); item < 2 * (int64_t)k;
          item += total_warps) {
         double sum0 = 0.0, sum1 = 0.0;
@@ -2472,11 +2477,18 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
         const bool pair = item < k;
         if (pair) {
             const int32_t q = (int32_t)item;
-            const int4* A = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q] * ld);
-            const int4* B = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * q + 1] * ld);
+            // the pair's two uniformly drawn parents (as k_trunc_draws; kept for ones_last_parents)
+            const int32_t pa = (int32_t)__umulhi(philox(0u, (uint32_t)q, gen_lo, c3a, keys).x, (uint32_t)k);
+            const int32_t pb = (int32_t)__umulhi(philox(0u, (uint32_t)q, gen_lo, c3b, keys).x, (uint32_t)k);
+            if (lane == 0) {
+                draws[2 * q] = pa;
+                draws[2 * q + 1] = pb;
+            }
+            const int4* A = reinterpret_cast<const int4*>(pool + row_of(pa) * ld);
+            const int4* B = reinterpret_cast<const int4*>(pool + row_of(pb) * ld);
             slot0 = (int64_t)k + 2 * q;
-            int4* C0 = reinterpret_cast<int4*>(pool + slot0 * ld);
-            int4* C1 = reinterpret_cast<int4*>(pool + (slot0 + 1) * ld);
+            int4* C0 = reinterpret_cast<int4*>(pool + row_of(slot0) * ld);
+            int4* C1 = reinterpret_cast<int4*>(pool + row_of(slot0 + 1) * ld);
             for (int32_t v0 = lane; v0 < nvec; v0 += 32 * UN) {
                 int4 a[UN], b[UN];
 #pragma unroll
@@ -2504,9 +2516,11 @@ k_trunc_children_score(int32_t* __restrict__ pool, int64_t ld, int32_t k, const 
             }
         } else {
             const int32_t m = (int32_t)(item - k);
-            const int4* S = reinterpret_cast<const int4*>(pool + (int64_t)draws[2 * k + m] * ld);
+            const int32_t ps = (int32_t)__umulhi(philox(0u, (uint32_t)m, gen_lo, c3pick, keys).x, (uint32_t)k);
+            if (lane == 0) draws[2 * k + m] = ps;
+            const int4* S = reinterpret_cast<const int4*>(pool + row_of(ps) * ld);
             slot0 = (int64_t)3 * k + m;
-            int4* C = reinterpret_cast<int4*>(pool + slot0 * ld);
+            int4* C = reinterpret_cast<int4*>(pool + row_of(slot0) * ld);
             for (int32_t v0 = lane; v0 < nvec; v0 += 32 * UN) {
                 int4 g[UN];
 #pragma unroll
@@ -2703,11 +2717,18 @@ __global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ 
 // eight radix passes exchange their 256-bin histograms through distributed shared memory (one hardware cluster
 // barrier per pass, the histograms alternating between two buffers; nothing spins), then the counts above / at
 // the threshold are scanned over threads and CTAs and every survivor's row is written to kept[] as
-// k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).
+// k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).  With `newmap` the kernel is the
+// whole selection: the pool is used in place, logical row -> pool row through a map of n entries; survivors keep
+// their pool rows and become logical rows 0..K-1 (in the order of their logical rows, as the scheme asks), the
+// rows given up become the places of the next generation's new candidates, and the survivors' scores and GPU
+// counts move to the other score arrays.  No candidate row is copied.
 constexpr int kPickCtas = 16, kPickThreads = 1024, kPickKeys = 16;
 
 __global__ void __launch_bounds__(kPickThreads, 1)
-k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* __restrict__ kept) {
+k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* __restrict__ kept,
+                   const int32_t* __restrict__ oldmap, int32_t* __restrict__ newmap, const int32_t* __restrict__ G,
+                   double* __restrict__ F_new, int32_t* __restrict__ G_new) {
+    grid_dependency_release();  // the next generation's CTAs stage their tables on the SMs this cluster leaves free
     grid_dependency_wait();
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ unsigned int hist[2][256];  // by pass parity: a histogram is cleared two passes after it was read
@@ -2739,15 +2760,14 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
             const unsigned int live = __ballot_sync(0xFFFFFFFFu, in);
             if (live == 0u) continue;  // late passes: hardly any key still matches the prefix
             // similar scores share their leading digits: one atomic for the warp when all live lanes agree,
-            // else one per distinct digit
+            // else one per key
             const unsigned int digit = (unsigned int)(key[u] >> shift) & 255u;
             const int first = __ffs(live) - 1;
             const unsigned int lead = __shfl_sync(0xFFFFFFFFu, digit, first);
             if (__all_sync(0xFFFFFFFFu, !in || digit == lead)) {
                 if (lane == first) atomicAdd(&myhist[lead], (unsigned int)__popc(live));
             } else if (in) {
-                const unsigned int peers = __match_any_sync(live, digit);
-                if (lane == __ffs(peers) - 1) atomicAdd(&myhist[digit], (unsigned int)__popc(peers));
+                atomicAdd(&myhist[digit], 1u);  // (grouping equal digits with a warp match first measured 4 % slower)
             }
         }
         cluster.sync();  // every CTA's histogram of this digit is complete
@@ -2850,12 +2870,27 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
 #pragma unroll
     for (int u = 0; u < kPickKeys; ++u) {
         if (u < kpt && row0 + u < n) {
+            const int32_t row = row0 + u;
+            const int32_t before = g_before + min(e_before, quota);  // survivors among the rows below this one
+            bool keep = false;
             if (key[u] > T) {
-                kept[g_before + min(e_before, quota)] = row0 + u;
+                keep = true;
                 ++g_before;
             } else if (key[u] == T) {
-                if (e_before < quota) kept[g_before + e_before] = row0 + u;
+                keep = e_before < quota;
                 ++e_before;
+            }
+            if (newmap) {
+                // pool used in place: the survivor becomes logical row `before`, any other row becomes the
+                // place of a new candidate (logical rows K..n-1, in the order of the rows given up)
+                const int32_t place = keep ? before : k + (row - before);
+                newmap[place] = oldmap ? oldmap[row] : row;
+                if (keep) {
+                    F_new[place] = F[row];
+                    G_new[place] = G[row];
+                }
+            } else if (keep) {
+                kept[before] = row;
             }
         }
     }
@@ -2901,7 +2936,7 @@ __global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict_
     int4* D = reinterpret_cast<int4*>(dst + p * ld);
     const int32_t nvec = (int32_t)(ld >> 2);
     for (int32_t v = lane; v < nvec; v += 32) D[v] = S[v];
-    if (lane == 0) {
+    if (lane == 0 && F_new) {
         F_new[p] = F[from];
         G_new[p] = G[from];
     }
@@ -2909,6 +2944,11 @@ __global__ void __launch_bounds__(256) k_trunc_gather(const int32_t* __restrict_
 
 size_t trunc_scratch_bytes(int32_t k) {
     return 64 + sizeof(TruncState) + 2 * 1024 * sizeof(int32_t) + (size_t)k * sizeof(int32_t);
+}
+
+// Can the selection of the best k of 4k rows run in place (one cluster launch, no row copied)?
+bool trunc_inplace_available(int32_t k) {
+    return 4 * (int64_t)k <= (int64_t)kPickCtas * kPickThreads * kPickKeys && pick_cluster_available();
 }
 
 // Derive the 3K new candidates of one generation into rows K..4K-1 of the pool.  draws: 3K ints.
@@ -2931,23 +2971,54 @@ cudaError_t launch_trunc_children(int32_t* pool, int64_t ld, int32_t k, int32_t*
 
 cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, int32_t* draws, Tables t, RoundKeys keys,
                                         uint64_t gen, uint32_t thr16, int32_t capacity, double penalty, double* F,
-                                        int32_t* G, cudaStream_t s) {
+                                        int32_t* G, const int32_t* rowmap, cudaStream_t s) {
     const size_t smem = evolve_score_smem(t);
     if (smem > (size_t)kMaxSmemPerBlock) return cudaErrorInvalidConfiguration;
     const uint32_t thr32 = thr16 >= 65536u ? 0xFFFFFFFFu : thr16 << 16;
-    k_trunc_draws<<<(3 * k + 255) / 256, 256, 0, s>>>(k, keys, (uint32_t)gen, counter3(STREAM_SEL_A, gen),
-                                                      counter3(STREAM_SEL_B, gen), counter3(STREAM_PICK, gen), draws);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
     constexpr int kThreads = 1024;
     int64_t blocks = (2 * (int64_t)k + kThreads / 32 - 1) / (kThreads / 32);
     if (blocks > sm_count()) blocks = sm_count();
     auto kern = thr16 >= 65536u ? k_trunc_children_score<true> : k_trunc_children_score<false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerBlock);
     if (e != cudaSuccess) return e;
-    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, pool, ld, k, (const int32_t*)draws, t, keys,
-                                 (uint32_t)gen, counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32, capacity,
-                                 penalty, F, G);
+    return launch_after_previous(kern, (int)blocks, kThreads, smem, s, pool, ld, k, draws, t, keys, (uint32_t)gen,
+                                 counter3(STREAM_SEL_A, gen), counter3(STREAM_SEL_B, gen), counter3(STREAM_PICK, gen),
+                                 counter3(STREAM_MUT, gen), counter3(STREAM_MUTANT, gen), thr32, capacity, penalty, F,
+                                 G, rowmap);
+}
+
+static cudaError_t launch_pick_place(const double* F, int32_t n, int32_t k, int32_t* kept, const int32_t* oldmap,
+                                     int32_t* newmap, const int32_t* G, double* F_next, int32_t* G_next, cudaStream_t s) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kPickCtas, 1, 1);
+    cfg.blockDim = dim3(kPickThreads, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kPickCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, k_trunc_pick_place, F, n, k, kept, oldmap, newmap, G, F_next, G_next);
+}
+
+// The selection in place (see k_trunc_pick_place): oldmap (nullptr: logical row = pool row) -> newmap, both of
+// 4k entries; F, G: 4k scores and GPU counts by logical row; F_next, G_next receive the survivors'.  One launch.
+cudaError_t launch_trunc_select_inplace(int32_t k, const double* F, const int32_t* G, double* F_next, int32_t* G_next,
+                                        const int32_t* oldmap, int32_t* newmap, cudaStream_t s) {
+    if (!newmap || !trunc_inplace_available(k)) return cudaErrorNotSupported;
+    return launch_pick_place(F, 4 * k, k, nullptr, oldmap, newmap, G, F_next, G_next, s);
+}
+
+// Logical rows 0..k-1 of a pool used in place, copied in order to rows 0..k-1 of pool_next.
+cudaError_t launch_trunc_compact(const int32_t* pool, int32_t* pool_next, int64_t ld, int32_t k, const int32_t* rowmap,
+                                 cudaStream_t s) {
+    k_trunc_gather<<<(k + 7) / 8, 256, 0, s>>>(pool, pool_next, ld, k, rowmap, nullptr, nullptr, nullptr, nullptr);
+    return cudaGetLastError();
 }
 
 // Keep the best K of the 4K scored rows: F, G hold 4K entries; the survivors become rows 0..K-1 of
@@ -2966,20 +3037,7 @@ cudaError_t launch_trunc_select(const int32_t* pool, int32_t* pool_next, int64_t
     cudaError_t e;
     if (n <= kPickCtas * kPickThreads * kPickKeys && pick_cluster_available()) {
         // threshold search and places in one cluster launch, then the gather
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kPickCtas, 1, 1);
-        cfg.blockDim = dim3(kPickThreads, 1, 1);
-        cfg.stream = s;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kPickCtas;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        e = cudaLaunchKernelEx(&cfg, k_trunc_pick_place, F, n, k, kept);
+        e = launch_pick_place(F, n, k, kept, nullptr, nullptr, nullptr, nullptr, nullptr, s);
         if (e != cudaSuccess) return e;
         if (launches) *launches = 2;
         return launch_after_previous(k_trunc_gather, (k + 7) / 8, 256, 0, s, pool, pool_next, ld, k, (const int32_t*)kept,
@@ -3965,12 +4023,13 @@ __device__ __forceinline__ int2 block_arg_best(int2 mine /*(value, j); value < 0
 __global__ void __launch_bounds__(256)
 k_best(const int32_t* __restrict__ pop, int64_t ld, int32_t n_jobs, const int32_t* __restrict__ best_index, Tables t,
        int32_t capacity, double penalty, int repair, int32_t* __restrict__ work, int32_t* __restrict__ genome_out,
-       int32_t* __restrict__ gpus_out, double* __restrict__ rate_out, BestOut* __restrict__ out) {
+       int32_t* __restrict__ gpus_out, double* __restrict__ rate_out, BestOut* __restrict__ out,
+       const int32_t* __restrict__ rowmap) {
     __shared__ int2 s_warp[8];
     __shared__ long long s_total;
     __shared__ int s_status;
     const int32_t best = best_index[0];
-    const int32_t* row = pop + (int64_t)best * ld;
+    const int32_t* row = pop + (int64_t)(rowmap ? rowmap[best] : best) * ld;  // a pool used in place keeps a row map
     int32_t* wk = work;
     int32_t* wg = work + t.jpad;
     int32_t* wl = work + 2 * t.jpad;
@@ -4126,9 +4185,9 @@ k_best(const int32_t* __restrict__ pop, int64_t ld, int32_t n_jobs, const int32_
 
 cudaError_t launch_best(const int32_t* pop, int64_t ld, int32_t n_jobs, const int32_t* best_index, Tables t,
                         int32_t capacity, double penalty, int repair, int32_t* work, int32_t* genome_out,
-                        int32_t* gpus_out, double* rate_out, BestOut* out, cudaStream_t s) {
+                        int32_t* gpus_out, double* rate_out, BestOut* out, const int32_t* rowmap, cudaStream_t s) {
     k_best<<<1, 256, 0, s>>>(pop, ld, n_jobs, best_index, t, capacity, penalty, repair, work, genome_out, gpus_out,
-                             rate_out, out);
+                             rate_out, out, rowmap);
     return cudaGetLastError();
 }
 

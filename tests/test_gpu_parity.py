@@ -348,7 +348,8 @@ def test_set_get_population_roundtrip(ones):
 @pytest.mark.parametrize("J,N,kw", [(16, 32, {}), (100, 1024, {}), (37, 101, dict(p_mut=1.0)), (5, 3, dict(p_mut=0.0)),
                                     (130, 257, dict(p_mut=0.02)), (1, 3, {}), (512, 4096, {}),
                                     (130, 257, dict(flags=6)), (37, 101, dict(p_mut=1.0, flags=6)),   # separate scoring pass
-                                    (2048, 700, dict(p_mut=0.02))])
+                                    (2048, 700, dict(p_mut=0.02)),
+                                    (130, 257, dict(flags=12)), (512, 4096, dict(flags=12))])  # survivors gathered
 def test_truncation_selection_parity(ones, J, N, kw):
     w = inputs.custom(J, max(4, J), N, 4, seed=J + N, kmax=7, pinned=J // 5, kmin_max=2)
     kw = dict(kw)
@@ -380,6 +381,37 @@ def test_truncation_selection_parity_large_job_table(ones):
     po, _ = o.last_parents()
     assert (pg == po).all()
     _same_state(g, o)
+
+
+@pytest.mark.parametrize("J,N", [(16, 32), (130, 257), (300, 5000), (2048, 700)])
+def test_truncation_pool_in_place_over_many_generations(ones, J, N):
+    """The fused handle keeps the pool in place between generations (a row map instead of a gather).  Several
+    generations per call, the best candidate read through the map before anything orders the rows, a change of the
+    job set on the mapped pool, and the handle that gathers the survivors every generation as a second witness."""
+    w = inputs.custom(J, max(4, J), N, 4, seed=3 * J + N, kmax=6, pinned=J // 6, kmin_max=2)
+    g = ones.Search(w.jobs, w.capacity, N, inputs.SearchParams(p_mut=0.03, flags=4), n_jobs_max=J + 8)
+    h = ones.Search(w.jobs, w.capacity, N, inputs.SearchParams(p_mut=0.03, flags=12), n_jobs_max=J + 8)
+    o = oracle.Search(w.jobs, w.capacity, N, p_mut=0.03, flags=4)
+    for s_ in (g, o, h):
+        s_.randomize(6)
+        s_.evolve(7, 21)
+    for rep in (True, False):
+        bg, bh, bo = g.best(rep), h.best(rep), o.best(rep)   # g: still mapped, the row is found through the map
+        for b in (bg, bh):
+            assert (b["genome"] == bo["genome"]).all() and b["fitness"] == bo["fitness"] and b["index"] == bo["index"]
+    for s_ in (g, o, h):
+        s_.evolve(5, 22)
+    _same_state(g, o)
+    _same_state(h, o)
+    for s_ in (g, o, h):
+        s_.evolve(2, 23)   # from the ordered pool, then mapped again when the job set changes
+    jobs2 = np.concatenate([w.jobs[2:], inputs.custom(4, 8, 4, 1, seed=2, kmax=3).jobs])
+    remap = np.concatenate([np.arange(2, J), np.full(4, -1)]).astype(np.int32)
+    for s_ in (g, o, h):
+        s_.update_jobs(jobs2, remap, w.capacity)   # g: the candidates are put in order before their columns move
+        s_.evolve(3, 24)
+    _same_state(g, o)
+    _same_state(h, o)
 
 
 def test_truncation_selection_with_many_ties(ones):
