@@ -2713,17 +2713,23 @@ __global__ void __launch_bounds__(256) k_trunc_place(const double* __restrict__ 
 }
 
 // The whole threshold search and the survivors' places in ONE launch of one thread-block cluster, for pools of
-// up to 16 x 1024 x 16 rows: every thread keeps the keys of its (up to 16) consecutive rows in registers, the
-// eight radix passes exchange their 256-bin histograms through distributed shared memory (one hardware cluster
-// barrier per pass, the histograms alternating between two buffers; nothing spins), then the counts above / at
-// the threshold are scanned over threads and CTAs and every survivor's row is written to kept[] as
-// k_trunc_place does.  Replaces 11 launches (8 passes, count, scan, place).  With `newmap` the kernel is the
-// whole selection: the pool is used in place, logical row -> pool row through a map of n entries; survivors keep
-// their pool rows and become logical rows 0..K-1 (in the order of their logical rows, as the scheme asks), the
-// rows given up become the places of the next generation's new candidates, and the survivors' scores and GPU
-// counts move to the other score arrays.  No candidate row is copied.
+// up to 16 x 1024 x 16 rows.  Every warp owns a contiguous run of 32 x kpt rows and every thread keeps the keys of
+// its (up to 16) rows, 32 apart, in registers, so that scores, GPU counts and the row map are read and written by
+// whole warps side by side.  The eight radix passes exchange their 256-bin histograms through distributed shared
+// memory (one hardware cluster barrier per pass, the histograms alternating between two buffers; nothing spins);
+// a thread remembers which of its keys still match the prefix, and a pass visits only the slots where some lane
+// of the warp has one.  Then the counts above / at the threshold are scanned over warps and CTAs (inside a warp a
+// ballot gives every row its rank) and every survivor's row is written to kept[] as k_trunc_place does.
+// Replaces 11 launches (8 passes, count, scan, place).  With `newmap` the kernel is the whole selection: the pool
+// is used in place, logical row -> pool row through a map of n entries; survivors keep their pool rows and become
+// logical rows 0..K-1 (in the order of their logical rows, as the scheme asks), the rows given up become the
+// places of the next generation's new candidates, and the survivors' scores and GPU counts move to the other
+// score arrays.  No candidate row is copied.
+// KEYS: rows a thread can hold (1, 4 or 16; the launch takes the smallest that covers the pool, so that small
+// pools do not pay for the unrolled slots of large ones).
 constexpr int kPickCtas = 16, kPickThreads = 1024, kPickKeys = 16;
 
+template <int KEYS, int NCTA>
 __global__ void __launch_bounds__(kPickThreads, 1)
 k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* __restrict__ kept,
                    const int32_t* __restrict__ oldmap, int32_t* __restrict__ newmap, const int32_t* __restrict__ G,
@@ -2731,6 +2737,10 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     grid_dependency_release();  // the next generation's CTAs stage their tables on the SMs this cluster leaves free
     grid_dependency_wait();
     cg::cluster_group cluster = cg::this_cluster();
+    auto sync_all = [&]() {  // every CTA of the launch
+        if (NCTA == 1) __syncthreads();
+        else cluster.sync();
+    };
     __shared__ unsigned int hist[2][256];  // by pass parity: a histogram is cleared two passes after it was read
     __shared__ unsigned int tot[256];
     __shared__ unsigned long long s_prefix;
@@ -2739,12 +2749,36 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     __shared__ int32_t s_cta[2];  // this CTA's counts above / at the threshold
     const unsigned int rank = cluster.block_rank();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // every thread owns `kpt` consecutive rows, so that all CTAs share the work whatever the pool's size
-    const int32_t kpt = (n + kPickCtas * kPickThreads - 1) / (kPickCtas * kPickThreads);
-    const int32_t row0 = ((int32_t)rank * kPickThreads + (int32_t)threadIdx.x) * kpt;
-    unsigned long long key[kPickKeys];
+    // rows per thread, so that all CTAs share the work whatever the pool's size; the warp's rows are
+    // wbase ... wbase + 32 * kpt - 1, slot u of lane l is row wbase + 32 u + l
+    constexpr int32_t ncta = NCTA;  // 16, or 1 for small pools (the passes then cost block barriers only)
+    const int32_t kpt = (n + ncta * kPickThreads - 1) / (ncta * kPickThreads);
+    const int32_t wbase = ((int32_t)rank * (kPickThreads / 32) + warp) * 32 * kpt;
+    unsigned long long key[KEYS];
+    unsigned int alive = 0u;  // bit u: key u is a row of the pool and still matches the prefix
+    // the scores were written throughout the kernel before and have mostly left L2: ask for all of this warp's
+    // lines at once (one lane per 128 bytes), and for what the last step reads of the map and the GPU counts
+    for (int32_t i = lane; i < kpt * 2; i += 32) {
+        const int32_t row = wbase + 16 * i;
+        if (row < n) {
+            l2_prefetch(reinterpret_cast<const unsigned char*>(F + row));
+            if (newmap && !(i & 1)) {
+                l2_prefetch(reinterpret_cast<const unsigned char*>(G + row));
+                if (oldmap) l2_prefetch(reinterpret_cast<const unsigned char*>(oldmap + row));
+            }
+        }
+    }
 #pragma unroll
-    for (int u = 0; u < kPickKeys; ++u) key[u] = (u < kpt && row0 + u < n) ? score_key(F[row0 + u]) : 0ull;
+    for (int u = 0; u < KEYS; ++u) {  // all the loads first, so that they are in flight together
+        const int32_t row = wbase + 32 * u + lane;
+        const bool have = u < kpt && row < n;
+        key[u] = have ? (unsigned long long)__double_as_longlong(F[row]) : 0ull;
+        alive |= have ? 1u << u : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < KEYS; ++u)
+        key[u] = ((alive >> u) & 1u) ? score_key(__longlong_as_double((long long)key[u])) : 0ull;
+    const unsigned int rows_here = alive;
     unsigned long long prefix = 0ull;
     int32_t remaining = k;
     for (int pass = 0; pass < 8; ++pass) {
@@ -2753,28 +2787,37 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
         __syncthreads();
         const int shift = 56 - 8 * pass;
         const unsigned long long mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
+        const unsigned int warp_alive = __reduce_or_sync(0xFFFFFFFFu, alive);
+        unsigned int run_digit = 0u, run_count = 0u;  // (uniform) slots in a row whose live keys all share one digit
 #pragma unroll
-        for (int u = 0; u < kPickKeys; ++u) {
-            if (u >= kpt) break;  // uniform
-            const bool in = row0 + u < n && (key[u] & mask) == prefix;
+        for (int u = 0; u < KEYS; ++u) {
+            if (!((warp_alive >> u) & 1u)) continue;  // uniform: no lane of the warp has a matching key in this slot
+            const bool in = ((alive >> u) & 1u) && (key[u] & mask) == prefix;
+            if (!in) alive &= ~(1u << u);
             const unsigned int live = __ballot_sync(0xFFFFFFFFu, in);
-            if (live == 0u) continue;  // late passes: hardly any key still matches the prefix
-            // similar scores share their leading digits: one atomic for the warp when all live lanes agree,
-            // else one per key
+            if (live == 0u) continue;
+            // similar scores share their leading digits: when all live lanes of a slot agree the warp counts in a
+            // register and adds once per run of such slots, else one atomic per key (grouping equal digits with a
+            // warp match first measured 4 % slower)
             const unsigned int digit = (unsigned int)(key[u] >> shift) & 255u;
-            const int first = __ffs(live) - 1;
-            const unsigned int lead = __shfl_sync(0xFFFFFFFFu, digit, first);
+            const unsigned int lead = __shfl_sync(0xFFFFFFFFu, digit, __ffs(live) - 1);
             if (__all_sync(0xFFFFFFFFu, !in || digit == lead)) {
-                if (lane == first) atomicAdd(&myhist[lead], (unsigned int)__popc(live));
+                if (lead != run_digit && run_count) {
+                    if (lane == 0) atomicAdd(&myhist[run_digit], run_count);
+                    run_count = 0u;
+                }
+                run_digit = lead;
+                run_count += (unsigned int)__popc(live);
             } else if (in) {
-                atomicAdd(&myhist[digit], 1u);  // (grouping equal digits with a warp match first measured 4 % slower)
+                atomicAdd(&myhist[digit], 1u);
             }
         }
-        cluster.sync();  // every CTA's histogram of this digit is complete
+        if (run_count && lane == 0) atomicAdd(&myhist[run_digit], run_count);
+        sync_all();  // every CTA's histogram of this digit is complete
         if (threadIdx.x < 256) {
             unsigned int sum = 0u;
 #pragma unroll
-            for (unsigned int r = 0; r < (unsigned int)kPickCtas; ++r) sum += *cluster.map_shared_rank(&myhist[threadIdx.x], r);
+            for (unsigned int r = 0; r < (unsigned int)NCTA; ++r) sum += *cluster.map_shared_rank(&myhist[threadIdx.x], r);
             tot[threadIdx.x] = sum;
         }
         __syncthreads();
@@ -2819,82 +2862,99 @@ k_trunc_pick_place(const double* __restrict__ F, int32_t n, int32_t k, int32_t* 
     // prefix = key of the k-th best, remaining = how many rows with exactly that key survive (lowest rows first)
     const unsigned long long T = prefix;
     const int32_t quota = remaining;
-    int32_t gt = 0, eq = 0;
+    // counts above / at the threshold: per warp by ballots, then an exclusive scan over the CTA's warps (rows ascend
+    // with the warp index), then over the CTAs
+    int32_t wg = 0, we = 0;
 #pragma unroll
-    for (int u = 0; u < kPickKeys; ++u) {
-        if (u < kpt && row0 + u < n) {
-            gt += key[u] > T;
-            eq += key[u] == T;
-        }
+    for (int u = 0; u < KEYS; ++u) {
+        if (u >= kpt) break;  // uniform
+        const bool have = (rows_here >> u) & 1u;
+        wg += __popc(__ballot_sync(0xFFFFFFFFu, have && key[u] > T));
+        we += __popc(__ballot_sync(0xFFFFFFFFu, have && key[u] == T));
     }
-    // exclusive scan over the CTA's threads (rows ascend with the thread index), then over the CTAs
-    int32_t sg = gt, se = eq;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int32_t a = __shfl_up_sync(0xFFFFFFFFu, sg, off), b = __shfl_up_sync(0xFFFFFFFFu, se, off);
-        if (lane >= off) {
-            sg += a;
-            se += b;
-        }
-    }
-    if (lane == 31) {
-        s_warp_g[warp] = sg;
-        s_warp_e[warp] = se;
+    if (lane == 0) {
+        s_warp_g[warp] = wg;
+        s_warp_e[warp] = we;
     }
     __syncthreads();
     if (warp == 0) {
-        int32_t wg = s_warp_g[lane], we = s_warp_e[lane];
+        int32_t sg = s_warp_g[lane], se = s_warp_e[lane];
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const int32_t a = __shfl_up_sync(0xFFFFFFFFu, wg, off), b = __shfl_up_sync(0xFFFFFFFFu, we, off);
+            const int32_t a = __shfl_up_sync(0xFFFFFFFFu, sg, off), b = __shfl_up_sync(0xFFFFFFFFu, se, off);
             if (lane >= off) {
-                wg += a;
-                we += b;
+                sg += a;
+                se += b;
             }
         }
-        s_warp_g[lane] = wg;  // inclusive over warps
-        s_warp_e[lane] = we;
+        s_warp_g[lane] = sg;  // inclusive over warps
+        s_warp_e[lane] = se;
         if (lane == 31) {
-            s_cta[0] = wg;
-            s_cta[1] = we;
+            s_cta[0] = sg;
+            s_cta[1] = se;
         }
     }
-    cluster.sync();  // every CTA's totals are in place
-    int32_t g_before = sg - gt + (warp > 0 ? s_warp_g[warp - 1] : 0);
-    int32_t e_before = se - eq + (warp > 0 ? s_warp_e[warp - 1] : 0);
-    for (unsigned int r = 0; r < rank; ++r) {
-        const int32_t* other = cluster.map_shared_rank(s_cta, r);
-        g_before += other[0];
-        e_before += other[1];
-    }
+    sync_all();  // every CTA's totals are in place
+    int32_t g_before = warp > 0 ? s_warp_g[warp - 1] : 0;  // rows of the warps (then CTAs) below this warp
+    int32_t e_before = warp > 0 ? s_warp_e[warp - 1] : 0;
 #pragma unroll
-    for (int u = 0; u < kPickKeys; ++u) {
-        if (u < kpt && row0 + u < n) {
-            const int32_t row = row0 + u;
-            const int32_t before = g_before + min(e_before, quota);  // survivors among the rows below this one
-            bool keep = false;
-            if (key[u] > T) {
-                keep = true;
-                ++g_before;
-            } else if (key[u] == T) {
-                keep = e_before < quota;
-                ++e_before;
-            }
-            if (newmap) {
-                // pool used in place: the survivor becomes logical row `before`, any other row becomes the
-                // place of a new candidate (logical rows K..n-1, in the order of the rows given up)
-                const int32_t place = keep ? before : k + (row - before);
-                newmap[place] = oldmap ? oldmap[row] : row;
-                if (keep) {
-                    F_new[place] = F[row];
-                    G_new[place] = G[row];
-                }
-            } else if (keep) {
-                kept[before] = row;
-            }
+    for (unsigned int r = 0; r < (unsigned int)NCTA; ++r) {  // unrolled: the remote reads are all in flight at once
+        if (r < rank) {
+            const int32_t* other = cluster.map_shared_rank(s_cta, r);
+            g_before += other[0];
+            e_before += other[1];
         }
     }
-    cluster.sync();  // no CTA leaves while a neighbour may still read its totals
+    const unsigned int below = (1u << lane) - 1u;
+    // eight slots at a time: what the slots read of the map and of the GPU counts is loaded first, so that a warp
+    // waits for memory twice and not once per slot; a score is taken back from its key where the key has an
+    // inverse (not for NaN and zero, whose sign or payload the key does not keep)
+    constexpr int BATCH = KEYS < 8 ? KEYS : 8;
+#pragma unroll
+    for (int h = 0; h < KEYS; h += BATCH) {
+        if (h >= kpt) break;  // uniform
+        int32_t from[BATCH], gpus[BATCH];
+#pragma unroll
+        for (int v = 0; v < BATCH; ++v) {
+            const int u = h + v;
+            const int32_t row = wbase + 32 * u + lane;
+            const bool have = (rows_here >> u) & 1u;
+            from[v] = (newmap && oldmap && have) ? oldmap[row] : row;
+            gpus[v] = (newmap && have && key[u] >= T) ? G[row] : 0;
+        }
+#pragma unroll
+        for (int v = 0; v < BATCH; ++v) {
+            const int u = h + v;
+            if (u >= kpt) break;  // uniform
+            const bool have = (rows_here >> u) & 1u;
+            const bool gt = have && key[u] > T, eq = have && key[u] == T;
+            const unsigned int bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
+            if (have) {
+                const int32_t row = wbase + 32 * u + lane;
+                const int32_t eb = e_before + __popc(be & below);
+                const int32_t before = g_before + __popc(bg & below) + min(eb, quota);  // survivors among the rows below
+                const bool keep = gt || (eq && eb < quota);
+                if (newmap) {
+                    // pool used in place: the survivor becomes logical row `before`, any other row becomes the
+                    // place of a new candidate (logical rows K..n-1, in the order of the rows given up)
+                    const int32_t place = keep ? before : k + (row - before);
+                    newmap[place] = from[v];
+                    if (keep) {
+                        const unsigned long long kk = key[u];
+                        const bool plain = kk != 0ull && kk != 0x8000000000000000ull;
+                        const unsigned long long bits = (kk >> 63) ? kk ^ 0x8000000000000000ull : ~kk;
+                        F_new[place] = plain ? __longlong_as_double((long long)bits) : F[row];
+                        G_new[place] = gpus[v];
+                    }
+                } else if (keep) {
+                    kept[before] = row;
+                }
+            }
+            g_before += __popc(bg);
+            e_before += __popc(be);
+        }
+    }
+    sync_all();  // no CTA leaves while a neighbour may still read its totals
 }
 
 // Can the device host that cluster (asked once per device)?
@@ -2914,8 +2974,10 @@ static bool pick_cluster_available() {
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        bool ok = cudaFuncSetAttribute(k_trunc_pick_place, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
-                  cudaOccupancyMaxActiveClusters(&clusters, k_trunc_pick_place, &cfg) == cudaSuccess && clusters >= 1;
+        bool ok = cudaFuncSetAttribute(k_trunc_pick_place<1, kPickCtas>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaFuncSetAttribute(k_trunc_pick_place<4, kPickCtas>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaFuncSetAttribute(k_trunc_pick_place<kPickKeys, kPickCtas>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                  cudaOccupancyMaxActiveClusters(&clusters, k_trunc_pick_place<kPickKeys, kPickCtas>, &cfg) == cudaSuccess && clusters >= 1;
         if (!ok) (void)cudaGetLastError();
         state[dev] = ok ? 1 : 2;
     }
@@ -2991,19 +3053,27 @@ cudaError_t launch_trunc_children_score(int32_t* pool, int64_t ld, int32_t k, in
 static cudaError_t launch_pick_place(const double* F, int32_t n, int32_t k, int32_t* kept, const int32_t* oldmap,
                                      int32_t* newmap, const int32_t* G, double* F_next, int32_t* G_next, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kPickCtas, 1, 1);
+    // pools of up to 4096 rows: one CTA with up to four rows per thread (the eight passes then cost block barriers
+    // only: 27 -> 19 us per selection at 4096 rows, 25 -> 12.5 at 128; with 16 rows per thread one CTA took 61 us
+    // where the cluster takes 25); larger ones: the 16-CTA cluster
+    const int ncta = n <= kPickThreads * 4 ? 1 : kPickCtas;
+    cfg.gridDim = dim3(ncta, 1, 1);
     cfg.blockDim = dim3(kPickThreads, 1, 1);
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kPickCtas;
+    attr[0].val.clusterDim.x = ncta;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, k_trunc_pick_place, F, n, k, kept, oldmap, newmap, G, F_next, G_next);
+    const int32_t kpt = (n + ncta * kPickThreads - 1) / (ncta * kPickThreads);
+    auto kern = ncta == 1 ? (kpt <= 1 ? k_trunc_pick_place<1, 1> : k_trunc_pick_place<4, 1>)
+                          : kpt <= 1 ? k_trunc_pick_place<1, kPickCtas>
+                                     : kpt <= 4 ? k_trunc_pick_place<4, kPickCtas> : k_trunc_pick_place<kPickKeys, kPickCtas>;
+    return cudaLaunchKernelEx(&cfg, kern, F, n, k, kept, oldmap, newmap, G, F_next, G_next);
 }
 
 // The selection in place (see k_trunc_pick_place): oldmap (nullptr: logical row = pool row) -> newmap, both of
