@@ -89,7 +89,9 @@ typedef struct {
 
 /* Small populations normally run all generations of a ones_evolve call in one launch of one
  * thread-block cluster, with the population in the cluster's shared memory.  This flag keeps the
- * launch-per-generation sequence instead (same results). */
+ * launch-per-generation sequence instead (same results).  With ONES_FLAG_TRUNCATION the flag keeps the
+ * survivors' gather into the second pool after every generation, where the default uses the pool in place
+ * through a row map and orders the candidates only when they are read (same results). */
 #define ONES_FLAG_NO_CLUSTER 8u
 
 /* The paper's own genome (Eq. 1-2, Fig. 1): a candidate is one int32 per GPU of the cluster holding the
