@@ -2060,17 +2060,23 @@ cudaError_t launch_evolve_score(const int32_t* src, int32_t* dst, int64_t ld, in
 // ---------------------------------------------------------------------------------------------
 // Small populations: all generations of one ones_evolve call in ONE launch of one thread-block
 // cluster.  Both population buffers, the scores and the model tables live in the shared memory of
-// the cluster's CTAs (CTA r owns rows r*rows_per_cta ...); parents and scores of other CTAs are read,
-// and children that belong to a neighbour written, through distributed shared memory; each CTA copies
-// all scores into its own shared memory once per generation for the tournaments and the elites.  One
-// hardware cluster barrier per generation replaces the kernel boundaries; nothing spins.  Lanes are grouped so that one group of `gs` lanes (gs = int4 per
+// the cluster's CTAs (CTA r owns rows r*rows_per_cta ...); parents of other CTAs are read, and children
+// that belong to a neighbour written, through distributed shared memory.  Every CTA keeps all scores of
+// both populations: before the generation's cluster barrier a CTA stores the scores of the children it
+// produced into every CTA's copy, so nothing is fetched after the barrier.  The elites of a new population
+// are its rows 0..E-1 (the old elites, copied) or children that beat the old E-th best: a CTA lists those
+// children (at most kClusterCand per generation, else every CTA falls back to the search over all
+// scores), the lists travel with the scores, and one warp merges them.  One hardware cluster barrier per
+// generation replaces the kernel boundaries; nothing spins.  Lanes are grouped so that one group of `gs` lanes (gs = int4 per
 // row rounded up to a power of two, at most 32) handles one pair of children: with 6 jobs a warp
 // runs 16 pairs at once.  Draws, operators, summation order and elites are those of the other paths.
 // ---------------------------------------------------------------------------------------------
 namespace cg = cooperative_groups;
 
+constexpr int kClusterCand = 8;  // children of one CTA and generation that may enter the elites without the full search
+
 struct ClusterSmem {  // byte offsets into dynamic shared memory
-    size_t X, F0, F1, Fall, G16, pop0, pop1, Gc, kmin, range, elit, total;
+    size_t X, Fall0, Fall1, G16, pop0, pop1, Gc0, Gc1, kmin, range, elit, cand_cnt, cand_in, total;
 };
 
 __host__ __device__ inline ClusterSmem cluster_smem(int32_t planes, int32_t jpad, int64_t ld, int32_t rows,
@@ -2080,16 +2086,18 @@ __host__ __device__ inline ClusterSmem cluster_smem(int32_t planes, int32_t jpad
     const size_t e = (size_t)(elitism > 0 ? elitism : 1);
 #define ONES_TAKE(field, bytes) m.field = at; at = (at + (size_t)(bytes) + 15) & ~(size_t)15
     ONES_TAKE(X, (size_t)planes * jpad * 8);
-    ONES_TAKE(F0, (size_t)rows * 8);
-    ONES_TAKE(F1, (size_t)rows * 8);
-    ONES_TAKE(Fall, (size_t)n * 8);
+    ONES_TAKE(Fall0, (size_t)n * 8);  // every candidate's score, population 0 / 1
+    ONES_TAKE(Fall1, (size_t)n * 8);
     ONES_TAKE(pop0, (size_t)rows * ld * 4);
     ONES_TAKE(pop1, (size_t)rows * ld * 4);
-    ONES_TAKE(Gc, (size_t)rows * 4);
+    ONES_TAKE(Gc0, (size_t)rows * 4);  // GPU counts of this CTA's rows, population 0 / 1
+    ONES_TAKE(Gc1, (size_t)rows * 4);
     ONES_TAKE(kmin, (size_t)jpad * 4);
     ONES_TAKE(range, (size_t)jpad * 4);
     ONES_TAKE(elit, e * 4);
     ONES_TAKE(G16, (size_t)planes * jpad * 2);
+    ONES_TAKE(cand_cnt, (size_t)2 * 16 * 4);                   // [population][producing CTA]
+    ONES_TAKE(cand_in, (size_t)2 * 16 * kClusterCand * 16);    // [population][producing CTA][kClusterCand] records
 #undef ONES_TAKE
     m.total = (at + 15) & ~(size_t)15;
     return m;
@@ -2105,6 +2113,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Rec s_warp[64];
     __shared__ Rec s_top[4];
+    __shared__ int s_full;  // the elites of this generation need the search over all scores
     cg::cluster_group cluster = cg::this_cluster();
     const int32_t C = (int32_t)cluster.num_blocks(), me = (int32_t)cluster.block_rank();
     const int32_t planes = t.k1 + 1, jpad = t.jpad;
@@ -2112,12 +2121,13 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
     const ClusterSmem m = cluster_smem(planes, jpad, ld, rows_per_cta, elitism, n);
     double* sX = reinterpret_cast<double*>(smem_raw + m.X);
     uint16_t* sG = reinterpret_cast<uint16_t*>(smem_raw + m.G16);
-    double* sF[2] = {reinterpret_cast<double*>(smem_raw + m.F0), reinterpret_cast<double*>(smem_raw + m.F1)};
+    double* sFall[2] = {reinterpret_cast<double*>(smem_raw + m.Fall0), reinterpret_cast<double*>(smem_raw + m.Fall1)};
+    int32_t* sCandCnt = reinterpret_cast<int32_t*>(smem_raw + m.cand_cnt);
+    Rec* sCandIn = reinterpret_cast<Rec*>(smem_raw + m.cand_in);
     int32_t* sPop[2] = {reinterpret_cast<int32_t*>(smem_raw + m.pop0), reinterpret_cast<int32_t*>(smem_raw + m.pop1)};
-    int32_t* sGc = reinterpret_cast<int32_t*>(smem_raw + m.Gc);
+    int32_t* sGc[2] = {reinterpret_cast<int32_t*>(smem_raw + m.Gc0), reinterpret_cast<int32_t*>(smem_raw + m.Gc1)};
     int4* sKmin = reinterpret_cast<int4*>(smem_raw + m.kmin);
     int4* sRange = reinterpret_cast<int4*>(smem_raw + m.range);
-    double* sFall = reinterpret_cast<double*>(smem_raw + m.Fall);  // every candidate's score, copied each generation
     int32_t* sElit = reinterpret_cast<int32_t*>(smem_raw + m.elit);
 
     const int32_t lo = me * rows_per_cta, hi = min(n, lo + rows_per_cta), mine = max(0, hi - lo);
@@ -2134,7 +2144,8 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         }
         const int4* src = reinterpret_cast<const int4*>(pop_io + (int64_t)lo * ld);
         for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) reinterpret_cast<int4*>(sPop[0])[i] = src[i];
-        for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) sF[0][i] = F_io[lo + i];
+        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) sFall[0][i] = F_io[i];  // every CTA takes all scores
+        for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) sGc[0][i] = G_out[lo + i];
     }
     __syncthreads();
     cluster.sync();  // everybody's rows and scores are staged
@@ -2147,23 +2158,73 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
     const int32_t first_child = max(lo, elitism);
     const int32_t q_lo = (first_child - elitism + 1) >> 1;                    // first q with elitism + 2q >= first_child
     const int32_t q_hi = hi > elitism ? min(pairs, (hi - elitism + 1) >> 1) : 0;  // first q with elitism + 2q >= hi
-    const int32_t n_items = (elite_hi - elite_lo) + max(0, q_hi - q_lo);
-    const int32_t trips = (n_items + groups - 1) / groups;
+    // work items of a group: a pair of children, or (after the pairs, where the last trip usually has idle groups)
+    // the copy of this CTA's elite rows, which keep their scores and GPU counts: all of them in one item when the
+    // elites come from the lists (at most four), else one row per item
+    const int32_t n_pairs = max(0, q_hi - q_lo);
+    const int32_t elite_span = (elitism > 0 && elitism <= 4) ? 4 : 1;
+    const int32_t n_elite_items = (max(0, elite_hi - elite_lo) + elite_span - 1) / elite_span;
+    // the copies start at a warp of their own, so that no warp runs both kinds of item one after the other
+    // (where that does not cost a trip)
+    const int32_t groups_per_warp = gs < 32 ? 32 / gs : 1;
+    const int32_t aligned0 = (n_pairs + groups_per_warp - 1) / groups_per_warp * groups_per_warp;
+    const int32_t trips = (n_pairs + n_elite_items + groups - 1) / groups;
+    const int32_t elite_item0 = aligned0 + n_elite_items <= trips * groups ? aligned0 : n_pairs;
+    // the rows this CTA produces: its elite rows and both children of its pairs (the last odd child may be
+    // a neighbour's row); over the cluster these ranges cover every row exactly once
+    const int32_t made_elites = max(0, elite_hi - elite_lo);
+    const int32_t child_lo = elitism + 2 * q_lo, child_hi = q_hi > q_lo ? min(n, elitism + 2 * q_hi) : child_lo;
+    const int32_t made = made_elites + (child_hi - child_lo);
+    const bool lists = elitism > 0 && elitism <= 4;  // elites by merging lists of promising children
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     for (int32_t g = 0; g < generations; ++g) {
         const int cur = g & 1, nxt = cur ^ 1;
         const uint64_t gen = gen0 + (uint64_t)g;
         const uint32_t gen_lo = (uint32_t)gen;
         const uint32_t c3 = counter3(STREAM_MUT, gen), c3a = counter3(STREAM_SEL_A, gen), c3b = counter3(STREAM_SEL_B, gen);
-        // ---- every CTA takes a private copy of all scores, then finds the elites for itself ----
-        for (int32_t i = threadIdx.x; i < n; i += blockDim.x) {
-            sFall[i] = *cluster.map_shared_rank(sF[cur] + (i & rows_mask), (unsigned int)(i >> rows_shift));
-        }
-        __syncthreads();
-        if (elitism > 0 && elitism <= 4) {  // sorted lists in registers, one barrier
-            if (elitism <= 2) block_top_small<2, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
-            else block_top_small<4, 0, false, 512>(sFall, n, 0, elitism, s_top, s_warp);
-            __syncthreads();
+        // ---- every CTA finds the elites of the population in force for itself ----
+        const double* Fcur = sFall[cur];
+        if (lists) {
+            bool full = g == 0;  // nothing is known about a population that came from outside
+            if (threadIdx.x == 0) sCandCnt[nxt * 16 + me] = 0;  // this generation's own list
+            if (!full) {
+                if (warp == 0) {
+                    // rows 0..E-1 hold the old elites; a child enters only with a score above the old E-th best
+                    const int32_t cnt = lane < C ? sCandCnt[cur * 16 + lane] : 0;
+                    const bool over = __any_sync(0xFFFFFFFFu, cnt > kClusterCand);
+                    if (!__any_sync(0xFFFFFFFFu, cnt > 0)) {
+                        // no child beat the old elites: they stay, in their order, now as rows 0..E-1
+                        if (lane < elitism) {
+                            Rec q;
+                            q.key = score_key(Fcur[lane]);
+                            q.idx = lane;
+                            q.pad = 0;
+                            s_top[lane] = q;
+                        }
+                    } else if (!over) {
+                        TopList<4> top;
+                        top_list_clear(top);
+                        if (lane < elitism) top_list_insert(top, score_key(Fcur[lane]), lane);
+                        for (int32_t c = 0; c < cnt; ++c) {
+                            const Rec q = sCandIn[(cur * 16 + lane) * kClusterCand + c];
+                            top_list_insert(top, q.key, q.idx);
+                        }
+                        for (int32_t r = 0; r < elitism; ++r) {
+                            const Rec best = warp_pop_best(top);
+                            if (lane == 0) s_top[r] = best;
+                        }
+                    }
+                    if (lane == 0) s_full = over;
+                }
+                __syncthreads();
+                full = s_full != 0;
+            }
+            if (full) {  // sorted lists in registers over all scores, one barrier
+                if (elitism <= 2) block_top_small<2, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
+                else block_top_small<4, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
+                __syncthreads();
+            }
             if ((int32_t)threadIdx.x < elitism) {
                 sElit[threadIdx.x] = s_top[threadIdx.x].idx;
                 if (me == 0) elites_out[threadIdx.x] = s_top[threadIdx.x].idx;
@@ -2174,7 +2235,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             prev.idx = -1;
             prev.pad = 0;
             for (int32_t r = 0; r < elitism; ++r) {
-                Rec best = block_next_best<0>(sFall, n, 0, r > 0, prev, s_warp);
+                Rec best = block_next_best<0>(Fcur, n, 0, r > 0, prev, s_warp);
                 if (threadIdx.x == 0) {
                     sElit[r] = best.idx;
                     if (me == 0) elites_out[r] = best.idx;
@@ -2186,18 +2247,29 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         // ---- children ----
         for (int32_t trip = 0; trip < trips; ++trip) {
             const int32_t item = trip * groups + gi;
-            const bool live = item < n_items;
-            const bool is_elite = live && item < elite_hi - elite_lo;
+            const bool is_elite = item >= elite_item0 && item < elite_item0 + n_elite_items;
+            const bool live = item < n_pairs || is_elite;
             int32_t pa = 0, pb = 0, slot0 = 0, slot1 = 0;
             bool has1 = false;
             uint32_t thr = 0u;
             if (is_elite) {
-                slot0 = elite_lo + item;
-                pa = pb = elitism <= 4 ? s_top[slot0].idx : sElit[slot0];
+                const int32_t ea = elite_lo + (item - elite_item0) * elite_span, eb = min(elite_hi, ea + elite_span);
+                for (int32_t r = ea; r < eb; ++r) {  // rows of this CTA
+                    const int32_t idx = elitism <= 4 ? s_top[r].idx : sElit[r];
+                    const int4* A = reinterpret_cast<const int4*>(cluster.map_shared_rank(
+                        sPop[cur] + (int64_t)(idx & rows_mask) * ld, (unsigned int)(idx >> rows_shift)));
+                    int4* Cd = reinterpret_cast<int4*>(sPop[nxt] + (int64_t)(r & rows_mask) * ld);
+                    for (int32_t v = gl; v < nvec; v += gs) Cd[v] = A[v];
+                    if (gl == 0) {
+                        sFall[nxt][r] = Fcur[idx];
+                        sGc[nxt][r & rows_mask] = *cluster.map_shared_rank(sGc[cur] + (idx & rows_mask), (unsigned int)(idx >> rows_shift));
+                    }
+                }
             } else if (live) {
-                const int32_t q = q_lo + (item - (elite_hi - elite_lo));
-                // both tournaments, every lane of the group for itself (same draws, same winner)
-                for (int which = 0; which < 2; ++which) {
+                const int32_t q = q_lo + item;
+                // the two tournaments: the lower half of the group's lanes runs the first parent's, the upper half
+                // the second's (a group of one lane runs both), every lane for itself (same draws, same winner)
+                for (int which = gs > 1 ? (gl >= (gs >> 1) ? 1 : 0) : 0; which < 2; ++which) {
                     int32_t win = -1;
                     double fwin = 0.0;
                     for (int32_t t0 = 0; t0 < tournament; t0 += 4) {
@@ -2207,7 +2279,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                         for (int u = 0; u < 4; ++u) {
                             if (t0 + u < tournament) {
                                 const int32_t idx = (int32_t)__umulhi(w[u], (uint32_t)n);
-                                const double f = sFall[idx];
+                                const double f = Fcur[idx];
                                 if (win < 0 || f > fwin || (f == fwin && idx < win)) {
                                     win = idx;
                                     fwin = f;
@@ -2216,19 +2288,29 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                         }
                     }
                     if (which) pb = win; else pa = win;
+                    if (gs > 1) break;
                 }
                 slot0 = elitism + 2 * q;
                 slot1 = slot0 + 1;
                 has1 = slot1 < n;
                 thr = thr32;
-                if (gl == 0) {
-                    parents_out[2 * q] = pa;
-                    parents_out[2 * q + 1] = pb;
+            }
+            if (gs > 1) {  // each half of a group learns the other half's winner (all lanes of the warp take part)
+                const int first = lane & ~(gs - 1);
+                const int32_t wa = __shfl_sync(0xFFFFFFFFu, pa, first), wb = __shfl_sync(0xFFFFFFFFu, pb, first + (gs >> 1));
+                if (live && !is_elite) {
+                    pa = wa;
+                    pb = wb;
                 }
+            }
+            if (live && !is_elite && gl == 0) {
+                const int32_t q = (slot0 - elitism) >> 1;
+                parents_out[2 * q] = pa;
+                parents_out[2 * q + 1] = pb;
             }
             double sum0 = 0.0, sum1 = 0.0;
             int32_t gp0 = 0, gp1 = 0;
-            if (live) {
+            if (live && !is_elite) {
                 const int32_t oa = pa >> rows_shift, ob = pb >> rows_shift;
                 const int4* A = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pa & rows_mask) * ld, (unsigned int)oa));
                 const int4* B = reinterpret_cast<const int4*>(cluster.map_shared_rank(sPop[cur] + (int64_t)(pb & rows_mask) * ld, (unsigned int)ob));
@@ -2237,12 +2319,10 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                 int4* C1 = reinterpret_cast<int4*>(cluster.map_shared_rank(sPop[nxt] + (int64_t)((has1 ? slot1 : slot0) & rows_mask) * ld, (unsigned int)o1));
                 for (int32_t v = gl; v < nvec; v += gs) {
                     const int4 a = A[v], b = B[v];
-                    int4 c0 = a, c1 = b;
-                    if (!is_elite) {
-                        const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
-                        if (ALWAYS) sibling_int4<true>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
-                        else sibling_int4<false>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
-                    }
+                    int4 c0, c1;
+                    const uint4 W = philox((uint32_t)v, (uint32_t)slot0, gen_lo, c3, keys);
+                    if (ALWAYS) sibling_int4<true>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
+                    else sibling_int4<false>(W, a, b, sKmin[v], sRange[v], thr, has1, c0, c1);
                     C0[v] = c0;
                     const int32_t base = (v >> 5) * 128 + (v & 31);
                     score4(c0, base, kcap, jpad, sX, sG, sum0, gp0);
@@ -2259,30 +2339,59 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                 sum1 = __dadd_rn(sum1, __shfl_xor_sync(0xFFFFFFFFu, sum1, off));
                 gp1 += __shfl_xor_sync(0xFFFFFFFFu, gp1, off);
             }
-            if (live && gl == 0) {
-                const int32_t o0 = slot0 >> rows_shift;
-                const int32_t over0 = gp0 > capacity ? gp0 - capacity : 0;
-                *cluster.map_shared_rank(sF[nxt] + (slot0 & rows_mask), (unsigned int)o0) =
-                    __dsub_rn(sum0, __dmul_rn(penalty, (double)over0));
-                *cluster.map_shared_rank(sGc + (slot0 & rows_mask), (unsigned int)o0) = gp0;
-                if (has1) {
-                    const int32_t o1 = slot1 >> rows_shift;
-                    const int32_t over1 = gp1 > capacity ? gp1 - capacity : 0;
-                    *cluster.map_shared_rank(sF[nxt] + (slot1 & rows_mask), (unsigned int)o1) =
-                        __dsub_rn(sum1, __dmul_rn(penalty, (double)over1));
-                    *cluster.map_shared_rank(sGc + (slot1 & rows_mask), (unsigned int)o1) = gp1;
+            if (live && !is_elite && gl == 0) {
+                // scores go to this CTA's copy first (sent to the others below); a child that beats the old
+                // E-th best is listed for the next generation's elites
+                const unsigned long long bar = lists ? s_top[elitism - 1].key : ~0ull;
+                auto leave = [&](int32_t slot, double sum, int32_t gp) {
+                    const int32_t over = gp > capacity ? gp - capacity : 0;
+                    const double f = __dsub_rn(sum, __dmul_rn(penalty, (double)over));
+                    sFall[nxt][slot] = f;
+                    *cluster.map_shared_rank(sGc[nxt] + (slot & rows_mask), (unsigned int)(slot >> rows_shift)) = gp;
+                    const unsigned long long key = score_key(f);
+                    if (key > bar) {
+                        const int32_t c = atomicAdd(&sCandCnt[nxt * 16 + me], 1);
+                        if (c < kClusterCand) {
+                            Rec q;
+                            q.key = key;
+                            q.idx = slot;
+                            q.pad = 0;
+                            sCandIn[(nxt * 16 + me) * kClusterCand + c] = q;
+                        }
+                    }
+                };
+                leave(slot0, sum0, gp0);
+                if (has1) leave(slot1, sum1, gp1);
+            }
+        }
+        __syncthreads();  // this CTA's scores and list are complete
+        if (C > 1) {
+            // what this CTA produced, to every other CTA's copy of the scores (and its list, one lane per CTA)
+            double* Fnext = sFall[nxt];
+            for (int32_t i = threadIdx.x; i < made; i += blockDim.x) {
+                const int32_t slot = i < made_elites ? elite_lo + i : child_lo + (i - made_elites);
+                const double f = Fnext[slot];
+                for (int32_t r = 0; r < C; ++r)
+                    if (r != me) *cluster.map_shared_rank(Fnext + slot, (unsigned int)r) = f;
+            }
+            if (lists && warp == 1 && lane < C && lane != me) {
+                const int32_t cnt = sCandCnt[nxt * 16 + me];
+                *cluster.map_shared_rank(sCandCnt + nxt * 16 + me, (unsigned int)lane) = cnt;
+                for (int32_t c = 0; c < min(cnt, kClusterCand); ++c) {
+                    Rec* at = sCandIn + (nxt * 16 + me) * kClusterCand + c;
+                    *cluster.map_shared_rank(at, (unsigned int)lane) = *at;
                 }
             }
         }
-        cluster.sync();  // all children and their scores written, also those that landed in a neighbour
+        cluster.sync();  // all children, their scores and the lists are where they belong
     }
     // ---- write my rows back ----
     const int fin = generations & 1;
     int4* dst = reinterpret_cast<int4*>(pop_io + (int64_t)lo * ld);
     for (int32_t i = threadIdx.x; i < mine * nvec; i += blockDim.x) dst[i] = reinterpret_cast<const int4*>(sPop[fin])[i];
     for (int32_t i = threadIdx.x; i < mine; i += blockDim.x) {
-        F_io[lo + i] = sF[fin][i];
-        G_out[lo + i] = sGc[i];
+        F_io[lo + i] = sFall[fin][lo + i];
+        G_out[lo + i] = sGc[fin][i];
     }
 }
 
