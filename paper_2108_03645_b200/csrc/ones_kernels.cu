@@ -2185,10 +2185,27 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         const uint32_t c3 = counter3(STREAM_MUT, gen), c3a = counter3(STREAM_SEL_A, gen), c3b = counter3(STREAM_SEL_B, gen);
         // ---- every CTA finds the elites of the population in force for itself ----
         const double* Fcur = sFall[cur];
-        if (lists) {
+        // With lists, warp 0 merges while the other warps already run their tournaments; everybody meets in
+        // settle_elites() before the first thing that needs the elites (the end of the first trip).
+        auto settle_elites = [&]() {
             bool full = g == 0;  // nothing is known about a population that came from outside
-            if (threadIdx.x == 0) sCandCnt[nxt * 16 + me] = 0;  // this generation's own list
             if (!full) {
+                __syncthreads();
+                full = s_full != 0;
+            }
+            if (full) {  // sorted lists in registers over all scores, one barrier
+                if (elitism <= 2) block_top_small<2, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
+                else block_top_small<4, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
+                __syncthreads();
+            }
+            if ((int32_t)threadIdx.x < elitism) {
+                sElit[threadIdx.x] = s_top[threadIdx.x].idx;
+                if (me == 0) elites_out[threadIdx.x] = s_top[threadIdx.x].idx;
+            }
+        };
+        if (lists) {
+            if (threadIdx.x == 0) sCandCnt[nxt * 16 + me] = 0;  // this generation's own list
+            if (g > 0) {
                 if (warp == 0) {
                     // rows 0..E-1 hold the old elites; a child enters only with a score above the old E-th best
                     const int32_t cnt = lane < C ? sCandCnt[cur * 16 + lane] : 0;
@@ -2217,18 +2234,8 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                     }
                     if (lane == 0) s_full = over;
                 }
-                __syncthreads();
-                full = s_full != 0;
             }
-            if (full) {  // sorted lists in registers over all scores, one barrier
-                if (elitism <= 2) block_top_small<2, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
-                else block_top_small<4, 0, false, 512>(Fcur, n, 0, elitism, s_top, s_warp);
-                __syncthreads();
-            }
-            if ((int32_t)threadIdx.x < elitism) {
-                sElit[threadIdx.x] = s_top[threadIdx.x].idx;
-                if (me == 0) elites_out[threadIdx.x] = s_top[threadIdx.x].idx;
-            }
+            if (trips == 0) settle_elites();
         } else if (elitism > 0) {
             Rec prev;
             prev.key = 0;
@@ -2252,7 +2259,7 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
             int32_t pa = 0, pb = 0, slot0 = 0, slot1 = 0;
             bool has1 = false;
             uint32_t thr = 0u;
-            if (is_elite) {
+            auto copy_elites = [&]() {
                 const int32_t ea = elite_lo + (item - elite_item0) * elite_span, eb = min(elite_hi, ea + elite_span);
                 for (int32_t r = ea; r < eb; ++r) {  // rows of this CTA
                     const int32_t idx = elitism <= 4 ? s_top[r].idx : sElit[r];
@@ -2265,6 +2272,10 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                         sGc[nxt][r & rows_mask] = *cluster.map_shared_rank(sGc[cur] + (idx & rows_mask), (unsigned int)(idx >> rows_shift));
                     }
                 }
+            };
+            const bool late = lists && trip == 0;  // the elites are settled at the end of this trip
+            if (is_elite) {
+                if (!late) copy_elites();
             } else if (live) {
                 const int32_t q = q_lo + item;
                 // the two tournaments: the lower half of the group's lanes runs the first parent's, the upper half
@@ -2332,6 +2343,10 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
                     }
                 }
             }
+            if (late) {
+                settle_elites();
+                if (is_elite) copy_elites();
+            }
             // fixed-order sum over the group's lanes (partials of absent lanes are +0)
             for (int off = gs >> 1; off >= 1; off >>= 1) {
                 sum0 = __dadd_rn(sum0, __shfl_xor_sync(0xFFFFFFFFu, sum0, off));
@@ -2368,11 +2383,10 @@ k_evolve_cluster(int32_t* __restrict__ pop_io, int64_t ld, int32_t n, int32_t n_
         if (C > 1) {
             // what this CTA produced, to every other CTA's copy of the scores (and its list, one lane per CTA)
             double* Fnext = sFall[nxt];
-            for (int32_t i = threadIdx.x; i < made; i += blockDim.x) {
+            for (int32_t w = threadIdx.x; w < made * C; w += blockDim.x) {  // neighbouring lanes: neighbouring rows
+                const int32_t r = w / made, i = w - r * made;
                 const int32_t slot = i < made_elites ? elite_lo + i : child_lo + (i - made_elites);
-                const double f = Fnext[slot];
-                for (int32_t r = 0; r < C; ++r)
-                    if (r != me) *cluster.map_shared_rank(Fnext + slot, (unsigned int)r) = f;
+                if (r != me) *cluster.map_shared_rank(Fnext + slot, (unsigned int)r) = Fnext[slot];
             }
             if (lists && warp == 1 && lane < C && lane != me) {
                 const int32_t cnt = sCandCnt[nxt * 16 + me];
