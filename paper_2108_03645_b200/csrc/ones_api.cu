@@ -354,8 +354,10 @@ int rebuild_tables(ones_ctx* c, const ones_job* h_jobs, int32_t n_jobs, const in
     bool all_pow2 = true;
     for (int32_t j = 0; j < n_jobs; ++j) {
         kmax = h_jobs[j].kmax > kmax ? h_jobs[j].kmax : kmax;
+        const int64_t b0 = h_jobs[j].b0, m = h_jobs[j].max_per_gpu;
+        if ((b0 & (b0 - 1)) == 0 && (m & (m - 1)) == 0) continue;  // powers of two: so is every GPU count (no division)
         for (int32_t k = 0; k <= h_jobs[j].kmax && all_pow2; ++k) {
-            const int64_t b = (int64_t)h_jobs[j].b0 << k, m = h_jobs[j].max_per_gpu, g = (b + m - 1) / m;
+            const int64_t g = ((b0 << k) + m - 1) / m;
             all_pow2 = (g & (g - 1)) == 0;
         }
     }
