@@ -295,6 +295,54 @@ def test_evolve_non_power_of_two_gpu_counts(ones, flags):
             _same_state(g2, o2)
 
 
+@pytest.mark.parametrize("elitism", [0, 1, 2, 3, 4, 5, 7])
+@pytest.mark.parametrize("J,N", [(16, 32), (100, 1024), (8, 4096), (40, 2048), (14, 999)])
+def test_cluster_path_elites_over_many_generations(ones, J, N, elitism):
+    """Populations that run all generations of a call inside one cluster launch: there the elites of a new population
+    come from the old elites and the children that beat the old E-th best (lists of at most eight children per CTA
+    and generation), and elite rows are copied with their scores.  Several generations per call, every number of
+    elites on both sides of the four that the lists handle."""
+    w = inputs.custom(J, max(4, 2 * J), N, 3, seed=J + N + elitism, kmax=6, kmin_max=1, pinned=J // 6)
+    g, o = _pair(ones, w, elitism=elitism, tournament=3, p_mut=0.05)
+    g.randomize(2)
+    o.randomize(2)
+    for gens in (1, 6, 13):
+        g.evolve(gens, 5)
+        o.evolve(gens, 5)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+    bg, bo = g.best(True), o.best(True)
+    assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"] and bg["index"] == bo["index"]
+
+
+@pytest.mark.parametrize("elitism", [1, 2, 4])
+@pytest.mark.parametrize("J,N", [(16, 32), (100, 1024), (8, 4096)])
+def test_cluster_path_many_children_beat_the_elites(ones, J, N, elitism):
+    """Every candidate starts as the same row and genes are redrawn at a high rate: where the common row is not
+    already the best one, far more than eight children of a CTA beat the old elites from one generation to the next,
+    so the lists overflow and every CTA falls back to the search over all scores inside the launch (seen on the 8 x
+    4096 case with p_mut = 1 and on the 100 x 1024 case with p_mut = 0.3); later generations return to the lists."""
+    w = inputs.custom(J, max(4, 2 * J), N, 3, seed=J + N, kmax=6)
+    g, o = _pair(ones, w, elitism=elitism, tournament=2, p_mut=1.0)
+    rows = np.tile(w.jobs["kmin"].astype(np.int32), (N, 1))
+    g.set_population(rows)
+    o.set_population(rows)
+    for gens in (4, 3):
+        g.evolve(gens, 9)
+        o.evolve(gens, 9)
+        pg, eg = g.last_parents()
+        po, eo = o.last_parents()
+        assert (pg == po).all() and (eg == eo).all()
+        _same_state(g, o)
+    g2, o2 = _pair(ones, w, elitism=elitism, tournament=2, p_mut=0.3)   # some generations with lists, some without
+    for s_ in (g2, o2):
+        s_.set_population(rows)
+        s_.evolve(12, 3)
+    _same_state(g2, o2)
+
+
 def test_split_runs_and_determinism(ones):
     w = inputs.paper_scale()
     a, _ = _pair(ones, w)
