@@ -462,6 +462,29 @@ def test_truncation_pool_in_place_over_many_generations(ones, J, N):
     _same_state(h, o)
 
 
+def test_truncation_pool_in_place_large_pool(ones):
+    """A pool of 80000 rows (five rows per thread of the selection cluster, the 16-rows-per-thread build of the
+    kernel) used in place over several generations: the second and later generations read their parents through
+    the row map that the selection before them wrote."""
+    J, N = 260, 20000
+    w = inputs.custom(J, 2 * J, N, 4, seed=77, kmax=6, pinned=J // 6, kmin_max=2)
+    g = ones.Search(w.jobs, w.capacity, N, inputs.SearchParams(p_mut=0.03, flags=4))
+    h = ones.Search(w.jobs, w.capacity, N, inputs.SearchParams(p_mut=0.03, flags=12))
+    o = oracle.Search(w.jobs, w.capacity, N, p_mut=0.03, flags=4)
+    for s_ in (g, o, h):
+        s_.randomize(3)
+    for gens in (1, 3, 2):
+        for s_ in (g, o, h):
+            s_.evolve(gens, 8)
+        pg, _ = g.last_parents()
+        po, _ = o.last_parents()
+        assert (pg == po).all()
+        bg, bo = g.best(False), o.best(False)   # read through the map
+        assert (bg["genome"] == bo["genome"]).all() and bg["fitness"] == bo["fitness"] and bg["index"] == bo["index"]
+        _same_state(g, o)
+        _same_state(h, o)
+
+
 def test_truncation_selection_with_many_ties(ones):
     # identical candidates: every score ties, survivors are decided by row order alone
     w = inputs.tiny()
