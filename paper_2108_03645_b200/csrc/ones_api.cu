@@ -956,10 +956,12 @@ int ones_update_jobs(ones_ctx* c, const ones_job* jobs, int32_t n_jobs, const in
                                       c->tab.jpad, c->stream));
         CU(c, launch_refresh_per_gpu(c->pop(c->cur), c->ld, c->N, c->W, old_J, n_jobs, c->tab, c->fit(), c->remap(n_jobs),
                                      c->refresh_inv(), c->refresh_cum(), c->stream));
-        CU(c, launch_reorder(c->pop(c->cur), c->ld, c->N, c->W, n_jobs, c->stream));
+        // "Reorder" of the refreshed rows, scored under the new tables in the same pass
+        CU(c, launch_reorder_score(c->pop(c->cur), c->ld, c->N, c->W, n_jobs, c->tab, c->fit(), c->narrow, c->F(), c->G(),
+                                   c->stream));
         c->launches += 4;
         c->J = n_jobs;
-        c->f_valid = false;
+        c->f_valid = true;
         c->elites_valid = false;
         return ONES_OK;
     }

@@ -3934,6 +3934,140 @@ __device__ void block_sort_service_order(double* __restrict__ key, int32_t* __re
     __syncthreads();
 }
 
+// Step (4) needs the order of service only as far as the idle GPUs reach: every job that is served takes at
+// least one GPU, so the first `need` = min(idle GPUs, jobs below their limit) records of the order are enough.
+// This finds the key of the need-th record by an eight-pass radix search over the gains (records in registers,
+// 256-bin histograms in shared memory), moves the records at or above it (all ties included: still a prefix
+// of the order) to the front of key[] / who[], pads to a power of two and sorts only those.  Returns the
+// length sorted, or 0 when more than kServeMax records would have to be sorted (the caller then sorts all).
+// hist: 256 + 2 words of shared memory; records beyond n_jobs carry gain -inf and are never selected.
+constexpr int32_t kServeMax = 1024;
+#ifndef ONES_SERVE_PASSES
+#define ONES_SERVE_PASSES 2
+#endif
+
+template <int PER>
+__device__ int32_t block_select_service_prefix(double* __restrict__ key, int32_t* __restrict__ who, int32_t need,
+                                               unsigned int* __restrict__ hist, int32_t* __restrict__ s_warp) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long k[PER];
+    double g[PER];
+    int32_t w[PER];
+#pragma unroll
+    for (int r = 0; r < PER; ++r) {  // record r of thread t: r * 256 + t (neighbouring lanes, neighbouring words)
+        g[r] = key[r * 256 + tid];
+        w[r] = who[r * 256 + tid];
+        // the search runs on the gain rounded down to fp32 (a monotone map: the records kept are still a prefix
+        // of the order, with a few more ties) and stops after ONES_SERVE_PASSES digits of that key
+        const uint32_t fb = __float_as_uint(__double2float_rd(g[r]) + 0.0f);
+        const uint32_t fk = g[r] != g[r] ? 0u : ((fb >> 31) ? ~fb : (fb | 0x80000000u));
+        k[r] = (unsigned long long)fk << 32;
+    }
+    unsigned long long prefix = 0ull;
+    int32_t remaining = need;
+    unsigned int alive = (1u << PER) - 1u;
+    for (int pass = 0; pass < ONES_SERVE_PASSES; ++pass) {
+        hist[tid] = 0u;
+        __syncthreads();
+        const int shift = 56 - 8 * pass;
+        const unsigned long long mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+            if (((alive >> r) & 1u) && (k[r] & mask) == prefix) atomicAdd(&hist[(unsigned int)(k[r] >> shift) & 255u], 1u);
+            else alive &= ~(1u << r);
+        }
+        __syncthreads();
+        if (warp == 0) {  // the digit that holds the remaining-th largest key, bins taken from 255 downwards
+            unsigned int c[8], mine = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                c[i] = hist[255 - (8 * lane + i)];
+                mine += c[i];
+            }
+            unsigned int incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned int a = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += a;
+            }
+            const unsigned int reached = __ballot_sync(0xFFFFFFFFu, (int32_t)incl >= remaining);
+            const int owner = reached ? __ffs(reached) - 1 : 31;
+            if (lane == owner) {
+                int32_t above = (int32_t)(incl - mine), d = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int32_t bin = 255 - (8 * lane + i);
+                    if (bin == 0 || above + (int32_t)c[i] >= remaining) {
+                        d = bin;
+                        break;
+                    }
+                    above += (int32_t)c[i];
+                }
+                hist[256] = (unsigned int)d;
+                hist[257] = (unsigned int)(remaining - above);
+            }
+        }
+        __syncthreads();
+        prefix |= (unsigned long long)hist[256] << shift;
+        remaining = (int32_t)hist[257];
+        __syncthreads();  // hist[256..257] are rewritten by the next pass
+    }
+    // prefix = key of the need-th record of the order: every record at or above it is kept
+    int32_t mine = 0;
+#pragma unroll
+    for (int r = 0; r < PER; ++r) mine += k[r] >= prefix;
+    int32_t incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();  // also: every thread holds its records in registers, key[] and who[] may be rewritten
+    int32_t at = incl - mine, total = 0;
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+        const int32_t c = s_warp[v];
+        if (v < warp) at += c;
+        total += c;
+    }
+    if (total > kServeMax) return 0;  // block-uniform
+    int32_t m2 = 2;
+    while (m2 < total) m2 <<= 1;
+#pragma unroll
+    for (int r = 0; r < PER; ++r)
+        if (k[r] >= prefix) {
+            key[at] = g[r];
+            who[at] = w[r];
+            ++at;
+        }
+    for (int32_t i = total + tid; i < m2; i += 256) {
+        key[i] = -CUDART_INF;
+        who[i] = 0x40000000 + i;
+    }
+    __syncthreads();
+    if (m2 == 1024) {
+        block_sort_service_order<4>(key, who);
+    } else if (m2 == 512) {
+        block_sort_service_order<2>(key, who);
+    } else {  // at most 256 records, one per thread, every step through shared memory
+        for (int32_t kk = 2; kk <= m2; kk <<= 1)
+            for (int32_t d = kk >> 1; d > 0; d >>= 1) {
+                const int32_t s = tid, p = tid ^ d;
+                if (s < m2 && p > s) {
+                    const double ka = key[s], kb = key[p];
+                    const int32_t ja = who[s], jb = who[p];
+                    if (served_first(kb, jb, ka, ja) == ((s & kk) == 0)) {
+                        key[s] = kb; key[p] = ka;
+                        who[s] = jb; who[p] = ja;
+                    }
+                }
+                __syncthreads();
+            }
+    }
+    return m2;
+}
+
 // Once per job-set change: inv[old id] = the new id of a surviving job (the highest, should several claim
 // one old job) or -1, and newcum[j] = the GPUs that the new jobs before j need for their smallest batch
 // (newcum[n_jobs] = all of them), capped at the cluster's size: needs beyond it can never be met.
@@ -4124,7 +4258,19 @@ k_refresh_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_
                 sj[s] = who;
             }
             __syncthreads();
-            if (j2 == 512) block_sort_service_order<2>(key, sj);
+            // only as much of the order as the idle GPUs can reach (every served job takes at least one)
+            int32_t len = 0;
+            if (j2 >= 512 && j2 <= 4096) {
+                const int32_t need = min(n_idle - U, j2);
+                unsigned int* hist = reinterpret_cast<unsigned int*>(cum);  // free until the prefix sums below
+                if (j2 == 512) len = block_select_service_prefix<2>(key, sj, need, hist, s_warp);
+                else if (j2 == 1024) len = block_select_service_prefix<4>(key, sj, need, hist, s_warp);
+                else if (j2 == 2048) len = block_select_service_prefix<8>(key, sj, need, hist, s_warp);
+                else len = block_select_service_prefix<16>(key, sj, need, hist, s_warp);
+            }
+            if (len > 0) {
+                // sorted already
+            } else if (j2 == 512) block_sort_service_order<2>(key, sj);
             else if (j2 == 1024) block_sort_service_order<4>(key, sj);
             else if (j2 == 2048) block_sort_service_order<8>(key, sj);
             else if (j2 == 4096) block_sort_service_order<16>(key, sj);
@@ -4145,16 +4291,17 @@ k_refresh_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_
                         }
                         __syncthreads();
                     }
-            for (int32_t s = tid; s < j2; s += 256) {
+            if (len == 0) len = j2;
+            for (int32_t s = tid; s < len; s += 256) {
                 const int32_t j = sj[s];
                 cum[s] = j < n_jobs ? min(lim[j] - count[j], n_gpus) : 0;
             }
             __syncthreads();
-            const int32_t wanted = block_scan_excl(cum, j2, s_warp);
+            const int32_t wanted = block_scan_excl(cum, len, s_warp);
             for (int32_t i = tid; i < n_gpus; i += 256) {
                 if (row[i] < 0) {
                     const int32_t r = rk[i] - U;
-                    if (r >= 0 && r < wanted) row[i] = sj[last_at_most(cum, j2, r)];
+                    if (r >= 0 && r < wanted) row[i] = sj[last_at_most(cum, len, r)];
                 }
             }
             __syncthreads();
