@@ -4243,19 +4243,34 @@ k_refresh_per_gpu(int32_t* __restrict__ slots, int64_t ld, int32_t n, int32_t n_
         __syncthreads();
         // (4) refill what is still idle (block-uniform condition)
         if (n_idle > U) {
-            for (int32_t s = tid; s < j2; s += 256) {
-                double gain = -CUDART_INF;
-                int32_t who = 0x40000000 + s;
-                if (s < n_jobs && count[s] < lim[s]) {
-                    const int32_t at = slot_of(s);
-                    const int4 q = __ldg(fit + at);
-                    const int32_t k = count[s] > 0 ? exponent_that_fits(q.x, q.y, q.z, q.w, count[s]) : -1;
-                    const double now = k >= 0 ? t.X[(int64_t)k * t.jpad + at] : 0.0;
-                    gain = __dsub_rn(t.X[(int64_t)q.w * t.jpad + at], now);
-                    who = s;
+            for (int32_t s0 = tid; s0 < j2; s0 += 4 * 256) {
+                // four jobs per step, each kind of load issued for all four before the next kind
+                int4 q[4];
+                int32_t at[4], have[4];
+                bool cand[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int32_t s = s0 + 256 * u;
+                    cand[u] = s < n_jobs && count[s] < lim[s];
+                    at[u] = slot_of(cand[u] ? s : 0);
+                    have[u] = cand[u] ? count[s] : 0;
+                    q[u] = cand[u] ? __ldg(fit + at[u]) : make_int4(1, 1, 0, 0);
                 }
-                key[s] = gain;
-                sj[s] = who;
+                double now[4], top[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int32_t k = (cand[u] && have[u] > 0) ? exponent_that_fits(q[u].x, q[u].y, q[u].z, q[u].w, have[u]) : -1;
+                    now[u] = k >= 0 ? __ldg(t.X + (int64_t)k * t.jpad + at[u]) : 0.0;
+                    top[u] = cand[u] ? __ldg(t.X + (int64_t)q[u].w * t.jpad + at[u]) : 0.0;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int32_t s = s0 + 256 * u;
+                    if (s < j2) {
+                        key[s] = cand[u] ? __dsub_rn(top[u], now[u]) : -CUDART_INF;
+                        sj[s] = cand[u] ? s : 0x40000000 + s;
+                    }
+                }
             }
             __syncthreads();
             // only as much of the order as the idle GPUs can reach (every served job takes at least one)
