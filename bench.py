@@ -313,13 +313,13 @@ def sha16(path: str) -> str:
 # captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
 # traffic as null whenever the file it runs differs from it.
 NCU_TRAFFIC = {
-    "captured_at": "299f447",
-    "source_sha16": "384a01d62f12b3f1",
+    "captured_at": "2810ec6",
+    "source_sha16": "cc88bdaf2718359c",
     "bytes_per_launch": {
-        ("large", 65536, "k_evolve_score"): 379.9e6 + 481.4e6,
-        ("large", 65536, "k_evolve"): 375.8e6 + 479.2e6,
+        ("large", 65536, "k_evolve_score"): 379.4e6 + 481.2e6,
+        ("large", 65536, "k_evolve"): 375.3e6 + 479.2e6,
         ("large", 65536, "k_fitness"): 537.1e6 + 0.7e6,
-        ("large", 65536, "k_evolve_score_packed"): 45.3e6 + 73.6e6,
+        ("large", 65536, "k_evolve_score_packed"): 45.3e6 + 73.7e6,
         ("large", 65536, "k_fitness_packed"): 134.5e6 + 0.3e6,
     },
 }
