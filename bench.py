@@ -302,19 +302,43 @@ def small_workload_figures(binding, name: str, min_s: float = 0.25):
             "timed_calls": len(ms), "hbm": "n/a (population resident in L2 or shared memory)"}
 
 
+# The functions whose source the traffic figures below belong to: the five timed kernels and the device
+# functions they call.  Their text (definition line to closing brace) is hashed, so that an edit elsewhere in the
+# kernel file does not orphan the capture and an edit to any of them does.
+TRAFFIC_FUNCTIONS = ("philox", "draw_gene", "slot_of", "sibling_gene", "sibling_int4", "ld_row", "ld_row_hint",
+                     "l2_policy_evict_last", "l2_prefetch", "score4", "k_fitness", "k_fitness_packed", "k_evolve",
+                     "mutate_gene", "sibling_pair", "score_int4", "k_evolve_score", "mutate_byte", "score_gene",
+                     "score_word", "k_evolve_score_packed", "launch_evolve_score", "launch_evolve_score_packed",
+                     "launch_evolve", "launch_fitness", "launch_fitness_packed")
+
+
 def sha16(path: str) -> str:
+    """Hash of the source text of TRAFFIC_FUNCTIONS in `path`; raises when one of them cannot be found."""
     import hashlib
-    with open(path, "rb") as fh:
-        return hashlib.sha256(fh.read()).hexdigest()[:16]
+    import re
+    with open(path, "r", encoding="utf-8") as fh:
+        text = fh.read()
+    h = hashlib.sha256()
+    for name in TRAFFIC_FUNCTIONS:
+        # a definition: the name at the start of a line or after the return type, followed by its parameter list
+        # and, later, a brace at the start of a line that closes it
+        m = re.search(r"^(?:[^\n;{}()]*[ \*&])?" + re.escape(name) + r"\(", text, flags=re.M)
+        if not m:
+            raise OSError(f"{name}: definition not found")
+        end = text.find("\n}\n", m.start())
+        if end < 0:
+            raise OSError(f"{name}: end not found")
+        h.update(text[m.start():end + 3].encode())
+    return h.hexdigest()[:16]
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of this
-# benchmark's default workload at its full population.  A figure belongs to the kernel source it was
-# captured on: `source_sha16` is the hash of the kernel file at that commit, and the benchmark reports
-# traffic as null whenever the file it runs differs from it.
+# benchmark's default workload at its full population.  A figure belongs to the source it was captured on:
+# `source_sha16` is sha16() of the kernel file at commit `captured_at` (the timed kernels, their device functions
+# and their launchers), and the benchmark reports traffic as null whenever the file it runs gives another hash.
 NCU_TRAFFIC = {
     "captured_at": "2810ec6",
-    "source_sha16": "cc88bdaf2718359c",
+    "source_sha16": "3a974a5302ea4351",
     "bytes_per_launch": {
         ("large", 65536, "k_evolve_score"): 379.4e6 + 481.2e6,
         ("large", 65536, "k_evolve"): 375.3e6 + 479.2e6,
