@@ -375,6 +375,35 @@ def test_checkpoint_and_resume(ones):
     _same_state(b, o)
 
 
+@pytest.mark.parametrize("flags,J,N", [(4, 130, 700), (4, 260, 20000), (0, 16, 32), (0, 8, 4096)])
+def test_checkpoint_and_resume_of_mapped_and_cluster_states(ones, flags, J, N):
+    """Saving and resuming where the handle keeps state of its own between generations: the truncation scheme's pool
+    used in place (the saved population is the ordered one) and the cluster path (a resumed call starts without the
+    lists of promising children).  Also: a change of the generation counter between two calls."""
+    w = inputs.custom(J, 2 * J, N, 3, seed=J + N, kmax=6, pinned=J // 6)
+    a, o = _pair(ones, w, flags=flags, p_mut=0.05)
+    a.randomize(3)
+    o.randomize(3)
+    a.evolve(4, 3)
+    a.evolve(3, 3)
+    o.evolve(12, 3)
+    saved, gen = a.get_population(), a.generation
+    b, _ = _pair(ones, w, flags=flags, p_mut=0.05)
+    b.set_population(saved)
+    b.set_generation(gen)
+    b.evolve(5, 3)
+    assert b.generation == 12
+    _same_state(b, o)
+    a.set_generation(gen)      # the first handle goes on from its own (mapped) state as well
+    a.evolve(5, 3)
+    _same_state(a, o)
+    a.set_generation(3)        # back in time: the draws of generations 3 and 4 on the current population
+    o.set_generation(3)
+    a.evolve(2, 3)
+    o.evolve(2, 3)
+    _same_state(a, o)
+
+
 def test_set_get_population_roundtrip(ones):
     w = inputs.custom(30, 64, 50, 1, seed=1)
     g, o = _pair(ones, w)
